@@ -1,0 +1,120 @@
+"""TEST INFRASTRUCTURE -- ctypes access to the CPU oracle (``atrex_oracle.cpp``).
+
+Only ``tests/``, ``__graft_entry__.smoke()`` and ``bench.py``'s CPU-baseline legs may import
+this package.  The product package never does, and this package never imports the product.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "atrex_oracle.cpp")
+_LIB = os.path.join(_HERE, "libatrex_oracle.so")
+
+ENTRY_DTYPE = np.dtype([("key", "<u8"), ("count", "<u8"), ("wt_lo", "<u8"), ("wt_hi", "<u8"),
+                        ("phase_weight", "<f8"), ("roofline_s", "<f8")])
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no fast-math, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["g++", "-O2", "-ffp-contract=off", "-std=c++17", "-fPIC", "-shared",
+                               "-pthread", "-o", _LIB, _SRC])
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        L.oracle_create.restype = C.c_void_p
+        L.oracle_create.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32]
+        L.oracle_destroy.argtypes = [C.c_void_p]
+        L.oracle_reset.argtypes = [C.c_void_p]
+        L.oracle_ingest.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
+        L.oracle_ingest_threads.restype = C.c_uint32
+        L.oracle_ingest_threads.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32]
+        L.oracle_set_work.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
+        L.oracle_n_keys.restype = C.c_uint64
+        L.oracle_n_keys.argtypes = [C.c_void_p]
+        L.oracle_stats.argtypes = [C.c_void_p, C.c_void_p]
+        L.oracle_finalize.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
+        L.oracle_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p]
+        L.oracle_u128_to_f64.restype = C.c_double
+        L.oracle_u128_to_f64.argtypes = [C.c_uint64, C.c_uint64]
+        _lib = L
+    return _lib
+
+
+def _peaks_buf(peak_bw: float, peak_flops) -> np.ndarray:
+    pf = list(peak_flops) + [1.0] * (8 - len(peak_flops))
+    return np.array([peak_bw] + pf[:8], dtype=np.float64)
+
+
+class Oracle:
+    """Thin handle around the C++ oracle."""
+
+    def __init__(self, app_weights, n_phases: int):
+        w = np.ascontiguousarray(app_weights, dtype=np.uint32)
+        self._h = lib().oracle_create(w.ctypes.data, w.shape[0], n_phases)
+        if not self._h:
+            raise ValueError("oracle_create rejected its arguments")
+
+    def close(self):
+        if self._h:
+            lib().oracle_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def reset(self):
+        lib().oracle_reset(self._h)
+
+    def ingest(self, records: np.ndarray, threads: int = 1) -> int:
+        r = np.ascontiguousarray(records)
+        assert r.dtype.itemsize == 16
+        if threads == 1:
+            lib().oracle_ingest(self._h, r.ctypes.data, r.shape[0])
+            return 1
+        return lib().oracle_ingest_threads(self._h, r.ctypes.data, r.shape[0], threads)
+
+    def set_work(self, rows: np.ndarray) -> int:
+        r = np.ascontiguousarray(rows)
+        assert r.dtype.itemsize == 24
+        return lib().oracle_set_work(self._h, r.ctypes.data, r.shape[0])
+
+    def n_keys(self) -> int:
+        return lib().oracle_n_keys(self._h)
+
+    def stats(self) -> dict:
+        out = np.zeros(19, dtype=np.uint64)
+        lib().oracle_stats(self._h, out.ctypes.data)
+        totals = [int(out[3 + 2 * p]) | (int(out[4 + 2 * p]) << 64) for p in range(8)]
+        return {"n_valid": int(out[0]), "n_rejected": int(out[1]), "n_keys": int(out[2]), "totals": totals}
+
+    def finalize(self, peak_bw: float, peak_flops) -> np.ndarray:
+        n = self.n_keys()
+        out = np.zeros(n, dtype=ENTRY_DTYPE)
+        n_out = C.c_uint64(0)
+        pk = _peaks_buf(peak_bw, peak_flops)
+        rc = lib().oracle_finalize(self._h, pk.ctypes.data, out.ctypes.data, n, C.byref(n_out))
+        assert rc == 0 and n_out.value == n
+        return out
+
+    def topk(self, peak_bw: float, peak_flops, phase: int, k: int) -> np.ndarray:
+        out = np.zeros(max(k, 1), dtype=ENTRY_DTYPE)
+        n_out = C.c_uint32(0)
+        pk = _peaks_buf(peak_bw, peak_flops)
+        lib().oracle_topk(self._h, pk.ctypes.data, phase, k, out.ctypes.data, C.byref(n_out))
+        return out[:n_out.value].copy()
+
+
+def u128_to_f64(x: int) -> float:
+    return lib().oracle_u128_to_f64((x >> 64) & 0xFFFFFFFFFFFFFFFF, x & 0xFFFFFFFFFFFFFFFF)

@@ -1,0 +1,278 @@
+// TEST INFRASTRUCTURE -- not part of the product path.
+//
+// Plain, slow, obviously-correct CPU statement of what the trace-aggregation path
+// computes, written from the paper's definitions.  Only the test-suite, the smoke
+// check and the benchmark's CPU-baseline leg may call it.  It shares no source,
+// header, table or helper with the CUDA library; the structs below restate the byte
+// layouts of the buffers independently.
+//
+// What it computes, per distinct (operator, shape, phase) key k:
+//   count[k]  = number of valid records carrying k           (Eq. 2: the sum over the
+//                                                              m_{a,phi,r} invocations)
+//   wt[k]     = sum over those records of                    (Eq. 2's cumulative device
+//               app_weight[app] * duration_ns, exact u128     time D, each application's
+//                                                              time scaled by its card-hour
+//                                                              weight as in Eq. 3's p_a)
+//   T[phi]    = sum of wt[k] over keys of phase phi           (Eq. 2's per-phase total)
+//   phase_weight[k] = fl(fl(wt[k]) / fl(T[phi]))              (Eq. 3's normalisation so that
+//                                                              weights sum to 1, done
+//                                                              separately per serving phase)
+//   roofline_s[k]   = max(F/P_dtype, M/beta)                  (Eq. 1)
+//   topk(phi, k)    = first k keys of phase phi by (wt descending, key ascending)
+//                                                             (Table 2's ranking)
+//
+// Readings where the paper is silent: invalid records (application or phase out of
+// range) are skipped and counted; the `pad` byte is ignored; a phase whose total is zero
+// gives weight +0.0; a key without a work-table row gets the quiet-NaN pattern
+// 0x7FF8000000000000; ties in the ranking go to the smaller packed key; the ranking
+// compares the exact integer wt, not the rounded double.
+//
+// Floating point: u128 -> binary64 is one round-to-nearest-even conversion (the compiler
+// runtime's integer-to-double conversion), then IEEE division.  Build with
+// -O2 -ffp-contract=off and without -ffast-math.
+//
+// Every function here is pinned by tests/test_oracle_*.py against hand-computed traces,
+// closed forms, brute force in Python integers, and invariants.
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <map>
+#include <thread>
+#include <vector>
+
+typedef unsigned __int128 u128;
+
+namespace {
+
+struct Rec {
+    uint32_t app_id;
+    uint16_t op_id;
+    uint8_t phase;
+    uint8_t pad;
+    uint32_t shape_id;
+    uint32_t duration_ns;
+};
+static_assert(sizeof(Rec) == 16, "record is 16 bytes");
+
+struct WorkRow {
+    uint32_t shape_id;
+    uint16_t op_id;
+    uint16_t dtype;
+    uint64_t flops;
+    uint64_t bytes;
+};
+static_assert(sizeof(WorkRow) == 24, "work row is 24 bytes");
+
+struct Entry {
+    uint64_t key;
+    uint64_t count;
+    uint64_t wt_lo;
+    uint64_t wt_hi;
+    double phase_weight;
+    double roofline_s;
+};
+static_assert(sizeof(Entry) == 48, "entry is 48 bytes");
+
+struct Peaks {
+    double peak_bw;
+    double peak_flops[8];
+};
+
+struct Acc {
+    uint64_t count = 0;
+    u128 wt = 0;
+};
+
+typedef std::map<uint64_t, Acc> Groups;
+
+struct Oracle {
+    uint32_t n_apps = 0, n_phases = 0;
+    std::vector<uint32_t> app_weight;
+    Groups groups;
+    std::map<uint64_t, WorkRow> work;  // (op << 32 | shape) -> row
+    uint64_t n_valid = 0, n_rejected = 0;
+};
+
+inline uint64_t pack_key(const Rec& r) {
+    return ((uint64_t)r.phase << 48) | ((uint64_t)r.op_id << 32) | (uint64_t)r.shape_id;
+}
+
+// Eq. 2 restricted to a slice of the trace: group-by sum into `g`.
+void aggregate_slice(const Oracle& o, const Rec* recs, uint64_t n, Groups& g,
+                     uint64_t& n_valid, uint64_t& n_rejected) {
+    for (uint64_t i = 0; i < n; ++i) {
+        const Rec& r = recs[i];
+        if (r.app_id >= o.n_apps || r.phase >= o.n_phases) {
+            ++n_rejected;
+            continue;
+        }
+        Acc& a = g[pack_key(r)];
+        a.count += 1;
+        a.wt += (u128)o.app_weight[r.app_id] * (u128)r.duration_ns;
+        ++n_valid;
+    }
+}
+
+void phase_totals(const Oracle& o, u128 totals[8]) {
+    for (int p = 0; p < 8; ++p) totals[p] = 0;
+    for (const auto& kv : o.groups) totals[kv.first >> 48] += kv.second.wt;
+}
+
+double quiet_nan() {
+    uint64_t bits = 0x7FF8000000000000ull;
+    double d;
+    std::memcpy(&d, &bits, 8);
+    return d;
+}
+
+// Eq. 1 for one (operator, shape) unit.
+double roofline_time(const Oracle& o, const Peaks& pk, uint64_t key) {
+    auto it = o.work.find(key & 0x0000FFFFFFFFFFFFull);
+    if (it == o.work.end()) return quiet_nan();
+    const WorkRow& w = it->second;
+    double t_compute = (double)w.flops / pk.peak_flops[w.dtype];
+    double t_memory = (double)w.bytes / pk.peak_bw;
+    return std::fmax(t_compute, t_memory);
+}
+
+Entry make_entry(const Oracle& o, const Peaks& pk, const u128 totals[8], uint64_t key, const Acc& a) {
+    Entry e;
+    e.key = key;
+    e.count = a.count;
+    e.wt_lo = (uint64_t)a.wt;
+    e.wt_hi = (uint64_t)(a.wt >> 64);
+    u128 t = totals[key >> 48];
+    e.phase_weight = (t == 0) ? 0.0 : (double)a.wt / (double)t;  // Eq. 3, per phase
+    e.roofline_s = roofline_time(o, pk, key);
+    return e;
+}
+
+}  // namespace
+
+extern "C" {
+
+void* oracle_create(const uint32_t* app_weights, uint32_t n_apps, uint32_t n_phases) {
+    if (!app_weights || n_apps == 0 || n_phases == 0 || n_phases > 8) return nullptr;
+    Oracle* o = new Oracle;
+    o->n_apps = n_apps;
+    o->n_phases = n_phases;
+    o->app_weight.assign(app_weights, app_weights + n_apps);
+    return o;
+}
+
+void oracle_destroy(void* h) { delete (Oracle*)h; }
+
+void oracle_reset(void* h) {
+    Oracle* o = (Oracle*)h;
+    o->groups.clear();
+    o->n_valid = o->n_rejected = 0;
+}
+
+// Single-threaded ingest of n records.
+void oracle_ingest(void* h, const void* records, uint64_t n) {
+    Oracle* o = (Oracle*)h;
+    aggregate_slice(*o, (const Rec*)records, n, o->groups, o->n_valid, o->n_rejected);
+}
+
+// Threaded variant: thread t aggregates a contiguous slice into its own map; the maps
+// are merged by key with integer adds (identical by associativity).  Returns the number
+// of threads used.
+uint32_t oracle_ingest_threads(void* h, const void* records, uint64_t n, uint32_t threads) {
+    Oracle* o = (Oracle*)h;
+    if (threads == 0) threads = std::thread::hardware_concurrency();
+    if (threads == 0) threads = 1;
+    if (n < threads) threads = 1;
+    std::vector<Groups> parts(threads);
+    std::vector<uint64_t> nv(threads, 0), nr(threads, 0);
+    std::vector<std::thread> pool;
+    const Rec* recs = (const Rec*)records;
+    for (uint32_t t = 0; t < threads; ++t) {
+        uint64_t lo = n * t / threads, hi = n * (t + 1) / threads;
+        pool.emplace_back([&, t, lo, hi] { aggregate_slice(*o, recs + lo, hi - lo, parts[t], nv[t], nr[t]); });
+    }
+    for (auto& th : pool) th.join();
+    for (uint32_t t = 0; t < threads; ++t) {
+        for (const auto& kv : parts[t]) {
+            Acc& a = o->groups[kv.first];
+            a.count += kv.second.count;
+            a.wt += kv.second.wt;
+        }
+        o->n_valid += nv[t];
+        o->n_rejected += nr[t];
+    }
+    return threads;
+}
+
+// Install the per-(operator, shape) semantic work table.  Returns 0, or -1 on a
+// duplicate pair or a dtype index >= 8 (table left empty).
+int oracle_set_work(void* h, const void* rows, uint64_t n) {
+    Oracle* o = (Oracle*)h;
+    o->work.clear();
+    const WorkRow* w = (const WorkRow*)rows;
+    for (uint64_t i = 0; i < n; ++i) {
+        uint64_t k = ((uint64_t)w[i].op_id << 32) | w[i].shape_id;
+        if (w[i].dtype >= 8 || !o->work.emplace(k, w[i]).second) {
+            o->work.clear();
+            return -1;
+        }
+    }
+    return 0;
+}
+
+uint64_t oracle_n_keys(void* h) { return ((Oracle*)h)->groups.size(); }
+
+// out[0] = valid records, out[1] = rejected records, out[2] = distinct keys,
+// out[3 + 2p], out[4 + 2p] = low and high 64 bits of T[p] for p in 0..7.
+void oracle_stats(void* h, uint64_t out[19]) {
+    Oracle* o = (Oracle*)h;
+    u128 totals[8];
+    phase_totals(*o, totals);
+    out[0] = o->n_valid;
+    out[1] = o->n_rejected;
+    out[2] = o->groups.size();
+    for (int p = 0; p < 8; ++p) {
+        out[3 + 2 * p] = (uint64_t)totals[p];
+        out[4 + 2 * p] = (uint64_t)(totals[p] >> 64);
+    }
+}
+
+// All entries, key ascending.  Returns 0, or -1 if cap is too small (*n_out = needed).
+int oracle_finalize(void* h, const void* peaks, void* out, uint64_t cap, uint64_t* n_out) {
+    Oracle* o = (Oracle*)h;
+    const Peaks& pk = *(const Peaks*)peaks;
+    *n_out = o->groups.size();
+    if (cap < o->groups.size()) return -1;
+    u128 totals[8];
+    phase_totals(*o, totals);
+    Entry* e = (Entry*)out;
+    uint64_t i = 0;
+    for (const auto& kv : o->groups) e[i++] = make_entry(*o, pk, totals, kv.first, kv.second);
+    return 0;
+}
+
+// The first min(k, n_phase) entries of `phase` ordered by (wt descending, key ascending).
+int oracle_topk(void* h, const void* peaks, uint32_t phase, uint32_t k, void* out, uint32_t* n_out) {
+    Oracle* o = (Oracle*)h;
+    const Peaks& pk = *(const Peaks*)peaks;
+    u128 totals[8];
+    phase_totals(*o, totals);
+    std::vector<std::pair<uint64_t, Acc>> v;
+    for (const auto& kv : o->groups)
+        if ((kv.first >> 48) == phase) v.push_back(kv);
+    std::sort(v.begin(), v.end(), [](const std::pair<uint64_t, Acc>& a, const std::pair<uint64_t, Acc>& b) {
+        if (a.second.wt != b.second.wt) return a.second.wt > b.second.wt;
+        return a.first < b.first;
+    });
+    uint32_t m = (uint32_t)std::min<uint64_t>(k, v.size());
+    Entry* e = (Entry*)out;
+    for (uint32_t i = 0; i < m; ++i) e[i] = make_entry(*o, pk, totals, v[i].first, v[i].second);
+    *n_out = m;
+    return 0;
+}
+
+// The integer -> binary64 conversion used above, exposed so tests can pin its rounding.
+double oracle_u128_to_f64(uint64_t hi, uint64_t lo) { return (double)(((u128)hi << 64) | lo); }
+
+}  // extern "C"

@@ -1,0 +1,285 @@
+"""Pins for the CPU oracle: hand-computed traces, closed forms, brute force, invariants.
+
+Each test is chosen so that a plausible slip in the oracle (a dropped weight, a swapped
+operand, a wrong shift in the key, a per-trace instead of per-phase normaliser, a double
+rounding) makes it fail.  None of them calls the CUDA path.
+"""
+from fractions import Fraction
+import math
+import random
+import struct
+
+import numpy as np
+import pytest
+
+import oracle
+import tracegen as tg
+from tracegen.configs import make_spec
+from tracegen.layout import RECORD_DTYPE, WORK_DTYPE
+from tests.helpers import (load_golden, f64_bits, records_from_dicts, work_from_dicts, brute_force,
+                           expected_entry_fields, check_entries_against, entry_wt, sorted_by_key)
+
+PEAK_BW = 8.0e12
+PEAK_FLOPS = [1.0e15, 2.0e15, 4.0e15, 5.0e14, 2.5e14, 1.0e15, 1.0e15, 1.0e15]
+
+
+def run_oracle(records, app_weights, n_phases, work=None, threads=1, peak_bw=PEAK_BW, peak_flops=PEAK_FLOPS):
+    o = oracle.Oracle(app_weights, n_phases)
+    if work is not None:
+        assert o.set_work(work) == 0
+    o.ingest(records, threads=threads)
+    return o, o.finalize(peak_bw, peak_flops)
+
+
+# ---------------------------------------------------------------- hand-computed traces
+
+def test_worked_example_a(golden_dir):
+    g = load_golden(golden_dir, "worked_example_a.json")
+    recs = records_from_dicts(g["records"])
+    work = work_from_dicts(g["work"])
+    o, ent = run_oracle(recs, g["app_weights"], g["n_phases"], work, peak_bw=g["peak_bw"], peak_flops=g["peak_flops"])
+    assert len(ent) == len(g["expected"])
+    for e, x in zip(ent, g["expected"]):  # finalize is key-ascending, so is the fixture
+        assert int(e["key"]) == int(x["key"], 16)
+        assert int(e["count"]) == x["count"]
+        assert entry_wt(e) == x["wt"]
+        assert f64_bits(float(e["phase_weight"])) == int(x["phase_weight_bits"], 16)
+        assert f64_bits(float(e["roofline_s"])) == int(x["roofline_bits"], 16)
+    st = o.stats()
+    assert st["n_valid"] == 7 and st["n_rejected"] == 0 and st["n_keys"] == 4
+    assert st["totals"][0] == g["phase_totals"]["0"] and st["totals"][1] == g["phase_totals"]["1"]
+    for t in g["topk"]:
+        top = o.topk(g["peak_bw"], g["peak_flops"], t["phase"], t["k"])
+        assert [int(k) for k in top["key"]] == [int(k, 16) for k in t["keys"]]
+
+
+def test_carry_closed_form(golden_dir):
+    g = load_golden(golden_dir, "carry_closed_form.json")
+    assert g["P"] == g["weight"] * g["duration_ns"] == (2**20 - 1) * (2**28 - 1)
+    for case in g["cases"]:
+        n = case["N"]
+        recs = np.zeros(n, dtype=RECORD_DTYPE)
+        recs["op_id"], recs["shape_id"], recs["phase"], recs["duration_ns"] = 3, 11, 1, g["duration_ns"]
+        o, ent = run_oracle(recs, [g["weight"]], 2)
+        assert len(ent) == 1
+        assert int(ent[0]["count"]) == n
+        assert int(ent[0]["wt_hi"]) == case["wt_hi"]
+        assert int(ent[0]["wt_lo"]) == int(case["wt_lo"], 16)
+        assert entry_wt(ent[0]) == n * g["P"]
+        assert f64_bits(oracle.u128_to_f64(n * g["P"])) == int(case["f64_bits"], 16)
+        assert f64_bits(float(ent[0]["phase_weight"])) == f64_bits(1.0)
+    big = g["large_case_not_run_on_cpu"]
+    x = big["N"] * g["P"]
+    assert x >> 64 == big["wt_hi"] and x & (2**64 - 1) == int(big["wt_lo"], 16)
+    assert f64_bits(oracle.u128_to_f64(x)) == int(big["f64_bits"], 16)
+
+
+def test_topk_uses_exact_integers_then_key(golden_dir):
+    g = load_golden(golden_dir, "topk_ties.json")
+    c = g["case_rounding"]
+    rows = []
+    for name in ("x", "y"):
+        k = c[name]
+        rows += [{"app": 0, "op": k["op"], "shape": k["shape"], "duration_ns": k["big_duration"]}] * k["n_big"]
+        if "extra_duration" in k:
+            rows.append({"app": 1, "op": k["op"], "shape": k["shape"], "duration_ns": k["extra_duration"]})
+    recs = records_from_dicts(rows)
+    o, ent = run_oracle(recs, c["app_weights"], 1)
+    by_key = {int(e["key"]): e for e in ent}
+    assert entry_wt(by_key[5]) == c["x"]["wt"] == 2**54 + 1
+    assert entry_wt(by_key[3]) == c["y"]["wt"] == 2**54
+    # the two doubles coincide, the integers do not
+    assert f64_bits(float(by_key[5]["phase_weight"])) == f64_bits(float(by_key[3]["phase_weight"]))
+    top = o.topk(PEAK_BW, PEAK_FLOPS, 0, 2)
+    assert [int(k) for k in top["key"]] == [int(k, 16) for k in c["top2_keys"]]
+
+    t = g["case_exact_ties"]
+    o, _ = run_oracle(records_from_dicts(t["records"]), t["app_weights"], 1)
+    assert [int(k) for k in o.topk(PEAK_BW, PEAK_FLOPS, 0, 3)["key"]] == [int(k, 16) for k in t["top3_keys"]]
+    assert [int(k) for k in o.topk(PEAK_BW, PEAK_FLOPS, 0, 9)["key"]] == [int(k, 16) for k in t["top4_keys"]]
+    assert len(o.topk(PEAK_BW, PEAK_FLOPS, 0, 0)) == 0
+
+
+# ---------------------------------------------------------------- integer -> binary64
+
+def test_u128_to_f64_vectors(golden_dir):
+    g = load_golden(golden_dir, "u128_to_f64_vectors.json")
+    for v in g["vectors"]:
+        x = (int(v["hi"], 16) << 64) | int(v["lo"], 16)
+        assert f64_bits(oracle.u128_to_f64(x)) == int(v["bits"], 16), v
+        if v.get("double_rounding_trap"):
+            naive = float(int(v["hi"], 16)) * 2.0**64 + float(int(v["lo"], 16))
+            assert f64_bits(naive) != int(v["bits"], 16)
+
+
+def _rne_reference(x: int) -> float:
+    """Round-to-nearest-even of a non-negative integer to binary64, from first principles."""
+    if x == 0:
+        return 0.0
+    e = x.bit_length() - 53
+    if e <= 0:
+        return math.ldexp(float(x), 0)
+    q, r = x >> e, x & ((1 << e) - 1)
+    half = 1 << (e - 1)
+    if r > half or (r == half and (q & 1)):
+        q += 1
+    return math.ldexp(float(q), e)
+
+
+def test_u128_to_f64_random_against_first_principles():
+    rng = random.Random(1234)
+    for _ in range(20000):
+        bits = rng.randrange(1, 129)
+        x = rng.getrandbits(bits)
+        if rng.random() < 0.3:  # force values near a rounding boundary
+            e = max(x.bit_length() - 53, 1)
+            x = ((x >> e) << e) | (1 << (e - 1)) | rng.choice([0, 0, 1])
+        x &= (1 << 128) - 1
+        assert oracle.u128_to_f64(x) == _rne_reference(x)
+
+
+# ---------------------------------------------------------------- brute force, every law
+
+@pytest.mark.parametrize("index", [0, 1, 2, 3, 4])
+def test_brute_force_python_ints(index):
+    spec = make_spec(index, small=True, n=4096, n_dtypes=3)
+    recs = tg.generate(spec)
+    # add a few invalid records and a key with no work row
+    bad = recs[:5].copy()
+    bad["app_id"][:2] = spec.n_apps
+    bad["app_id"][2] = 0xFFFFFFFF
+    bad["phase"][3:] = spec.n_phases
+    orphan = recs[:1].copy()
+    orphan["op_id"], orphan["shape_id"], orphan["pad"] = 0xFFFF, 0xFFFFFFFF, 0xAB
+    recs = np.concatenate([recs, bad, orphan])
+    work = spec.work_table()
+    o, ent = run_oracle(recs, spec.app_weights, spec.n_phases, work)
+    groups, totals, rejected = brute_force(recs, spec.app_weights, spec.n_phases)
+    assert rejected == 5 and o.stats()["n_rejected"] == 5
+    assert o.stats()["n_valid"] == len(recs) - 5
+    assert o.stats()["totals"] == totals
+    exp = expected_entry_fields(groups, totals, work, PEAK_BW, PEAK_FLOPS)
+    check_entries_against(ent, exp)
+    assert list(ent["key"]) == sorted(groups)  # key ascending
+    orphan_key = (int(orphan["phase"][0]) << 48) | (0xFFFF << 32) | 0xFFFFFFFF
+    assert exp[orphan_key][3] == 0x7FF8000000000000
+    for phase in range(spec.n_phases):
+        ranked = sorted((k for k in groups if k >> 48 == phase), key=lambda k: (-groups[k][1], k))
+        for k in (1, 7, len(ranked) + 3):
+            top = o.topk(PEAK_BW, PEAK_FLOPS, phase, k)
+            assert [int(x) for x in top["key"]] == ranked[:k]
+            check = {int(e["key"]): exp[int(e["key"])] for e in top}
+            check_entries_against(top, check)
+
+
+def test_phase_weight_is_quotient_of_rounded_operands_and_near_exact_ratio():
+    spec = make_spec(1, small=True, n=20000)
+    recs = tg.generate(spec)
+    o, ent = run_oracle(recs, spec.app_weights, spec.n_phases)
+    totals = o.stats()["totals"]
+    for e in ent[:: max(1, len(ent) // 200)]:
+        wt, t = entry_wt(e), totals[int(e["key"]) >> 48]
+        assert float(e["phase_weight"]) == float(wt) / float(t)
+        exact = Fraction(wt, t)
+        assert abs(Fraction(float(e["phase_weight"])) - exact) <= exact * Fraction(3, 2**53)
+
+
+# ---------------------------------------------------------------- invariants
+
+@pytest.mark.parametrize("index", [0, 1, 2, 3, 4])
+def test_invariants(index):
+    spec = make_spec(index, small=True, n=1 << 17)
+    recs = tg.generate(spec)
+    o, ent = run_oracle(recs, spec.app_weights, spec.n_phases, spec.work_table())
+    st = o.stats()
+    assert int(ent["count"].sum()) == st["n_valid"] == len(recs)
+    for p in range(spec.n_phases):
+        sel = ent[(ent["key"] >> np.uint64(48)) == p]
+        assert sum(entry_wt(e) for e in sel) == st["totals"][p]
+        s = math.fsum(sel["phase_weight"].tolist())
+        assert abs(s - 1.0) <= 3 * len(sel) * 2.0**-53          # Eq. 3: weights sum to 1
+    # independent total: sum of weight*duration over all records, per phase
+    w = spec.app_weights.astype(object)
+    for p in range(spec.n_phases):
+        m = recs["phase"] == p
+        tot = int(np.sum(w[recs["app_id"][m]] * recs["duration_ns"][m].astype(object)))
+        assert tot == st["totals"][p]
+    # permutation invariance
+    perm = np.random.default_rng(7).permutation(len(recs))
+    _, ent_p = run_oracle(recs[perm], spec.app_weights, spec.n_phases, spec.work_table())
+    assert ent_p.tobytes() == ent.tobytes()
+    # chunked == whole, threaded == single
+    o2 = oracle.Oracle(spec.app_weights, spec.n_phases)
+    o2.set_work(spec.work_table())
+    for c in np.array_split(recs, 8):
+        o2.ingest(c)
+    assert o2.finalize(PEAK_BW, PEAK_FLOPS).tobytes() == ent.tobytes()
+    _, ent_t = run_oracle(recs, spec.app_weights, spec.n_phases, spec.work_table(), threads=4)
+    assert ent_t.tobytes() == ent.tobytes()
+
+
+def test_unit_weights_reduce_to_a_library_group_sum():
+    # with every weight 1, wt is a plain per-key sum of durations: numpy sort + reduceat
+    spec = make_spec(0)
+    recs = tg.generate(spec)
+    _, ent = run_oracle(recs, np.ones(spec.n_apps, dtype=np.uint32), spec.n_phases)
+    key = (recs["phase"].astype(np.uint64) << np.uint64(48)) | (recs["op_id"].astype(np.uint64) << np.uint64(32)) \
+        | recs["shape_id"].astype(np.uint64)
+    order = np.argsort(key, kind="stable")
+    ks, first, counts = np.unique(key[order], return_index=True, return_counts=True)
+    sums = np.add.reduceat(recs["duration_ns"][order].astype(np.uint64), first)
+    assert np.array_equal(ent["key"], ks)
+    assert np.array_equal(ent["count"], counts.astype(np.uint64))
+    assert np.array_equal(ent["wt_lo"], sums) and not ent["wt_hi"].any()
+
+
+def test_skew_config_closed_form():
+    spec = make_spec(4, small=True, n=1 << 18)
+    recs = tg.generate(spec)
+    _, ent = run_oracle(recs, spec.app_weights, spec.n_phases)
+    P = (2**20 - 1) * (2**28 - 1)
+    for e in ent:
+        assert entry_wt(e) == int(e["count"]) * P
+    hot = ent[ent["key"] == ((1 << 48) | 0)]
+    assert len(hot) == 1 and int(hot[0]["count"]) > 65537 and int(hot[0]["wt_hi"]) >= 1
+
+
+# ---------------------------------------------------------------- edge cases
+
+def test_edge_cases():
+    o = oracle.Oracle([5], 2)
+    assert len(o.finalize(PEAK_BW, PEAK_FLOPS)) == 0 and o.stats()["n_keys"] == 0
+    # zero weight and zero durations: counts accumulate, totals stay 0, weight is +0.0
+    o = oracle.Oracle([0, 7], 2)
+    recs = records_from_dicts([{"app": 0, "op": 1, "shape": 1, "phase": 0, "duration_ns": 99},
+                               {"app": 1, "op": 1, "shape": 2, "phase": 0, "duration_ns": 0},
+                               {"app": 1, "op": 1, "shape": 2, "phase": 1, "duration_ns": 4}])
+    o.ingest(recs)
+    ent = o.finalize(PEAK_BW, PEAK_FLOPS)
+    assert [int(c) for c in ent["count"]] == [1, 1, 1]
+    assert f64_bits(float(ent[0]["phase_weight"])) == 0 and f64_bits(float(ent[1]["phase_weight"])) == 0
+    assert float(ent[2]["phase_weight"]) == 1.0
+    assert all(f64_bits(float(x)) == 0x7FF8000000000000 for x in ent["roofline_s"])
+    # key packing: the three fields must not alias
+    o = oracle.Oracle([1], 8)
+    recs = records_from_dicts([{"op": 0, "shape": 1, "phase": 0, "duration_ns": 1},
+                               {"op": 1, "shape": 0, "phase": 0, "duration_ns": 1},
+                               {"op": 0, "shape": 0, "phase": 1, "duration_ns": 1},
+                               {"op": 0xFFFF, "shape": 0xFFFFFFFF, "phase": 7, "duration_ns": 1}])
+    o.ingest(recs)
+    assert [int(k) for k in o.finalize(PEAK_BW, PEAK_FLOPS)["key"]] == [1, 1 << 32, 1 << 48, 0x0007FFFFFFFFFFFF]
+    # duplicate work rows and out-of-range dtype are refused
+    w = work_from_dicts([{"op": 1, "shape": 2, "flops": 1, "bytes": 1}, {"op": 1, "shape": 2, "flops": 2, "bytes": 2}])
+    assert o.set_work(w) == -1
+    w = work_from_dicts([{"op": 1, "shape": 2, "dtype": 8, "flops": 1, "bytes": 1}])
+    assert o.set_work(w) == -1
+
+
+def test_roofline_picks_the_larger_side_per_dtype():
+    # F/P for dtype 2 (4e15) vs M/beta: rows constructed so each side wins once
+    w = work_from_dicts([{"op": 0, "shape": 0, "dtype": 2, "flops": 8 * 10**15, "bytes": 8 * 10**12},   # 2 s vs 1 s
+                         {"op": 0, "shape": 1, "dtype": 2, "flops": 4 * 10**15, "bytes": 24 * 10**12},  # 1 s vs 3 s
+                         {"op": 0, "shape": 2, "dtype": 0, "flops": 4 * 10**15, "bytes": 8 * 10**12}])  # 4 s vs 1 s
+    recs = records_from_dicts([{"op": 0, "shape": s, "duration_ns": 1} for s in (0, 1, 2)])
+    _, ent = run_oracle(recs, [1], 1, w)
+    assert [float(x) for x in ent["roofline_s"]] == [2.0, 3.0, 4.0]
