@@ -1,0 +1,191 @@
+/*
+ * atrex_agg.h -- C ABI of the B200 trace-aggregation library.
+ *
+ * The library turns production inference-trace records into per-problem importance
+ * weights and roofline ceilings, as defined by the paper's benchmark construction:
+ *
+ *   Eq. 2  cumulative observed device time per (operator, phase), summed over kernel
+ *          invocations; here kept per (operator, shape, phase) key and scaled by the
+ *          application's card-hour weight (Eq. 3's p_a) as an exact 128-bit integer;
+ *   Eq. 3  normalisation so that weights sum to 1, taken separately for each serving
+ *          phase (Sec. 3.1 "computed separately for the serving phases");
+ *   Eq. 1  roofline time max(F / P_dtype, M / beta) per (operator, shape) unit;
+ *   Table 2  ranking of units by weight (deterministic top-k).
+ *
+ * Conventions
+ *   - Plain C, no exceptions, no global state: every call takes the handle.
+ *   - "DEVICE" pointers are CUDA device memory on the handle's device; "HOST" pointers are
+ *     ordinary host memory.  `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - All integers are little-endian; structs are packed as declared (no padding occurs).
+ *   - Every function returns ATREX_OK (0) or a negative atrex_status_t; nothing aborts,
+ *     traps or waits without a bound.
+ *   - A handle must not be used from two host threads at once.
+ *
+ * Arithmetic contract (what makes results unique, so they can be compared bit for bit)
+ *   key          = phase << 48 | op_id << 32 | shape_id
+ *   count[key]   = number of valid records with that key                      (u64)
+ *   wt[key]      = sum of app_weight[app_id] * duration_ns over those records  (u128, exact,
+ *                  independent of ingestion order and chunking)
+ *   T[phase]     = sum of wt over the phase's keys                             (u128)
+ *   phase_weight = fl(fl(wt) / fl(T[phase])), or +0.0 when T[phase] == 0, where fl() of an
+ *                  integer is ONE round-to-nearest-even conversion to binary64 and the
+ *                  division is IEEE-754 binary64
+ *   roofline_s   = fmax(fl(flops) / peak_flops[dtype], fl(bytes) / peak_bw); a key whose
+ *                  (op_id, shape_id) has no work-table row gets the quiet NaN 0x7FF8000000000000
+ *   A record is valid iff app_id < n_apps and phase < n_phases; invalid records are skipped
+ *   and counted.  The `pad` byte is ignored.
+ *   Limits: fewer than 2^40 records per handle between resets (so wt < 2^88).
+ */
+#ifndef ATREX_AGG_H
+#define ATREX_AGG_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ATREX_MAX_PHASES 8
+#define ATREX_MAX_DTYPES 8
+#define ATREX_MAX_TOPK 65536u
+
+typedef enum {
+    ATREX_OK = 0,
+    ATREX_ERR_INVALID = -1,        /* bad argument: null/misaligned pointer, range, duplicate work row */
+    ATREX_ERR_CAPACITY = -2,       /* more distinct keys than provisioned; results are not valid        */
+    ATREX_ERR_OUT_TOO_SMALL = -3,  /* output buffer too small; *n_out holds the needed count            */
+    ATREX_ERR_CUDA = -4,           /* a CUDA runtime call failed (see atrex_agg_last_cuda_error)        */
+    ATREX_ERR_TIMEOUT = -5,        /* a bounded device-side wait gave up                                */
+    ATREX_ERR_STATE = -6,          /* call order: topk before finalize, or > 2^40 records               */
+    ATREX_ERR_NOMEM = -7           /* workspace too small / allocation failed                           */
+} atrex_status_t;
+
+/* One observed device-kernel invocation (Sec. 3.1; the d_{a,phi,r,l} of Eq. 2). 16 bytes. */
+typedef struct {
+    uint32_t app_id;       /* application index a                      */
+    uint16_t op_id;        /* operator family i                        */
+    uint8_t  phase;        /* serving phase phi: 0 = prefill, 1 = decode, ... < n_phases */
+    uint8_t  pad;          /* ignored                                  */
+    uint32_t shape_id;     /* shape bucket s                           */
+    uint32_t duration_ns;  /* observed device time of this invocation  */
+} atrex_record_t;
+
+/* Semantic work of one (operator, shape) unit (Sec. 3.3: F_j, M_j and the dtype tau_j). 24 bytes. */
+typedef struct {
+    uint32_t shape_id;
+    uint16_t op_id;
+    uint16_t dtype;        /* index into atrex_hw_peaks_t.peak_flops, < ATREX_MAX_DTYPES */
+    uint64_t flops;
+    uint64_t bytes;
+} atrex_work_t;
+
+/* Calibrated accelerator peaks (Sec. 3.3: P_tau and beta). All must be finite and > 0. */
+typedef struct {
+    double peak_bw;                        /* bytes / s  */
+    double peak_flops[ATREX_MAX_DTYPES];   /* FLOP / s per dtype index */
+} atrex_hw_peaks_t;
+
+/* One aggregated unit. 48 bytes. */
+typedef struct {
+    uint64_t key;           /* phase << 48 | op_id << 32 | shape_id */
+    uint64_t count;
+    uint64_t wt_lo;         /* weighted time, low and high 64 bits  */
+    uint64_t wt_hi;
+    double   phase_weight;
+    double   roofline_s;
+} atrex_entry_t;
+
+typedef struct {
+    uint32_t n_apps;              /* >= 1 */
+    uint32_t n_phases;            /* 1 .. ATREX_MAX_PHASES */
+    uint64_t max_keys;            /* distinct (op, shape, phase) keys to provision for, >= 1 */
+    uint64_t max_work_rows;       /* rows atrex_agg_set_work_table may receive (0 = none)    */
+    const uint32_t* app_weights;  /* HOST, n_apps card-hour weights; copied by create        */
+    void*    workspace;           /* DEVICE memory owned by the caller, 256-byte aligned, or */
+    uint64_t workspace_bytes;     /*   NULL/0: the library allocates and frees its own       */
+    int32_t  device;              /* CUDA device ordinal */
+    uint32_t flags;               /* ATREX_FLAG_* */
+} atrex_agg_config_t;
+
+#define ATREX_FLAG_NO_HOT_DIRECTORY 1u  /* disable the shared-memory hot-key stage (debug / A-B) */
+
+typedef struct {
+    uint64_t n_valid;                     /* valid records ingested since create/reset */
+    uint64_t n_rejected;                  /* records skipped as invalid                */
+    uint64_t n_dropped;                   /* records lost to a full table (ATREX_ERR_CAPACITY) */
+    uint64_t n_keys;                      /* distinct keys                             */
+    uint64_t total_lo[ATREX_MAX_PHASES];  /* T[phase], low / high 64 bits              */
+    uint64_t total_hi[ATREX_MAX_PHASES];
+    uint64_t keys_per_phase[ATREX_MAX_PHASES];
+    uint64_t table_slots;                 /* capacity of the key table                 */
+    uint64_t hot_slots;                   /* keys currently in the shared-memory hot directory */
+} atrex_stats_t;
+
+typedef struct atrex_agg atrex_agg_t;
+
+/* Bytes of DEVICE workspace a handle with this configuration needs (0 on invalid config). */
+uint64_t atrex_agg_workspace_bytes(const atrex_agg_config_t* cfg);
+
+/* Create a handle.  The workspace (caller's or library-allocated) is cleared on the device's
+ * default stream and the call returns after that completes.  The caller keeps ownership of
+ * cfg->workspace and must keep it alive until atrex_agg_destroy. */
+int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out);
+
+/* Install the per-(operator, shape) work table used by Eq. 1.  `host_rows` is HOST memory, read
+ * before the call returns.  n <= max_work_rows.  Duplicate (op, shape) pairs or dtype >=
+ * ATREX_MAX_DTYPES give ATREX_ERR_INVALID (the table is then empty).  Synchronises `stream`. */
+int atrex_agg_set_work_table(atrex_agg_t*, const atrex_work_t* host_rows, uint64_t n, void* stream);
+
+/* Eq. 2: fold n records into the per-key sums.  `d_records` is DEVICE memory, 16-byte aligned,
+ * and must stay valid until `stream` has passed this call.  Asynchronous: returns after
+ * enqueueing; device-side conditions (table full) are latched and reported by the next
+ * finalize / stats.  May be called any number of times; the result is independent of how the
+ * records are split into calls and of their order. */
+int atrex_agg_ingest(atrex_agg_t*, const atrex_record_t* d_records, uint64_t n, void* stream);
+
+/* Same, for records in HOST memory (pinned memory gives asynchronous copies): the records are
+ * copied through two device staging buffers inside the workspace, each copy overlapping the
+ * previous piece's aggregation.  Returns after enqueueing the last piece; `h_records` must
+ * stay valid until `stream` has passed this call. */
+int atrex_agg_ingest_host(atrex_agg_t*, const atrex_record_t* h_records, uint64_t n, void* stream);
+
+/* Fold already aggregated units (for instance another GPU's partial result: key, count, wt_lo,
+ * wt_hi are read; the two doubles are ignored) into the table.  DEVICE pointer, asynchronous.
+ * Exact: merging partial aggregates in any order equals aggregating all records at once. */
+int atrex_agg_merge(atrex_agg_t*, const atrex_entry_t* d_entries, uint64_t n, void* stream);
+
+/* Eq. 3 (per phase) and Eq. 1 for every key.  Writes one entry per distinct key to `d_out`
+ * (DEVICE, capacity out_cap entries, order unspecified) and the number of entries to *n_out
+ * (HOST).  d_out may be NULL with out_cap 0 to only obtain the count, refresh the totals and
+ * set the peaks used by atrex_agg_topk.  Synchronises `stream`.  Non-destructive: ingest may
+ * continue afterwards and finalize may be repeated, e.g. with other peaks. */
+int atrex_agg_finalize(atrex_agg_t*, const atrex_hw_peaks_t* peaks, atrex_entry_t* d_out,
+                       uint64_t out_cap, uint64_t* n_out, void* stream);
+
+/* Table 2: the min(k, keys of `phase`) entries with the largest weighted time, compared as
+ * exact 128-bit integers, ties broken by ascending key; written in that order to `h_out`
+ * (HOST, capacity k).  k <= ATREX_MAX_TOPK.  Uses the totals and peaks of the last finalize
+ * (ATREX_ERR_STATE if there was none since the last ingest).  Synchronises `stream`. */
+int atrex_agg_topk(atrex_agg_t*, uint32_t phase, uint32_t k, atrex_entry_t* h_out, uint32_t* n_out,
+                   void* stream);
+
+/* Counters and per-phase totals (HOST output).  Synchronises `stream`. */
+int atrex_agg_stats(atrex_agg_t*, atrex_stats_t* h_out, void* stream);
+
+/* Forget all records (the work table and weights are kept).  Asynchronous on `stream`. */
+int atrex_agg_reset(atrex_agg_t*, void* stream);
+
+void atrex_agg_destroy(atrex_agg_t*);
+
+const char* atrex_strerror(int status);
+
+/* cudaError_t value of the last failed CUDA call on this handle (0 if none). */
+int atrex_agg_last_cuda_error(const atrex_agg_t*);
+
+/* Number of kernels this handle has launched so far (for launch accounting in benchmarks). */
+uint64_t atrex_agg_launch_count(const atrex_agg_t*);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATREX_AGG_H */

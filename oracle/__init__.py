@@ -41,6 +41,8 @@ def lib():
         L.oracle_ingest.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
         L.oracle_ingest_threads.restype = C.c_uint32
         L.oracle_ingest_threads.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32]
+        L.oracle_ingest_filtered.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64]
+        L.oracle_direct_totals.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p]
         L.oracle_set_work.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
         L.oracle_n_keys.restype = C.c_uint64
         L.oracle_n_keys.argtypes = [C.c_void_p]
@@ -84,6 +86,17 @@ class Oracle:
             lib().oracle_ingest(self._h, r.ctypes.data, r.shape[0])
             return 1
         return lib().oracle_ingest_threads(self._h, r.ctypes.data, r.shape[0], threads)
+
+    def ingest_filtered(self, records: np.ndarray, keys) -> None:
+        r = np.ascontiguousarray(records)
+        k = np.ascontiguousarray(keys, dtype=np.uint64)
+        lib().oracle_ingest_filtered(self._h, r.ctypes.data, r.shape[0], k.ctypes.data, k.shape[0])
+
+    def direct_totals(self, records: np.ndarray, acc: np.ndarray, valid: np.ndarray) -> None:
+        """acc: uint64[16] (lo, hi per phase), valid: uint64[2]; both updated in place."""
+        r = np.ascontiguousarray(records)
+        assert acc.dtype == np.uint64 and acc.shape == (16,) and valid.dtype == np.uint64 and valid.shape == (2,)
+        lib().oracle_direct_totals(self._h, r.ctypes.data, r.shape[0], acc.ctypes.data, valid.ctypes.data)
 
     def set_work(self, rows: np.ndarray) -> int:
         r = np.ascontiguousarray(rows)

@@ -205,6 +205,48 @@ uint32_t oracle_ingest_threads(void* h, const void* records, uint64_t n, uint32_
     return threads;
 }
 
+// Full-size spot checks: aggregate only the records whose key is in `keys` (n_keys values,
+// any order).  Same definition as oracle_ingest restricted to those keys, so that sampled
+// outputs of a trace too large for the full map can be computed one by one.
+void oracle_ingest_filtered(void* h, const void* records, uint64_t n, const uint64_t* keys, uint64_t n_keys) {
+    Oracle* o = (Oracle*)h;
+    std::vector<uint64_t> want(keys, keys + n_keys);
+    std::sort(want.begin(), want.end());
+    const Rec* recs = (const Rec*)records;
+    for (uint64_t i = 0; i < n; ++i) {
+        const Rec& r = recs[i];
+        if (r.app_id >= o->n_apps || r.phase >= o->n_phases) continue;
+        uint64_t k = pack_key(r);
+        if (!std::binary_search(want.begin(), want.end(), k)) continue;
+        Acc& a = o->groups[k];
+        a.count += 1;
+        a.wt += (u128)o->app_weight[r.app_id] * (u128)r.duration_ns;
+    }
+}
+
+// Per-phase totals straight from the records, without any grouping: Eq. 2's D^phi as a plain
+// sum.  acc[2p], acc[2p+1] (low, high) are updated in place so the call can be repeated per
+// chunk; valid[0] / valid[1] accumulate the valid and rejected record counts.
+void oracle_direct_totals(void* h, const void* records, uint64_t n, uint64_t acc[16], uint64_t valid[2]) {
+    Oracle* o = (Oracle*)h;
+    const Rec* recs = (const Rec*)records;
+    u128 t[8];
+    for (int p = 0; p < 8; ++p) t[p] = ((u128)acc[2 * p + 1] << 64) | acc[2 * p];
+    for (uint64_t i = 0; i < n; ++i) {
+        const Rec& r = recs[i];
+        if (r.app_id >= o->n_apps || r.phase >= o->n_phases) {
+            ++valid[1];
+            continue;
+        }
+        ++valid[0];
+        t[r.phase] += (u128)o->app_weight[r.app_id] * (u128)r.duration_ns;
+    }
+    for (int p = 0; p < 8; ++p) {
+        acc[2 * p] = (uint64_t)t[p];
+        acc[2 * p + 1] = (uint64_t)(t[p] >> 64);
+    }
+}
+
 // Install the per-(operator, shape) semantic work table.  Returns 0, or -1 on a
 // duplicate pair or a dtype index >= 8 (table left empty).
 int oracle_set_work(void* h, const void* rows, uint64_t n) {

@@ -1,0 +1,251 @@
+"""ctypes binding of the C ABI declared in ``include/atrex_agg.h``.
+
+Argument marshalling only: every step of the aggregation path runs in the library's CUDA
+kernels.  PyTorch appears here for device memory (workspace, output buffers) and streams.
+There is no CPU fallback: if the shared library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libatrex_agg.so")
+
+ATREX_MAX_PHASES = 8
+ATREX_MAX_DTYPES = 8
+ATREX_MAX_TOPK = 65536
+ATREX_FLAG_NO_HOT_DIRECTORY = 1
+
+ATREX_OK = 0
+ATREX_ERR_INVALID = -1
+ATREX_ERR_CAPACITY = -2
+ATREX_ERR_OUT_TOO_SMALL = -3
+ATREX_ERR_CUDA = -4
+ATREX_ERR_TIMEOUT = -5
+ATREX_ERR_STATE = -6
+ATREX_ERR_NOMEM = -7
+
+RECORD_DTYPE = np.dtype([("app_id", "<u4"), ("op_id", "<u2"), ("phase", "u1"), ("pad", "u1"),
+                         ("shape_id", "<u4"), ("duration_ns", "<u4")])
+WORK_DTYPE = np.dtype([("shape_id", "<u4"), ("op_id", "<u2"), ("dtype", "<u2"), ("flops", "<u8"), ("bytes", "<u8")])
+ENTRY_DTYPE = np.dtype([("key", "<u8"), ("count", "<u8"), ("wt_lo", "<u8"), ("wt_hi", "<u8"),
+                        ("phase_weight", "<f8"), ("roofline_s", "<f8")])
+
+EXPORTED_SYMBOLS = [
+    "atrex_agg_workspace_bytes", "atrex_agg_create", "atrex_agg_set_work_table", "atrex_agg_ingest",
+    "atrex_agg_ingest_host", "atrex_agg_merge", "atrex_agg_finalize", "atrex_agg_topk", "atrex_agg_stats",
+    "atrex_agg_reset", "atrex_agg_destroy", "atrex_strerror", "atrex_agg_last_cuda_error",
+    "atrex_agg_launch_count",
+]
+
+
+class atrex_agg_config_t(C.Structure):
+    _fields_ = [("n_apps", C.c_uint32), ("n_phases", C.c_uint32), ("max_keys", C.c_uint64),
+                ("max_work_rows", C.c_uint64), ("app_weights", C.c_void_p), ("workspace", C.c_void_p),
+                ("workspace_bytes", C.c_uint64), ("device", C.c_int32), ("flags", C.c_uint32)]
+
+
+class atrex_hw_peaks_t(C.Structure):
+    _fields_ = [("peak_bw", C.c_double), ("peak_flops", C.c_double * ATREX_MAX_DTYPES)]
+
+
+class atrex_stats_t(C.Structure):
+    _fields_ = [("n_valid", C.c_uint64), ("n_rejected", C.c_uint64), ("n_dropped", C.c_uint64),
+                ("n_keys", C.c_uint64), ("total_lo", C.c_uint64 * ATREX_MAX_PHASES),
+                ("total_hi", C.c_uint64 * ATREX_MAX_PHASES), ("keys_per_phase", C.c_uint64 * ATREX_MAX_PHASES),
+                ("table_slots", C.c_uint64), ("hot_slots", C.c_uint64)]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is not built; run `python -m paper_2607_14541_b200.build` "
+                          "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, u64, u32 = C.c_void_p, C.c_uint64, C.c_uint32
+    L.atrex_agg_workspace_bytes.restype = u64
+    L.atrex_agg_workspace_bytes.argtypes = [C.POINTER(atrex_agg_config_t)]
+    L.atrex_agg_create.argtypes = [C.POINTER(atrex_agg_config_t), C.POINTER(vp)]
+    L.atrex_agg_set_work_table.argtypes = [vp, vp, u64, vp]
+    L.atrex_agg_ingest.argtypes = [vp, vp, u64, vp]
+    L.atrex_agg_ingest_host.argtypes = [vp, vp, u64, vp]
+    L.atrex_agg_merge.argtypes = [vp, vp, u64, vp]
+    L.atrex_agg_finalize.argtypes = [vp, C.POINTER(atrex_hw_peaks_t), vp, u64, C.POINTER(u64), vp]
+    L.atrex_agg_topk.argtypes = [vp, u32, u32, vp, C.POINTER(u32), vp]
+    L.atrex_agg_stats.argtypes = [vp, C.POINTER(atrex_stats_t), vp]
+    L.atrex_agg_reset.argtypes = [vp, vp]
+    L.atrex_agg_destroy.argtypes = [vp]
+    L.atrex_agg_destroy.restype = None
+    L.atrex_strerror.restype = C.c_char_p
+    L.atrex_strerror.argtypes = [C.c_int]
+    L.atrex_agg_last_cuda_error.argtypes = [vp]
+    L.atrex_agg_launch_count.restype = u64
+    L.atrex_agg_launch_count.argtypes = [vp]
+    return L
+
+
+lib = _load()
+
+# the C entry points under their own names
+atrex_agg_workspace_bytes = lib.atrex_agg_workspace_bytes
+atrex_agg_create = lib.atrex_agg_create
+atrex_agg_set_work_table = lib.atrex_agg_set_work_table
+atrex_agg_ingest = lib.atrex_agg_ingest
+atrex_agg_ingest_host = lib.atrex_agg_ingest_host
+atrex_agg_merge = lib.atrex_agg_merge
+atrex_agg_finalize = lib.atrex_agg_finalize
+atrex_agg_topk = lib.atrex_agg_topk
+atrex_agg_stats = lib.atrex_agg_stats
+atrex_agg_reset = lib.atrex_agg_reset
+atrex_agg_destroy = lib.atrex_agg_destroy
+atrex_strerror = lib.atrex_strerror
+atrex_agg_last_cuda_error = lib.atrex_agg_last_cuda_error
+atrex_agg_launch_count = lib.atrex_agg_launch_count
+
+
+class AtrexError(RuntimeError):
+    def __init__(self, status: int, where: str, cuda_error: int = 0):
+        self.status = status
+        msg = f"{where}: {atrex_strerror(status).decode()} ({status})"
+        if cuda_error:
+            msg += f" [cudaError {cuda_error}]"
+        super().__init__(msg)
+
+
+def make_peaks(peak_bw: float, peak_flops) -> atrex_hw_peaks_t:
+    pk = atrex_hw_peaks_t()
+    pk.peak_bw = float(peak_bw)
+    pf = list(peak_flops) + [1.0] * (ATREX_MAX_DTYPES - len(peak_flops))
+    for i in range(ATREX_MAX_DTYPES):
+        pk.peak_flops[i] = float(pf[i])
+    return pk
+
+
+class Aggregator:
+    """One aggregation handle on one GPU.  Thin object wrapper over the C calls."""
+
+    def __init__(self, app_weights, n_phases: int, max_keys: int, max_work_rows: int = 0, device: int = 0,
+                 flags: int = 0, own_workspace: bool = False):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("the aggregation path is CUDA-only and no CUDA device is available")
+        self._torch = torch
+        self.device = int(device)
+        w = np.ascontiguousarray(app_weights, dtype=np.uint32)
+        cfg = atrex_agg_config_t()
+        cfg.n_apps, cfg.n_phases = int(w.shape[0]), int(n_phases)
+        cfg.max_keys, cfg.max_work_rows = int(max_keys), int(max_work_rows)
+        cfg.app_weights = w.ctypes.data
+        cfg.device, cfg.flags = self.device, int(flags)
+        self._ws = None
+        if not own_workspace:
+            nbytes = atrex_agg_workspace_bytes(C.byref(cfg))
+            if nbytes == 0:
+                raise AtrexError(ATREX_ERR_INVALID, "atrex_agg_workspace_bytes")
+            self._ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=f"cuda:{self.device}")
+            base = (self._ws.data_ptr() + 255) // 256 * 256
+            cfg.workspace, cfg.workspace_bytes = base, nbytes
+        h = C.c_void_p()
+        rc = atrex_agg_create(C.byref(cfg), C.byref(h))
+        if rc != ATREX_OK:
+            raise AtrexError(rc, "atrex_agg_create")
+        self._h = h
+        self.workspace_bytes = int(cfg.workspace_bytes)
+
+    # -- helpers
+    def _stream(self, stream=None):
+        if stream is None:
+            return self._torch.cuda.current_stream(self.device).cuda_stream
+        return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+    def _check(self, rc, where):
+        if rc != ATREX_OK:
+            raise AtrexError(rc, where, atrex_agg_last_cuda_error(self._h))
+
+    def close(self):
+        if getattr(self, "_h", None):
+            atrex_agg_destroy(self._h)
+            self._h = None
+            self._ws = None
+
+    __del__ = close
+
+    # -- the path
+    def set_work_table(self, rows: np.ndarray, stream=None):
+        r = np.ascontiguousarray(rows)
+        assert r.dtype.itemsize == 24
+        self._check(atrex_agg_set_work_table(self._h, r.ctypes.data, r.shape[0], self._stream(stream)),
+                    "atrex_agg_set_work_table")
+
+    def ingest(self, records, n: int | None = None, stream=None):
+        """``records``: CUDA uint8 tensor holding 16-byte records (or a raw device pointer with ``n``)."""
+        if isinstance(records, int):
+            ptr = records
+        else:
+            assert records.is_cuda and records.device.index == self.device
+            ptr = records.data_ptr()
+            if n is None:
+                n = records.numel() * records.element_size() // 16
+        self._check(atrex_agg_ingest(self._h, ptr, int(n), self._stream(stream)), "atrex_agg_ingest")
+
+    def ingest_host(self, records, n: int | None = None, stream=None):
+        """``records``: numpy array or CPU (ideally pinned) tensor of 16-byte records."""
+        if isinstance(records, np.ndarray):
+            r = np.ascontiguousarray(records)
+            ptr, nb = r.ctypes.data, r.nbytes
+        else:
+            assert not records.is_cuda and records.is_contiguous()
+            ptr, nb = records.data_ptr(), records.numel() * records.element_size()
+        if n is None:
+            n = nb // 16
+        self._check(atrex_agg_ingest_host(self._h, ptr, int(n), self._stream(stream)), "atrex_agg_ingest_host")
+
+    def merge(self, entries, n: int | None = None, stream=None):
+        assert entries.is_cuda
+        if n is None:
+            n = entries.numel() * entries.element_size() // 48
+        self._check(atrex_agg_merge(self._h, entries.data_ptr(), int(n), self._stream(stream)), "atrex_agg_merge")
+
+    def finalize(self, peak_bw: float, peak_flops, out=None, stream=None):
+        """Returns (entries, n): a CUDA uint8 tensor of 48-byte entries and the entry count."""
+        torch = self._torch
+        pk = make_peaks(peak_bw, peak_flops)
+        n_out = C.c_uint64(0)
+        if out is None:
+            rc = atrex_agg_finalize(self._h, C.byref(pk), None, 0, C.byref(n_out), self._stream(stream))
+            self._check(rc, "atrex_agg_finalize")
+            out = torch.empty(max(int(n_out.value), 1) * 48, dtype=torch.uint8, device=f"cuda:{self.device}")
+        cap = out.numel() * out.element_size() // 48
+        rc = atrex_agg_finalize(self._h, C.byref(pk), out.data_ptr(), cap, C.byref(n_out), self._stream(stream))
+        self._check(rc, "atrex_agg_finalize")
+        return out, int(n_out.value)
+
+    def finalize_numpy(self, peak_bw: float, peak_flops, stream=None) -> np.ndarray:
+        out, n = self.finalize(peak_bw, peak_flops, stream=stream)
+        return out[: n * 48].cpu().numpy().view(ENTRY_DTYPE).copy()
+
+    def topk(self, phase: int, k: int, stream=None) -> np.ndarray:
+        out = np.zeros(max(k, 1), dtype=ENTRY_DTYPE)
+        n_out = C.c_uint32(0)
+        rc = atrex_agg_topk(self._h, int(phase), int(k), out.ctypes.data, C.byref(n_out), self._stream(stream))
+        self._check(rc, "atrex_agg_topk")
+        return out[: n_out.value].copy()
+
+    def stats(self, stream=None, check: bool = True) -> dict:
+        st = atrex_stats_t()
+        rc = atrex_agg_stats(self._h, C.byref(st), self._stream(stream))
+        if check:
+            self._check(rc, "atrex_agg_stats")
+        return {"status": rc, "n_valid": st.n_valid, "n_rejected": st.n_rejected, "n_dropped": st.n_dropped,
+                "n_keys": st.n_keys,
+                "totals": [int(st.total_lo[p]) | (int(st.total_hi[p]) << 64) for p in range(ATREX_MAX_PHASES)],
+                "keys_per_phase": [int(x) for x in st.keys_per_phase], "table_slots": st.table_slots,
+                "hot_slots": st.hot_slots}
+
+    def reset(self, stream=None):
+        self._check(atrex_agg_reset(self._h, self._stream(stream)), "atrex_agg_reset")
+
+    def launch_count(self) -> int:
+        return int(atrex_agg_launch_count(self._h))

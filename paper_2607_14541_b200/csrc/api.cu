@@ -1,0 +1,529 @@
+// C ABI of the trace-aggregation library: argument checks, workspace carving, launches.
+// The declarations and their contracts are in include/atrex_agg.h.
+#include <cmath>
+#include <cstddef>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "kernels.h"
+
+using namespace atrex;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+constexpr size_t STAGING_BYTES = 64ull << 20;          // per staging buffer (two of them)
+constexpr ull MAX_RECORDS_PER_LAUNCH = 1ull << 31;      // keeps per-CTA 32-bit counts from wrapping
+constexpr ull MAX_RECORDS_TOTAL = 1ull << 40;
+constexpr uint32_t HOT_MIN_RECORDS = 32768;             // smaller calls run without a directory
+constexpr uint32_t HOT_SAMPLE = 131072;
+constexpr uint32_t APPW_SMEM_MAX = 4096;
+constexpr uint32_t MAX_PROBE = 4096;
+constexpr uint32_t SEL_CAP = ATREX_MAX_TOPK + TOPK_CAND_CAP;
+
+size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+ull pow2_at_least(ull x) {
+    ull p = 1;
+    while (p < x) p <<= 1;
+    return p;
+}
+
+int log2_of(ull p) {
+    int l = 0;
+    while ((1ull << l) < p) ++l;
+    return l;
+}
+
+struct Layout {
+    size_t off_ctl, off_table, off_work, off_appw, off_hot, off_staging[2], off_sel, off_topk_out, total;
+    ull n_slots, work_slots;
+    uint32_t hot_slots;
+    bool appw_in_smem;
+};
+
+bool config_ok(const atrex_agg_config_t* c) {
+    if (!c) return false;
+    if (c->n_apps == 0 || c->n_phases == 0 || c->n_phases > ATREX_MAX_PHASES) return false;
+    if (c->max_keys == 0 || c->max_keys > (1ull << 30)) return false;
+    if (c->max_work_rows > (1ull << 30)) return false;
+    return true;
+}
+
+void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, Layout* L) {
+    L->n_slots = pow2_at_least(c->max_keys * 2 < 1024 ? 1024 : c->max_keys * 2);
+    L->work_slots = c->max_work_rows ? pow2_at_least(c->max_work_rows * 2 < 1024 ? 1024 : c->max_work_rows * 2) : 0;
+    L->appw_in_smem = c->n_apps <= APPW_SMEM_MAX;
+    size_t appw_smem = L->appw_in_smem ? (size_t)c->n_apps * 4 : 0;
+    size_t budget = smem_optin > appw_smem + 2048 ? smem_optin - appw_smem - 2048 : 0;
+    L->hot_slots = (uint32_t)(budget / 20) & ~1u;
+    if (c->flags & ATREX_FLAG_NO_HOT_DIRECTORY) L->hot_slots = 0;
+    size_t o = 0;
+    L->off_ctl = o;            o += round_up(sizeof(Control), ALIGN);
+    L->off_table = o;          o += round_up(L->n_slots * sizeof(Slot), ALIGN);
+    L->off_work = o;           o += round_up(L->work_slots * sizeof(WorkSlot), ALIGN);
+    L->off_appw = o;           o += round_up((size_t)c->n_apps * 4, ALIGN);
+    L->off_hot = o;            o += round_up((size_t)(L->hot_slots ? L->hot_slots : 2) * 8, ALIGN);
+    L->off_staging[0] = o;     o += STAGING_BYTES;
+    L->off_staging[1] = o;     o += STAGING_BYTES;
+    L->off_sel = o;            o += round_up((size_t)SEL_CAP * 32, ALIGN);
+    L->off_topk_out = o;       o += round_up((size_t)ATREX_MAX_TOPK * sizeof(atrex_entry_t), ALIGN);
+    L->total = o;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) cudaSetDevice(dev);
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+struct atrex_agg {
+    atrex_agg_config_t cfg;
+    Layout L;
+    int n_sms = 0;
+    bool owns_workspace = false;
+    unsigned char* ws = nullptr;
+    Control* ctl = nullptr;
+    Slot* table = nullptr;
+    WorkSlot* work = nullptr;
+    uint32_t* d_appw = nullptr;
+    ull* hot_keys = nullptr;
+    unsigned char* staging[2] = {nullptr, nullptr};
+    ull* sel = nullptr;
+    atrex_entry_t* topk_out = nullptr;
+    Control* h_ctl = nullptr;  // pinned mirror
+    bool hot_ready = false;
+    bool finalized = false;
+    atrex_hw_peaks_t peaks;
+    ull n_records = 0;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_ready[2] = {nullptr, nullptr}, ev_free[2] = {nullptr, nullptr};
+    int last_cuda_error = 0;
+    uint64_t launches = 0;
+
+    TableRef table_ref() const {
+        TableRef t;
+        t.table = table;
+        t.mask = L.n_slots - 1;
+        t.shift = 64 - log2_of(L.n_slots);
+        t.max_probe = (uint32_t)(L.n_slots < MAX_PROBE ? L.n_slots : MAX_PROBE);
+        t.ctl = ctl;
+        return t;
+    }
+    WorkRef work_ref() const {
+        WorkRef w;
+        w.table = L.work_slots ? work : nullptr;
+        w.mask = L.work_slots ? L.work_slots - 1 : 0;
+        w.shift = L.work_slots ? 64 - log2_of(L.work_slots) : 0;
+        w.max_probe = (uint32_t)(L.work_slots < MAX_PROBE ? L.work_slots : MAX_PROBE);
+        return w;
+    }
+    int scan_grid(ull n_items, int threads) const {
+        ull g = (n_items + threads - 1) / threads;
+        ull cap = (ull)n_sms * 8;
+        if (g > cap) g = cap;
+        return g < 1 ? 1 : (int)g;
+    }
+};
+
+#define CU(h, call)                                   \
+    do {                                              \
+        cudaError_t e_ = (call);                      \
+        if (e_ != cudaSuccess) {                      \
+            (h)->last_cuda_error = (int)e_;           \
+            return ATREX_ERR_CUDA;                    \
+        }                                             \
+    } while (0)
+
+static int device_status_to_error(const Control* c) {
+    if (c->status & ST_TIMEOUT) return ATREX_ERR_TIMEOUT;
+    if (c->status & ST_TABLE_FULL) return ATREX_ERR_CAPACITY;
+    return ATREX_OK;
+}
+
+static int query_smem_optin(int device, size_t* out) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) return -1;
+    *out = (size_t)v;
+    return 0;
+}
+
+extern "C" {
+
+uint64_t atrex_agg_workspace_bytes(const atrex_agg_config_t* cfg) {
+    if (!config_ok(cfg)) return 0;
+    // the directory size depends on the device's shared memory; without a device, size for
+    // the sm_100 maximum (the layout only grows with it)
+    size_t smem = 232448;
+    size_t q;
+    if (query_smem_optin(cfg->device, &q) == 0 && q > 0) smem = q;
+    Layout L;
+    compute_layout(cfg, smem, &L);
+    return L.total;
+}
+
+int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out) {
+    if (!out) return ATREX_ERR_INVALID;
+    *out = nullptr;
+    if (!config_ok(cfg) || !cfg->app_weights) return ATREX_ERR_INVALID;
+    if (cfg->workspace && ((uintptr_t)cfg->workspace % ALIGN) != 0) return ATREX_ERR_INVALID;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device < 0 || cfg->device >= n_dev) {
+        cudaGetLastError();
+        return ATREX_ERR_CUDA;
+    }
+    atrex_agg* h = new (std::nothrow) atrex_agg;
+    if (!h) return ATREX_ERR_NOMEM;
+    h->cfg = *cfg;
+    h->cfg.app_weights = nullptr;
+    DeviceGuard guard(cfg->device);
+    size_t smem = 0;
+    int rc = ATREX_OK;
+    do {
+        if (query_smem_optin(cfg->device, &smem) != 0) { rc = ATREX_ERR_CUDA; break; }
+        compute_layout(cfg, smem, &h->L);
+        if (cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) { rc = ATREX_ERR_CUDA; break; }
+        if (cfg->workspace) {
+            if (cfg->workspace_bytes < h->L.total) { rc = ATREX_ERR_NOMEM; break; }
+            h->ws = (unsigned char*)cfg->workspace;
+        } else {
+            if (cudaMalloc((void**)&h->ws, h->L.total) != cudaSuccess) { cudaGetLastError(); rc = ATREX_ERR_NOMEM; break; }
+            h->owns_workspace = true;
+        }
+        const Layout& L = h->L;
+        h->ctl = (Control*)(h->ws + L.off_ctl);
+        h->table = (Slot*)(h->ws + L.off_table);
+        h->work = (WorkSlot*)(h->ws + L.off_work);
+        h->d_appw = (uint32_t*)(h->ws + L.off_appw);
+        h->hot_keys = (ull*)(h->ws + L.off_hot);
+        h->staging[0] = h->ws + L.off_staging[0];
+        h->staging[1] = h->ws + L.off_staging[1];
+        h->sel = (ull*)(h->ws + L.off_sel);
+        h->topk_out = (atrex_entry_t*)(h->ws + L.off_topk_out);
+        cudaError_t e = cudaSuccess;
+        if (e == cudaSuccess) e = cudaMemset(h->ws + L.off_ctl, 0, L.off_appw - L.off_ctl);  // control, table, work
+        if (e == cudaSuccess) e = cudaMemcpy(h->d_appw, cfg->app_weights, (size_t)cfg->n_apps * 4, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemset(h->hot_keys, 0, (size_t)(L.hot_slots ? L.hot_slots : 2) * 8);
+        if (e == cudaSuccess) e = cudaHostAlloc((void**)&h->h_ctl, sizeof(Control), cudaHostAllocDefault);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
+        for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+            e = cudaEventCreateWithFlags(&h->ev_ready[i], cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->ev_free[i], cudaEventDisableTiming);
+        }
+        if (e == cudaSuccess) e = ingest_prepare();
+        if (e == cudaSuccess) e = finalize_prepare();
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) { h->last_cuda_error = (int)e; rc = ATREX_ERR_CUDA; break; }
+    } while (0);
+    if (rc != ATREX_OK) {
+        atrex_agg_destroy(h);
+        return rc;
+    }
+    *out = h;
+    return ATREX_OK;
+}
+
+void atrex_agg_destroy(atrex_agg_t* h) {
+    if (!h) return;
+    DeviceGuard guard(h->cfg.device);
+    cudaDeviceSynchronize();
+    for (int i = 0; i < 2; ++i) {
+        if (h->ev_ready[i]) cudaEventDestroy(h->ev_ready[i]);
+        if (h->ev_free[i]) cudaEventDestroy(h->ev_free[i]);
+    }
+    if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+    if (h->h_ctl) cudaFreeHost(h->h_ctl);
+    if (h->owns_workspace && h->ws) cudaFree(h->ws);
+    delete h;
+}
+
+int atrex_agg_reset(atrex_agg_t* h, void* stream) {
+    if (!h) return ATREX_ERR_INVALID;
+    DeviceGuard guard(h->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    CU(h, cudaMemsetAsync(h->ctl, 0, sizeof(Control), s));
+    CU(h, cudaMemsetAsync(h->table, 0, h->L.n_slots * sizeof(Slot), s));
+    h->hot_ready = false;
+    h->finalized = false;
+    h->n_records = 0;
+    return ATREX_OK;
+}
+
+int atrex_agg_set_work_table(atrex_agg_t* h, const atrex_work_t* rows, uint64_t n, void* stream) {
+    if (!h || (n && !rows) || n > h->cfg.max_work_rows) return ATREX_ERR_INVALID;
+    DeviceGuard guard(h->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (h->L.work_slots == 0) return ATREX_OK;
+    CU(h, cudaMemsetAsync(h->work, 0, h->L.work_slots * sizeof(WorkSlot), s));
+    CU(h, cudaMemsetAsync(&h->ctl->work_status, 0, sizeof(ull), s));
+    const uint64_t per_piece = STAGING_BYTES / sizeof(atrex_work_t);
+    for (uint64_t off = 0; off < n; off += per_piece) {
+        uint64_t m = n - off < per_piece ? n - off : per_piece;
+        CU(h, cudaMemcpyAsync(h->staging[0], rows + off, m * sizeof(atrex_work_t), cudaMemcpyHostToDevice, s));
+        CU(h, launch_work_insert((const atrex_work_t*)h->staging[0], m, h->work_ref(), h->ctl, h->scan_grid(m, 256), s));
+        h->launches++;
+        CU(h, cudaStreamSynchronize(s));  // the staging buffer and the host rows are reused
+    }
+    CU(h, cudaMemcpyAsync(h->h_ctl, h->ctl, sizeof(Control), cudaMemcpyDeviceToHost, s));
+    CU(h, cudaStreamSynchronize(s));
+    h->finalized = false;
+    if (h->h_ctl->work_status != 0) {
+        CU(h, cudaMemsetAsync(h->work, 0, h->L.work_slots * sizeof(WorkSlot), s));
+        CU(h, cudaStreamSynchronize(s));
+        return ATREX_ERR_INVALID;
+    }
+    return ATREX_OK;
+}
+
+static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, cudaStream_t s) {
+    // hot directory from a sample of the first sufficiently large call after create/reset
+    if (h->L.hot_slots && !h->hot_ready && n >= HOT_MIN_RECORDS) {
+        HotBuildParams b;
+        b.recs = (const uint4*)recs;
+        b.n_sample = (uint32_t)(n < HOT_SAMPLE ? n : HOT_SAMPLE);
+        b.stride = n / b.n_sample;
+        b.n_apps = h->cfg.n_apps;
+        b.n_phases = h->cfg.n_phases;
+        b.hot_keys = h->hot_keys;
+        b.hot_slots = h->L.hot_slots;
+        b.ctl = h->ctl;
+        CU(h, launch_hot_build(b, s));
+        h->launches++;
+        h->hot_ready = true;
+    }
+    IngestParams p;
+    memset(&p, 0, sizeof(p));
+    const unsigned char* base = (const unsigned char*)recs;
+    uint64_t head = (((uintptr_t)base & 31u) != 0 && n > 0) ? 1 : 0;
+    uint64_t n_body = n - head;
+    p.body = base + head * 16;
+    p.n_pairs = n_body / 2;
+    p.n_single = 0;
+    if (head) p.single[p.n_single++] = base;
+    if (n_body & 1) p.single[p.n_single++] = base + (n - 1) * 16;
+    p.n_apps = h->cfg.n_apps;
+    p.n_phases = h->cfg.n_phases;
+    p.appw_in_smem = h->L.appw_in_smem ? 1u : 0u;
+    p.app_w = h->d_appw;
+    p.hot_keys = h->hot_keys;
+    p.hot_slots = h->L.hot_slots;
+    p.hot_buckets = h->L.hot_slots / 2;
+    p.t = h->table_ref();
+    const ull pairs_per_cta_iter = 2048;
+    ull want = (p.n_pairs + pairs_per_cta_iter - 1) / pairs_per_cta_iter;
+    int grid = (int)(want < 1 ? 1 : (want > (ull)h->n_sms ? (ull)h->n_sms : want));
+    CU(h, launch_ingest(p, h->hot_ready, grid, s));
+    h->launches++;
+    return ATREX_OK;
+}
+
+int atrex_agg_ingest(atrex_agg_t* h, const atrex_record_t* d_records, uint64_t n, void* stream) {
+    if (!h) return ATREX_ERR_INVALID;
+    if (n == 0) return ATREX_OK;
+    if (!d_records || ((uintptr_t)d_records & 15u) != 0) return ATREX_ERR_INVALID;
+    if (h->n_records + n >= MAX_RECORDS_TOTAL) return ATREX_ERR_STATE;
+    DeviceGuard guard(h->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    h->finalized = false;
+    for (uint64_t off = 0; off < n; off += MAX_RECORDS_PER_LAUNCH) {
+        uint64_t m = n - off < MAX_RECORDS_PER_LAUNCH ? n - off : MAX_RECORDS_PER_LAUNCH;
+        int rc = ingest_launch(h, d_records + off, m, s);
+        if (rc != ATREX_OK) return rc;
+    }
+    h->n_records += n;
+    return ATREX_OK;
+}
+
+int atrex_agg_ingest_host(atrex_agg_t* h, const atrex_record_t* h_records, uint64_t n, void* stream) {
+    if (!h) return ATREX_ERR_INVALID;
+    if (n == 0) return ATREX_OK;
+    if (!h_records) return ATREX_ERR_INVALID;
+    if (h->n_records + n >= MAX_RECORDS_TOTAL) return ATREX_ERR_STATE;
+    DeviceGuard guard(h->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    h->finalized = false;
+    const uint64_t per_piece = STAGING_BYTES / sizeof(atrex_record_t);
+    int b = 0;
+    for (uint64_t off = 0; off < n; off += per_piece, b ^= 1) {
+        uint64_t m = n - off < per_piece ? n - off : per_piece;
+        CU(h, cudaStreamWaitEvent(h->copy_stream, h->ev_free[b], 0));
+        CU(h, cudaMemcpyAsync(h->staging[b], h_records + off, m * sizeof(atrex_record_t), cudaMemcpyHostToDevice, h->copy_stream));
+        CU(h, cudaEventRecord(h->ev_ready[b], h->copy_stream));
+        CU(h, cudaStreamWaitEvent(s, h->ev_ready[b], 0));
+        int rc = ingest_launch(h, (const atrex_record_t*)h->staging[b], m, s);
+        if (rc != ATREX_OK) return rc;
+        CU(h, cudaEventRecord(h->ev_free[b], s));
+    }
+    h->n_records += n;
+    return ATREX_OK;
+}
+
+int atrex_agg_merge(atrex_agg_t* h, const atrex_entry_t* d_entries, uint64_t n, void* stream) {
+    if (!h) return ATREX_ERR_INVALID;
+    if (n == 0) return ATREX_OK;
+    if (!d_entries || ((uintptr_t)d_entries & 15u) != 0) return ATREX_ERR_INVALID;
+    DeviceGuard guard(h->cfg.device);
+    h->finalized = false;
+    CU(h, launch_merge(d_entries, n, h->table_ref(), h->scan_grid(n, 256), (cudaStream_t)stream));
+    h->launches++;
+    return ATREX_OK;
+}
+
+static int run_totals(atrex_agg* h, cudaStream_t s) {
+    size_t off = offsetof(Control, total_lo);
+    CU(h, cudaMemsetAsync((unsigned char*)h->ctl + off, 0, offsetof(Control, hist) - off, s));
+    CU(h, launch_totals(h->table, h->L.n_slots, h->ctl, h->scan_grid(h->L.n_slots, 128 * 8), s));
+    h->launches++;
+    return ATREX_OK;
+}
+
+static FinalizeParams finalize_params(const atrex_agg* h, atrex_entry_t* out, uint64_t cap) {
+    FinalizeParams p;
+    p.table = h->table;
+    p.n_slots = h->L.n_slots;
+    p.ctl = h->ctl;
+    p.work = h->work_ref();
+    p.peaks = h->peaks;
+    p.out = out;
+    p.out_cap = cap;
+    return p;
+}
+
+int atrex_agg_finalize(atrex_agg_t* h, const atrex_hw_peaks_t* peaks, atrex_entry_t* d_out, uint64_t out_cap,
+                       uint64_t* n_out, void* stream) {
+    if (!h || !peaks || !n_out) return ATREX_ERR_INVALID;
+    if (d_out && ((uintptr_t)d_out & 15u) != 0) return ATREX_ERR_INVALID;
+    if (!d_out) out_cap = 0;
+    if (!(std::isfinite(peaks->peak_bw) && peaks->peak_bw > 0)) return ATREX_ERR_INVALID;
+    for (int i = 0; i < ATREX_MAX_DTYPES; ++i)
+        if (!(std::isfinite(peaks->peak_flops[i]) && peaks->peak_flops[i] > 0)) return ATREX_ERR_INVALID;
+    DeviceGuard guard(h->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    h->peaks = *peaks;
+    int rc = run_totals(h, s);
+    if (rc != ATREX_OK) return rc;
+    CU(h, cudaMemsetAsync(&h->ctl->n_out, 0, sizeof(ull), s));
+    CU(h, launch_emit(finalize_params(h, d_out, out_cap), h->scan_grid(h->L.n_slots, 256 * 4), s));
+    h->launches++;
+    CU(h, cudaMemcpyAsync(h->h_ctl, h->ctl, offsetof(Control, hist), cudaMemcpyDeviceToHost, s));
+    CU(h, cudaStreamSynchronize(s));
+    *n_out = h->h_ctl->n_out;
+    rc = device_status_to_error(h->h_ctl);
+    if (rc != ATREX_OK) return rc;
+    h->finalized = true;
+    if (d_out && h->h_ctl->n_out > out_cap) return ATREX_ERR_OUT_TOO_SMALL;
+    return ATREX_OK;
+}
+
+int atrex_agg_topk(atrex_agg_t* h, uint32_t phase, uint32_t k, atrex_entry_t* h_out, uint32_t* n_out, void* stream) {
+    if (!h || !n_out || (k && !h_out) || k > ATREX_MAX_TOPK || phase >= h->cfg.n_phases) return ATREX_ERR_INVALID;
+    *n_out = 0;
+    if (!h->finalized) return ATREX_ERR_STATE;
+    if (k == 0) return ATREX_OK;
+    DeviceGuard guard(h->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    const ull n_phase = h->h_ctl->keys_per_phase[phase];
+    if (n_phase == 0) return ATREX_OK;
+
+    TopkParams p;
+    memset(&p, 0, sizeof(p));
+    p.table = h->table;
+    p.n_slots = h->L.n_slots;
+    p.ctl = h->ctl;
+    p.phase = phase;
+    p.sel = h->sel;
+    p.sel_cap = SEL_CAP;
+    const int grid = h->scan_grid(h->L.n_slots, 256 * 4);
+    ull total;
+    if (n_phase <= k) {
+        p.collect_all = 1;
+        total = n_phase;
+    } else {
+        // most-significant-digit radix select on the ranking composite
+        ull need = k, cand = 0;
+        uint32_t* hist = h->h_ctl->hist;
+        while (true) {
+            CU(h, cudaMemsetAsync(h->ctl->hist, 0, sizeof(h->ctl->hist), s));
+            CU(h, launch_topk_hist(p, grid, s));
+            h->launches++;
+            CU(h, cudaMemcpyAsync(hist, h->ctl->hist, sizeof(h->ctl->hist), cudaMemcpyDeviceToHost, s));
+            CU(h, cudaStreamSynchronize(s));
+            ull above = 0;
+            int bin = TOPK_BINS - 1;
+            for (; bin > 0; --bin) {
+                if (above + hist[bin] >= need) break;
+                above += hist[bin];
+            }
+            need -= above;
+            cand = hist[bin];
+            p.prefix_digit[p.n_prefix_digits++] = (uint16_t)bin;
+            if (cand <= TOPK_CAND_CAP || p.n_prefix_digits == (uint32_t)TOPK_DIGITS) break;
+        }
+        total = (k - need) + cand;
+    }
+    if (total > SEL_CAP) return ATREX_ERR_STATE;  // cannot happen: composites are unique
+    uint32_t n_pow2 = (uint32_t)pow2_at_least(total < 2 ? 2 : total);
+    CU(h, cudaMemsetAsync(&h->ctl->sel_count, 0, sizeof(ull), s));
+    CU(h, cudaMemsetAsync(h->sel, 0, (size_t)n_pow2 * 32, s));
+    CU(h, launch_topk_collect(p, grid, s));
+    CU(h, launch_topk_sort(h->sel, n_pow2, s));
+    uint32_t m = (uint32_t)(total < k ? total : k);
+    CU(h, launch_topk_emit(finalize_params(h, h->topk_out, m), h->sel, m, s));
+    h->launches += 3;
+    CU(h, cudaMemcpyAsync(h_out, h->topk_out, (size_t)m * sizeof(atrex_entry_t), cudaMemcpyDeviceToHost, s));
+    CU(h, cudaStreamSynchronize(s));
+    *n_out = m;
+    return ATREX_OK;
+}
+
+int atrex_agg_stats(atrex_agg_t* h, atrex_stats_t* out, void* stream) {
+    if (!h || !out) return ATREX_ERR_INVALID;
+    DeviceGuard guard(h->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    int rc = run_totals(h, s);
+    if (rc != ATREX_OK) return rc;
+    CU(h, cudaMemcpyAsync(h->h_ctl, h->ctl, offsetof(Control, hist), cudaMemcpyDeviceToHost, s));
+    CU(h, cudaStreamSynchronize(s));
+    memset(out, 0, sizeof(*out));
+    const Control* c = h->h_ctl;
+    out->n_rejected = c->n_rejected;
+    out->n_dropped = c->n_dropped;
+    for (int p = 0; p < ATREX_MAX_PHASES; ++p) {
+        out->total_lo[p] = c->total_lo[p];
+        out->total_hi[p] = c->total_hi[p];
+        out->keys_per_phase[p] = c->keys_per_phase[p];
+        out->n_keys += c->keys_per_phase[p];
+        out->n_valid += c->count_per_phase[p];
+    }
+    out->table_slots = h->L.n_slots;
+    out->hot_slots = c->hot_n;
+    return device_status_to_error(c);
+}
+
+const char* atrex_strerror(int status) {
+    switch (status) {
+        case ATREX_OK: return "ok";
+        case ATREX_ERR_INVALID: return "invalid argument";
+        case ATREX_ERR_CAPACITY: return "more distinct keys than provisioned";
+        case ATREX_ERR_OUT_TOO_SMALL: return "output buffer too small";
+        case ATREX_ERR_CUDA: return "CUDA runtime error";
+        case ATREX_ERR_TIMEOUT: return "bounded device wait gave up";
+        case ATREX_ERR_STATE: return "call not valid in this state";
+        case ATREX_ERR_NOMEM: return "workspace too small or allocation failed";
+        default: return "unknown status";
+    }
+}
+
+int atrex_agg_last_cuda_error(const atrex_agg_t* h) { return h ? h->last_cuda_error : 0; }
+
+uint64_t atrex_agg_launch_count(const atrex_agg_t* h) { return h ? h->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,76 @@
+// Kernel parameter blocks and host-side launchers (internal to the library).
+#pragma once
+#include "atrex_dev.cuh"
+
+namespace atrex {
+
+struct IngestParams {
+    const void* body;          // first record of the 32-byte aligned run of record pairs
+    ull n_pairs;               // pairs in the body
+    const void* single[2];     // records outside the body (unaligned head, odd tail)
+    uint32_t n_single;
+    uint32_t n_apps, n_phases;
+    uint32_t appw_in_smem;
+    const uint32_t* app_w;     // device copy of the card-hour weights
+    const ull* hot_keys;       // directory image, hot_slots entries of ~key (0 = empty)
+    uint32_t hot_slots;        // even
+    uint32_t hot_buckets;      // hot_slots / 2
+    TableRef t;
+};
+
+struct HotBuildParams {
+    const uint4* recs;
+    ull stride;
+    uint32_t n_sample;
+    uint32_t n_apps, n_phases;
+    ull* hot_keys;
+    uint32_t hot_slots;
+    Control* ctl;
+};
+
+struct WorkRef {
+    WorkSlot* table;
+    ull mask;
+    int shift;
+    uint32_t max_probe;
+};
+
+struct FinalizeParams {
+    const Slot* table;
+    ull n_slots;
+    Control* ctl;
+    WorkRef work;
+    atrex_hw_peaks_t peaks;
+    atrex_entry_t* out;
+    ull out_cap;
+};
+
+struct TopkParams {
+    const Slot* table;
+    ull n_slots;
+    Control* ctl;
+    uint32_t phase;
+    uint32_t n_prefix_digits;   // leading 12-bit digits of the ranking composite already fixed
+    uint16_t prefix_digit[12];  // their values, most significant first
+    int collect_all;
+    ull* sel;                   // [sel_cap][4]: composite words 2,1,0 and the slot index
+    uint32_t sel_cap;
+};
+
+size_t ingest_smem_bytes(bool hot, uint32_t hot_slots, uint32_t n_apps, bool appw_in_smem);
+cudaError_t ingest_prepare();
+cudaError_t launch_ingest(const IngestParams& p, bool hot, int grid, cudaStream_t stream);
+cudaError_t launch_hot_build(const HotBuildParams& p, cudaStream_t stream);
+cudaError_t launch_merge(const atrex_entry_t* in, ull n, const TableRef& t, int grid, cudaStream_t stream);
+
+cudaError_t finalize_prepare();
+cudaError_t launch_totals(const Slot* table, ull n_slots, Control* ctl, int grid, cudaStream_t stream);
+cudaError_t launch_emit(const FinalizeParams& p, int grid, cudaStream_t stream);
+cudaError_t launch_work_insert(const atrex_work_t* rows, ull n, const WorkRef& w, Control* ctl, int grid,
+                               cudaStream_t stream);
+cudaError_t launch_topk_hist(const TopkParams& p, int grid, cudaStream_t stream);
+cudaError_t launch_topk_collect(const TopkParams& p, int grid, cudaStream_t stream);
+cudaError_t launch_topk_sort(ull* sel, uint32_t n_pow2, cudaStream_t stream);
+cudaError_t launch_topk_emit(const FinalizeParams& p, const ull* sel, uint32_t n, cudaStream_t stream);
+
+}  // namespace atrex

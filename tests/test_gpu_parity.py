@@ -1,0 +1,328 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle: bit-exact on every
+field, on the same seeded inputs, for the five benchmark laws at sizes the oracle finishes
+in seconds (several CTA tiles plus a ragged tail), and on the edge cases."""
+import ctypes as C
+
+import numpy as np
+import pytest
+
+import oracle
+import tracegen as tg
+from tracegen.configs import make_spec
+from tracegen.layout import RECORD_DTYPE, WORK_DTYPE
+from tests.helpers import (load_golden, f64_bits, records_from_dicts, work_from_dicts, entry_wt, sorted_by_key)
+
+pytestmark = pytest.mark.gpu
+
+PEAK_BW = 8.0e12
+PEAK_FLOPS = [1.0e15, 2.0e15, 4.0e15, 5.0e14, 2.5e14, 1.0e15, 1.0e15, 1.0e15]
+
+
+@pytest.fixture(scope="module")
+def lib():
+    import paper_2607_14541_b200 as p
+    return p
+
+
+def to_dev(recs: np.ndarray, misalign: bool = False):
+    import torch
+    raw = torch.from_numpy(np.ascontiguousarray(recs).view(np.uint8).reshape(-1))
+    if misalign:  # 16-byte aligned but not 32-byte aligned start
+        buf = torch.empty(raw.numel() + 64, dtype=torch.uint8, device="cuda:0")
+        off = 16 if buf.data_ptr() % 32 == 0 else 0
+        view = buf[off: off + raw.numel()]
+        view.copy_(raw)
+        assert view.data_ptr() % 32 == 16
+        return view
+    return raw.cuda()
+
+
+def gpu_aggregate(lib, recs, app_weights, n_phases, work=None, max_keys=None, chunks=1, flags=0, misalign=False,
+                  host=False):
+    n_keys_bound = max_keys or max(len(recs), 16)
+    agg = lib.Aggregator(app_weights, n_phases, n_keys_bound, max_work_rows=0 if work is None else len(work), flags=flags)
+    if work is not None:
+        agg.set_work_table(work)
+    for c in np.array_split(recs, chunks):
+        if host:
+            agg.ingest_host(c)
+        else:
+            agg.ingest(to_dev(c, misalign), n=len(c))
+    return agg
+
+
+def assert_same_as_oracle(agg, o, n_phases, ks=(1, 10)):
+    got = sorted_by_key(agg.finalize_numpy(PEAK_BW, PEAK_FLOPS))
+    exp = o.finalize(PEAK_BW, PEAK_FLOPS)
+    assert len(got) == len(exp)
+    assert got.tobytes() == exp.tobytes()          # every field, bit for bit
+    st, so = agg.stats(), o.stats()
+    assert st["n_valid"] == so["n_valid"] and st["n_rejected"] == so["n_rejected"] and st["n_keys"] == so["n_keys"]
+    assert st["totals"] == so["totals"] and st["n_dropped"] == 0
+    for phase in range(n_phases):
+        for k in ks:
+            assert agg.topk(phase, k).tobytes() == o.topk(PEAK_BW, PEAK_FLOPS, phase, k).tobytes(), (phase, k)
+    return got
+
+
+def oracle_of(recs, app_weights, n_phases, work=None, threads=4):
+    o = oracle.Oracle(app_weights, n_phases)
+    if work is not None:
+        assert o.set_work(work) == 0
+    o.ingest(recs, threads=threads)
+    return o
+
+
+# ---------------------------------------------------------------- the five laws
+
+CASES = [
+    # index, small key domain, n (odd sizes leave a ragged tail), chunks
+    (0, False, 1 << 20, 1),
+    (1, False, (1 << 22) + 12345, 1),
+    (2, True, (1 << 22) + 1, 1),
+    (3, True, (1 << 23) + 777, 8),
+    (4, True, (1 << 22) + 3, 1),
+]
+
+
+@pytest.mark.parametrize("index,small,n,chunks", CASES)
+def test_parity_five_configs(lib, index, small, n, chunks):
+    spec = make_spec(index, small=small, n=n, n_dtypes=3)
+    recs = tg.generate(spec)
+    work = spec.work_table()
+    o = oracle_of(recs, spec.app_weights, spec.n_phases, work)
+    agg = gpu_aggregate(lib, recs, spec.app_weights, spec.n_phases, work, max_keys=spec.max_keys, chunks=chunks)
+    got = assert_same_as_oracle(agg, o, spec.n_phases, ks=(1, spec.topk, 4096))
+    assert agg.stats()["hot_slots"] > 0            # the shared-memory stage was active
+    if index == 4:  # the u128 carry path was exercised
+        assert int(got["wt_hi"].max()) >= 1
+    if chunks > 1:  # chunked == single pass
+        agg1 = gpu_aggregate(lib, recs, spec.app_weights, spec.n_phases, work, max_keys=spec.max_keys, chunks=1)
+        assert sorted_by_key(agg1.finalize_numpy(PEAK_BW, PEAK_FLOPS)).tobytes() == got.tobytes()
+
+
+@pytest.mark.parametrize("index", [1, 4])
+def test_parity_without_hot_directory_and_misaligned_start(lib, index):
+    spec = make_spec(index, small=True, n=(1 << 20) + 5)
+    recs = tg.generate(spec)
+    o = oracle_of(recs, spec.app_weights, spec.n_phases)
+    agg = gpu_aggregate(lib, recs, spec.app_weights, spec.n_phases, max_keys=spec.max_keys,
+                        flags=lib.ATREX_FLAG_NO_HOT_DIRECTORY)
+    assert_same_as_oracle(agg, o, spec.n_phases)
+    assert agg.stats()["hot_slots"] == 0
+    agg = gpu_aggregate(lib, recs, spec.app_weights, spec.n_phases, max_keys=spec.max_keys, misalign=True, chunks=3)
+    assert_same_as_oracle(agg, o, spec.n_phases)
+
+
+def test_host_ingest_equals_device_ingest(lib):
+    spec = make_spec(1, small=True, n=(1 << 23) + 9)   # > one 64 MiB staging piece
+    recs = tg.generate(spec)
+    o = oracle_of(recs, spec.app_weights, spec.n_phases)
+    agg = gpu_aggregate(lib, recs, spec.app_weights, spec.n_phases, max_keys=spec.max_keys, host=True)
+    assert_same_as_oracle(agg, o, spec.n_phases)
+
+
+def test_permutation_and_many_small_calls(lib):
+    spec = make_spec(3, small=True, n=200_001)
+    recs = tg.generate(spec)
+    o = oracle_of(recs, spec.app_weights, spec.n_phases)
+    perm = np.random.default_rng(3).permutation(len(recs))
+    agg = gpu_aggregate(lib, recs[perm], spec.app_weights, spec.n_phases, max_keys=spec.max_keys, chunks=37)
+    assert_same_as_oracle(agg, o, spec.n_phases)
+
+
+def test_merge_of_partial_aggregates_equals_whole(lib):
+    import torch
+    spec = make_spec(2, small=True, n=1 << 20)
+    recs = tg.generate(spec)
+    o = oracle_of(recs, spec.app_weights, spec.n_phases)
+    a = gpu_aggregate(lib, recs[: 400_000], spec.app_weights, spec.n_phases, max_keys=spec.max_keys)
+    b = gpu_aggregate(lib, recs[400_000:], spec.app_weights, spec.n_phases, max_keys=spec.max_keys)
+    part, n = b.finalize(PEAK_BW, PEAK_FLOPS)
+    a.merge(part, n)
+    assert_same_as_oracle(a, o, spec.n_phases)
+
+
+# ---------------------------------------------------------------- hand-computed traces on the GPU
+
+def test_worked_example_a_on_gpu(lib, golden_dir):
+    g = load_golden(golden_dir, "worked_example_a.json")
+    recs, work = records_from_dicts(g["records"]), work_from_dicts(g["work"])
+    agg = lib.Aggregator(g["app_weights"], g["n_phases"], 64, max_work_rows=8)
+    agg.set_work_table(work)
+    agg.ingest(to_dev(recs), n=len(recs))
+    ent = sorted_by_key(agg.finalize_numpy(g["peak_bw"], g["peak_flops"] + [1.0] * 7))
+    assert len(ent) == 4
+    for e, x in zip(ent, g["expected"]):
+        assert int(e["key"]) == int(x["key"], 16) and int(e["count"]) == x["count"] and entry_wt(e) == x["wt"]
+        assert f64_bits(float(e["phase_weight"])) == int(x["phase_weight_bits"], 16)
+        assert f64_bits(float(e["roofline_s"])) == int(x["roofline_bits"], 16)
+    for t in g["topk"]:
+        assert [int(k) for k in agg.topk(t["phase"], t["k"])["key"]] == [int(k, 16) for k in t["keys"]]
+
+
+def test_carry_closed_form_on_gpu(lib, golden_dir):
+    g = load_golden(golden_dir, "carry_closed_form.json")
+    for case in g["cases"]:
+        n = case["N"]
+        recs = np.zeros(n, dtype=RECORD_DTYPE)
+        recs["op_id"], recs["shape_id"], recs["phase"], recs["duration_ns"] = 3, 11, 1, g["duration_ns"]
+        for flags in (0, lib.ATREX_FLAG_NO_HOT_DIRECTORY):
+            agg = lib.Aggregator([g["weight"]], 2, 16, flags=flags)
+            agg.ingest(to_dev(recs), n=n)
+            ent = agg.finalize_numpy(PEAK_BW, PEAK_FLOPS)
+            assert len(ent) == 1 and int(ent[0]["count"]) == n
+            assert int(ent[0]["wt_hi"]) == case["wt_hi"] and int(ent[0]["wt_lo"]) == int(case["wt_lo"], 16)
+            assert float(ent[0]["phase_weight"]) == 1.0
+
+
+def test_topk_ties_on_gpu(lib, golden_dir):
+    g = load_golden(golden_dir, "topk_ties.json")
+    c = g["case_rounding"]
+    rows = []
+    for name in ("x", "y"):
+        k = c[name]
+        rows += [{"app": 0, "op": k["op"], "shape": k["shape"], "duration_ns": k["big_duration"]}] * k["n_big"]
+        if "extra_duration" in k:
+            rows.append({"app": 1, "op": k["op"], "shape": k["shape"], "duration_ns": k["extra_duration"]})
+    recs = records_from_dicts(rows)
+    agg = lib.Aggregator(c["app_weights"], 1, 16)
+    agg.ingest(to_dev(recs), n=len(recs))
+    agg.finalize(PEAK_BW, PEAK_FLOPS)
+    assert [int(k) for k in agg.topk(0, 2)["key"]] == [int(k, 16) for k in c["top2_keys"]]
+    t = g["case_exact_ties"]
+    recs = records_from_dicts(t["records"])
+    agg = lib.Aggregator(t["app_weights"], 1, 16)
+    agg.ingest(to_dev(recs), n=len(recs))
+    agg.finalize(PEAK_BW, PEAK_FLOPS)
+    assert [int(k) for k in agg.topk(0, 3)["key"]] == [int(k, 16) for k in t["top3_keys"]]
+    assert [int(k) for k in agg.topk(0, 9)["key"]] == [int(k, 16) for k in t["top4_keys"]]
+
+
+def test_topk_with_a_huge_tie_class_needs_deeper_digits(lib):
+    # 150k keys with identical weighted time: the candidate class exceeds the sorter's
+    # capacity until the radix select reaches the key digits
+    n = 150_000
+    recs = np.zeros(n, dtype=RECORD_DTYPE)
+    recs["op_id"] = np.arange(n) % 50
+    recs["shape_id"] = np.arange(n) // 50 + 17
+    recs["duration_ns"] = 5000
+    recs = np.concatenate([recs, recs[:3]])          # three keys get twice the weight
+    o = oracle_of(recs, [9], 1)
+    agg = lib.Aggregator([9], 1, 1 << 18)
+    agg.ingest(to_dev(recs), n=len(recs))
+    agg.finalize(PEAK_BW, PEAK_FLOPS)
+    for k in (1, 3, 4, 100, 70_000 if False else 65_536):
+        assert agg.topk(0, k).tobytes() == o.topk(PEAK_BW, PEAK_FLOPS, 0, k).tobytes(), k
+
+
+# ---------------------------------------------------------------- edge cases and errors
+
+def test_empty_single_and_invalid_records(lib):
+    agg = lib.Aggregator([3, 5], 2, 64)
+    assert len(agg.finalize_numpy(PEAK_BW, PEAK_FLOPS)) == 0
+    assert len(agg.topk(0, 5)) == 0
+    import torch
+    agg.ingest(torch.empty(0, dtype=torch.uint8, device="cuda:0"), n=0)
+    recs = records_from_dicts([{"app": 1, "op": 2, "shape": 3, "phase": 1, "duration_ns": 10}])
+    agg.ingest(to_dev(recs), n=1)
+    ent = agg.finalize_numpy(PEAK_BW, PEAK_FLOPS)
+    assert len(ent) == 1 and int(ent[0]["key"]) == (1 << 48) | (2 << 32) | 3 and entry_wt(ent[0]) == 50
+    assert f64_bits(float(ent[0]["roofline_s"])) == 0x7FF8000000000000
+    bad = records_from_dicts([{"app": 2, "op": 1, "shape": 1, "duration_ns": 1},
+                              {"app": 0xFFFFFFFF, "op": 1, "shape": 1, "duration_ns": 1},
+                              {"app": 0, "op": 1, "shape": 1, "phase": 2, "duration_ns": 1},
+                              {"app": 0, "op": 1, "shape": 1, "phase": 255, "duration_ns": 1}])
+    bad["pad"] = 0x5A
+    agg.ingest(to_dev(bad), n=4)
+    st = agg.stats()
+    assert st["n_rejected"] == 4 and st["n_valid"] == 1 and st["n_keys"] == 1
+    # zero weight / zero duration: counted, total stays zero, weight +0.0
+    agg = lib.Aggregator([0, 7], 2, 64)
+    z = records_from_dicts([{"app": 0, "op": 1, "shape": 1, "duration_ns": 99},
+                            {"app": 1, "op": 1, "shape": 2, "duration_ns": 0}])
+    agg.ingest(to_dev(z), n=2)
+    ent = sorted_by_key(agg.finalize_numpy(PEAK_BW, PEAK_FLOPS))
+    assert [int(c) for c in ent["count"]] == [1, 1] and all(f64_bits(float(x)) == 0 for x in ent["phase_weight"])
+
+
+def test_finalize_is_repeatable_and_peaks_only_change_the_roofline(lib):
+    spec = make_spec(0, n=100_000, n_dtypes=3)
+    recs, work = tg.generate(spec), spec.work_table()
+    agg = gpu_aggregate(lib, recs[:50_000], spec.app_weights, spec.n_phases, work, max_keys=spec.max_keys)
+    first = sorted_by_key(agg.finalize_numpy(PEAK_BW, PEAK_FLOPS))
+    again = sorted_by_key(agg.finalize_numpy(PEAK_BW, PEAK_FLOPS))
+    assert first.tobytes() == again.tobytes()
+    other = sorted_by_key(agg.finalize_numpy(2 * PEAK_BW, [2 * x for x in PEAK_FLOPS]))
+    assert np.array_equal(other["phase_weight"], first["phase_weight"])
+    assert np.array_equal(other["roofline_s"], first["roofline_s"] / 2)
+    agg.ingest(to_dev(recs[50_000:]), n=50_000)       # refresh: keep ingesting after a finalize
+    o = oracle_of(recs, spec.app_weights, spec.n_phases, work)
+    assert_same_as_oracle(agg, o, spec.n_phases)
+    agg.reset()
+    assert len(agg.finalize_numpy(PEAK_BW, PEAK_FLOPS)) == 0 and agg.stats()["n_rejected"] == 0
+    agg.ingest(to_dev(recs), n=len(recs))
+    assert_same_as_oracle(agg, o, spec.n_phases)
+
+
+def test_error_codes(lib):
+    import torch
+    p = lib
+    # capacity: far more distinct keys than provisioned -> ATREX_ERR_CAPACITY, no hang
+    n = 60_000
+    recs = np.zeros(n, dtype=RECORD_DTYPE)
+    recs["shape_id"] = np.arange(n)
+    recs["duration_ns"] = 1
+    agg = p.Aggregator([1], 1, 8)
+    agg.ingest(to_dev(recs), n=n)
+    with pytest.raises(p.AtrexError) as ei:
+        agg.finalize(PEAK_BW, PEAK_FLOPS)
+    assert ei.value.status == p.ATREX_ERR_CAPACITY
+    st = agg.stats(check=False)
+    assert st["status"] == p.ATREX_ERR_CAPACITY and st["n_dropped"] > 0
+    assert st["n_dropped"] + st["n_valid"] == n
+    # output buffer too small
+    agg = p.Aggregator([1], 1, 1 << 17)
+    agg.ingest(to_dev(recs), n=n)
+    small = torch.empty(48 * 10, dtype=torch.uint8, device="cuda:0")
+    pk = p.make_peaks(PEAK_BW, PEAK_FLOPS)
+    n_out = C.c_uint64(0)
+    rc = p.atrex_agg_finalize(agg._h, C.byref(pk), small.data_ptr(), 10, C.byref(n_out), None)
+    assert rc == p.ATREX_ERR_OUT_TOO_SMALL and n_out.value == n
+    # invalid arguments
+    assert p.atrex_agg_ingest(agg._h, small.data_ptr() + 8, 1, None) == p.ATREX_ERR_INVALID
+    assert p.atrex_agg_ingest(agg._h, None, 1, None) == p.ATREX_ERR_INVALID
+    bad = p.make_peaks(0.0, PEAK_FLOPS)
+    assert p.atrex_agg_finalize(agg._h, C.byref(bad), None, 0, C.byref(n_out), None) == p.ATREX_ERR_INVALID
+    bad = p.make_peaks(PEAK_BW, [float("nan")] * 8)
+    assert p.atrex_agg_finalize(agg._h, C.byref(bad), None, 0, C.byref(n_out), None) == p.ATREX_ERR_INVALID
+    out = np.zeros(4, dtype=p.ENTRY_DTYPE)
+    k_out = C.c_uint32(0)
+    assert p.atrex_agg_topk(agg._h, 5, 1, out.ctypes.data, C.byref(k_out), None) == p.ATREX_ERR_INVALID
+    agg.ingest(to_dev(recs[:10]), n=10)
+    assert p.atrex_agg_topk(agg._h, 0, 1, out.ctypes.data, C.byref(k_out), None) == p.ATREX_ERR_STATE
+    cfg = p.atrex_agg_config_t()
+    cfg.n_apps, cfg.n_phases, cfg.max_keys = 1, 9, 8
+    h = C.c_void_p()
+    w = np.array([1], dtype=np.uint32)
+    cfg.app_weights = w.ctypes.data
+    assert p.atrex_agg_create(C.byref(cfg), C.byref(h)) == p.ATREX_ERR_INVALID
+    # duplicate work rows / bad dtype
+    agg = p.Aggregator([1], 1, 16, max_work_rows=4)
+    dup = work_from_dicts([{"op": 1, "shape": 2, "flops": 1, "bytes": 1}, {"op": 1, "shape": 2, "flops": 2, "bytes": 2}])
+    assert p.atrex_agg_set_work_table(agg._h, dup.ctypes.data, 2, None) == p.ATREX_ERR_INVALID
+    bad_dt = work_from_dicts([{"op": 1, "shape": 2, "dtype": 8, "flops": 1, "bytes": 1}])
+    assert p.atrex_agg_set_work_table(agg._h, bad_dt.ctypes.data, 1, None) == p.ATREX_ERR_INVALID
+    assert p.atrex_agg_set_work_table(agg._h, dup.ctypes.data, 5, None) == p.ATREX_ERR_INVALID
+
+
+def test_gpu_sampler_matches_numpy_sampler():
+    import torch
+    from tracegen.gpu import GpuSampler
+    for index in range(5):
+        spec = make_spec(index, small=True, n=300_001)
+        ref = tg.generate(spec, start=1000, count=200_001)
+        out = torch.empty(200_001 * 16, dtype=torch.uint8, device="cuda:0")
+        GpuSampler(spec).fill(out, start=1000, count=200_001)
+        torch.cuda.synchronize()
+        assert out.cpu().numpy().tobytes() == ref.tobytes(), index

@@ -283,3 +283,24 @@ def test_roofline_picks_the_larger_side_per_dtype():
     recs = records_from_dicts([{"op": 0, "shape": s, "duration_ns": 1} for s in (0, 1, 2)])
     _, ent = run_oracle(recs, [1], 1, w)
     assert [float(x) for x in ent["roofline_s"]] == [2.0, 3.0, 4.0]
+
+
+def test_filtered_and_direct_totals_agree_with_the_full_group_by():
+    spec = make_spec(3, small=True, n=1 << 16)
+    recs = tg.generate(spec)
+    recs[:3]["app_id"] = spec.n_apps  # a few invalid ones
+    o, ent = run_oracle(recs, spec.app_weights, spec.n_phases, spec.work_table())
+    groups, totals, rejected = brute_force(recs, spec.app_weights, spec.n_phases)
+    pick = ent["key"][:: max(1, len(ent) // 50)]
+    f = oracle.Oracle(spec.app_weights, spec.n_phases)
+    for c in np.array_split(recs, 3):
+        f.ingest_filtered(c, pick)
+    got = f.finalize(PEAK_BW, PEAK_FLOPS)
+    assert list(got["key"]) == sorted(int(k) for k in pick)
+    for e in got:
+        assert int(e["count"]) == groups[int(e["key"])][0] and entry_wt(e) == groups[int(e["key"])][1]
+    acc, valid = np.zeros(16, dtype=np.uint64), np.zeros(2, dtype=np.uint64)
+    for c in np.array_split(recs, 3):
+        f.direct_totals(c, acc, valid)
+    assert [int(acc[2 * p]) | (int(acc[2 * p + 1]) << 64) for p in range(8)] == totals
+    assert int(valid[0]) == len(recs) - 3 and int(valid[1]) == 3 == rejected
