@@ -119,6 +119,8 @@ typedef struct {
     uint64_t keys_per_phase[ATREX_MAX_PHASES];
     uint64_t table_slots;                 /* capacity of the key table                 */
     uint64_t hot_slots;                   /* keys currently in the shared-memory hot directory */
+    uint64_t n_spilled;                   /* records that went through the partition spill buffers */
+    uint64_t n_overflow;                  /* records that found their spill buffer full (slow exact path) */
 } atrex_stats_t;
 
 typedef struct atrex_agg atrex_agg_t;

@@ -56,7 +56,8 @@ class atrex_stats_t(C.Structure):
     _fields_ = [("n_valid", C.c_uint64), ("n_rejected", C.c_uint64), ("n_dropped", C.c_uint64),
                 ("n_keys", C.c_uint64), ("total_lo", C.c_uint64 * ATREX_MAX_PHASES),
                 ("total_hi", C.c_uint64 * ATREX_MAX_PHASES), ("keys_per_phase", C.c_uint64 * ATREX_MAX_PHASES),
-                ("table_slots", C.c_uint64), ("hot_slots", C.c_uint64)]
+                ("table_slots", C.c_uint64), ("hot_slots", C.c_uint64), ("n_spilled", C.c_uint64),
+                ("n_overflow", C.c_uint64)]
 
 
 def _load():
@@ -242,7 +243,7 @@ class Aggregator:
                 "n_keys": st.n_keys,
                 "totals": [int(st.total_lo[p]) | (int(st.total_hi[p]) << 64) for p in range(ATREX_MAX_PHASES)],
                 "keys_per_phase": [int(x) for x in st.keys_per_phase], "table_slots": st.table_slots,
-                "hot_slots": st.hot_slots}
+                "hot_slots": st.hot_slots, "n_spilled": st.n_spilled, "n_overflow": st.n_overflow}
 
     def reset(self, stream=None):
         self._check(atrex_agg_reset(self._h, self._stream(stream)), "atrex_agg_reset")

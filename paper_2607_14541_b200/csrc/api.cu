@@ -14,12 +14,13 @@ namespace {
 
 constexpr size_t ALIGN = 256;
 constexpr size_t STAGING_BYTES = 64ull << 20;          // per staging buffer (two of them)
-constexpr ull MAX_RECORDS_PER_LAUNCH = 1ull << 31;      // keeps per-CTA 32-bit counts from wrapping
+constexpr uint32_t LP_MIN = 8, LP_MAX = 12;             // 256 .. 4096 partitions
+constexpr ull MAX_KEYS = 1ull << 25;
 constexpr ull MAX_RECORDS_TOTAL = 1ull << 40;
 constexpr uint32_t HOT_MIN_RECORDS = 32768;             // smaller calls run without a directory
 constexpr uint32_t HOT_SAMPLE = 131072;
 constexpr uint32_t APPW_SMEM_MAX = 4096;
-constexpr uint32_t MAX_PROBE = 4096;
+constexpr uint32_t MAX_PROBE = 4096;                   // work-table probe bound
 constexpr uint32_t SEL_CAP = ATREX_MAX_TOPK + TOPK_CAND_CAP;
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -37,8 +38,12 @@ int log2_of(ull p) {
 }
 
 struct Layout {
-    size_t off_ctl, off_table, off_work, off_appw, off_hot, off_staging[2], off_sel, off_topk_out, total;
+    size_t off_ctl, off_keys, off_vals, off_work, off_appw, off_hot, off_staging[2], off_sel, off_topk_out,
+        off_spill_cnt, off_spill, total;
     ull n_slots, work_slots;
+    uint32_t lp, C;              // partitions = 1 << lp, slots per partition
+    uint32_t n_groups, cap;      // spill buffers: [P][n_groups][cap] entries
+    ull sub_launch;              // records per scatter + partition launch pair
     uint32_t hot_slots;
     bool appw_in_smem;
 };
@@ -46,22 +51,39 @@ struct Layout {
 bool config_ok(const atrex_agg_config_t* c) {
     if (!c) return false;
     if (c->n_apps == 0 || c->n_phases == 0 || c->n_phases > ATREX_MAX_PHASES) return false;
-    if (c->max_keys == 0 || c->max_keys > (1ull << 30)) return false;
+    if (c->max_keys == 0 || c->max_keys > MAX_KEYS) return false;
     if (c->max_work_rows > (1ull << 30)) return false;
     return true;
 }
 
-void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, Layout* L) {
-    L->n_slots = pow2_at_least(c->max_keys * 2 < 1024 ? 1024 : c->max_keys * 2);
+void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, Layout* L) {
+    // partition geometry: one partition's keys + per-launch accumulators (20 B per slot) must
+    // fit one SM's shared memory; provision 1.3 slots per key
+    const uint32_t c_max = (uint32_t)((smem_optin - 2048) / 20) & ~127u;
+    const ull need = c->max_keys + c->max_keys * 3 / 10 + 1;
+    L->lp = LP_MIN;
+    while (L->lp < LP_MAX && (need + (1ull << L->lp) - 1) / (1ull << L->lp) > c_max) ++L->lp;
+    ull per = (need + (1ull << L->lp) - 1) >> L->lp;
+    if (per > c_max) per = c_max;
+    if (per < 128) per = 128;
+    L->C = (uint32_t)((per + 31) / 32 * 32);
+    L->n_slots = (ull)L->C << L->lp;
+    L->n_groups = (uint32_t)n_sms;
+    L->sub_launch = c->max_keys >= (1ull << 21) ? (1ull << 27) : (c->max_keys >= (1ull << 16) ? (1ull << 25) : (1ull << 24));
+    ull per_buf = (L->sub_launch * 5 / 2) / (((ull)n_sms) << L->lp);
+    if (per_buf < 64) per_buf = 64;
+    L->cap = (uint32_t)((per_buf + 7) / 8 * 8);
     L->work_slots = c->max_work_rows ? pow2_at_least(c->max_work_rows * 2 < 1024 ? 1024 : c->max_work_rows * 2) : 0;
     L->appw_in_smem = c->n_apps <= APPW_SMEM_MAX;
     size_t appw_smem = L->appw_in_smem ? (size_t)c->n_apps * 4 : 0;
-    size_t budget = smem_optin > appw_smem + 2048 ? smem_optin - appw_smem - 2048 : 0;
+    size_t fixed = appw_smem + 2048 + ((size_t)4 << L->lp);
+    size_t budget = smem_optin > fixed ? smem_optin - fixed : 0;
     L->hot_slots = (uint32_t)(budget / 20) & ~1u;
     if (c->flags & ATREX_FLAG_NO_HOT_DIRECTORY) L->hot_slots = 0;
     size_t o = 0;
     L->off_ctl = o;            o += round_up(sizeof(Control), ALIGN);
-    L->off_table = o;          o += round_up(L->n_slots * sizeof(Slot), ALIGN);
+    L->off_keys = o;           o += round_up(L->n_slots * 8, ALIGN);
+    L->off_vals = o;           o += round_up(L->n_slots * 16, ALIGN);
     L->off_work = o;           o += round_up(L->work_slots * sizeof(WorkSlot), ALIGN);
     L->off_appw = o;           o += round_up((size_t)c->n_apps * 4, ALIGN);
     L->off_hot = o;            o += round_up((size_t)(L->hot_slots ? L->hot_slots : 2) * 8, ALIGN);
@@ -69,6 +91,8 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, Layout* L) {
     L->off_staging[1] = o;     o += STAGING_BYTES;
     L->off_sel = o;            o += round_up((size_t)SEL_CAP * 32, ALIGN);
     L->off_topk_out = o;       o += round_up((size_t)ATREX_MAX_TOPK * sizeof(atrex_entry_t), ALIGN);
+    L->off_spill_cnt = o;      o += round_up(((size_t)L->n_groups << L->lp) * 4, ALIGN);
+    L->off_spill = o;          o += round_up(((size_t)L->n_groups << L->lp) * L->cap * 16, ALIGN);
     L->total = o;
 }
 
@@ -92,7 +116,10 @@ struct atrex_agg {
     bool owns_workspace = false;
     unsigned char* ws = nullptr;
     Control* ctl = nullptr;
-    Slot* table = nullptr;
+    ull* keys = nullptr;
+    ulonglong2* vals = nullptr;
+    uint32_t* spill_cnt = nullptr;
+    unsigned char* spill = nullptr;
     WorkSlot* work = nullptr;
     uint32_t* d_appw = nullptr;
     ull* hot_keys = nullptr;
@@ -111,10 +138,10 @@ struct atrex_agg {
 
     TableRef table_ref() const {
         TableRef t;
-        t.table = table;
-        t.mask = L.n_slots - 1;
-        t.shift = 64 - log2_of(L.n_slots);
-        t.max_probe = (uint32_t)(L.n_slots < MAX_PROBE ? L.n_slots : MAX_PROBE);
+        t.keys = keys;
+        t.vals = vals;
+        t.lp = L.lp;
+        t.C = L.C;
         t.ctl = ctl;
         return t;
     }
@@ -149,6 +176,15 @@ static int device_status_to_error(const Control* c) {
     return ATREX_OK;
 }
 
+static int query_sm_count(int device) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || v <= 0) {
+        cudaGetLastError();
+        return 148;  // B200
+    }
+    return v;
+}
+
 static int query_smem_optin(int device, size_t* out) {
     int v = 0;
     if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) return -1;
@@ -166,7 +202,7 @@ uint64_t atrex_agg_workspace_bytes(const atrex_agg_config_t* cfg) {
     size_t q;
     if (query_smem_optin(cfg->device, &q) == 0 && q > 0) smem = q;
     Layout L;
-    compute_layout(cfg, smem, &L);
+    compute_layout(cfg, smem, query_sm_count(cfg->device), &L);
     return L.total;
 }
 
@@ -189,8 +225,8 @@ int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out) {
     int rc = ATREX_OK;
     do {
         if (query_smem_optin(cfg->device, &smem) != 0) { rc = ATREX_ERR_CUDA; break; }
-        compute_layout(cfg, smem, &h->L);
         if (cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) { rc = ATREX_ERR_CUDA; break; }
+        compute_layout(cfg, smem, h->n_sms, &h->L);
         if (cfg->workspace) {
             if (cfg->workspace_bytes < h->L.total) { rc = ATREX_ERR_NOMEM; break; }
             h->ws = (unsigned char*)cfg->workspace;
@@ -200,7 +236,10 @@ int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out) {
         }
         const Layout& L = h->L;
         h->ctl = (Control*)(h->ws + L.off_ctl);
-        h->table = (Slot*)(h->ws + L.off_table);
+        h->keys = (ull*)(h->ws + L.off_keys);
+        h->vals = (ulonglong2*)(h->ws + L.off_vals);
+        h->spill_cnt = (uint32_t*)(h->ws + L.off_spill_cnt);
+        h->spill = h->ws + L.off_spill;
         h->work = (WorkSlot*)(h->ws + L.off_work);
         h->d_appw = (uint32_t*)(h->ws + L.off_appw);
         h->hot_keys = (ull*)(h->ws + L.off_hot);
@@ -250,7 +289,7 @@ int atrex_agg_reset(atrex_agg_t* h, void* stream) {
     DeviceGuard guard(h->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
     CU(h, cudaMemsetAsync(h->ctl, 0, sizeof(Control), s));
-    CU(h, cudaMemsetAsync(h->table, 0, h->L.n_slots * sizeof(Slot), s));
+    CU(h, cudaMemsetAsync(h->keys, 0, h->L.off_work - h->L.off_keys, s));  // keys and vals
     h->hot_ready = false;
     h->finalized = false;
     h->n_records = 0;
@@ -317,11 +356,23 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
     p.hot_slots = h->L.hot_slots;
     p.hot_buckets = h->L.hot_slots / 2;
     p.t = h->table_ref();
+    p.spill = h->spill;
+    p.spill_cnt = h->spill_cnt;
+    p.n_groups = h->L.n_groups;
+    p.cap = h->L.cap;
     const ull pairs_per_cta_iter = 2048;
     ull want = (p.n_pairs + pairs_per_cta_iter - 1) / pairs_per_cta_iter;
     int grid = (int)(want < 1 ? 1 : (want > (ull)h->n_sms ? (ull)h->n_sms : want));
-    CU(h, launch_ingest(p, h->hot_ready, grid, s));
-    h->launches++;
+    CU(h, launch_scatter(p, h->hot_ready, grid, s));
+    PartitionParams q;
+    q.t = p.t;
+    q.spill = h->spill;
+    q.spill_cnt = h->spill_cnt;
+    q.n_groups = h->L.n_groups;
+    q.n_used = (uint32_t)grid;
+    q.cap = h->L.cap;
+    CU(h, launch_partition(q, s));
+    h->launches += 2;
     return ATREX_OK;
 }
 
@@ -333,8 +384,8 @@ int atrex_agg_ingest(atrex_agg_t* h, const atrex_record_t* d_records, uint64_t n
     DeviceGuard guard(h->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
     h->finalized = false;
-    for (uint64_t off = 0; off < n; off += MAX_RECORDS_PER_LAUNCH) {
-        uint64_t m = n - off < MAX_RECORDS_PER_LAUNCH ? n - off : MAX_RECORDS_PER_LAUNCH;
+    for (uint64_t off = 0; off < n; off += h->L.sub_launch) {
+        uint64_t m = n - off < h->L.sub_launch ? n - off : h->L.sub_launch;
         int rc = ingest_launch(h, d_records + off, m, s);
         if (rc != ATREX_OK) return rc;
     }
@@ -380,14 +431,14 @@ int atrex_agg_merge(atrex_agg_t* h, const atrex_entry_t* d_entries, uint64_t n, 
 static int run_totals(atrex_agg* h, cudaStream_t s) {
     size_t off = offsetof(Control, total_lo);
     CU(h, cudaMemsetAsync((unsigned char*)h->ctl + off, 0, offsetof(Control, hist) - off, s));
-    CU(h, launch_totals(h->table, h->L.n_slots, h->ctl, h->scan_grid(h->L.n_slots, 128 * 8), s));
+    CU(h, launch_totals(h->table_ref(), h->L.n_slots, h->scan_grid(h->L.n_slots, 128 * 8), s));
     h->launches++;
     return ATREX_OK;
 }
 
 static FinalizeParams finalize_params(const atrex_agg* h, atrex_entry_t* out, uint64_t cap) {
     FinalizeParams p;
-    p.table = h->table;
+    p.t = h->table_ref();
     p.n_slots = h->L.n_slots;
     p.ctl = h->ctl;
     p.work = h->work_ref();
@@ -435,7 +486,7 @@ int atrex_agg_topk(atrex_agg_t* h, uint32_t phase, uint32_t k, atrex_entry_t* h_
 
     TopkParams p;
     memset(&p, 0, sizeof(p));
-    p.table = h->table;
+    p.t = h->table_ref();
     p.n_slots = h->L.n_slots;
     p.ctl = h->ctl;
     p.phase = phase;
@@ -505,6 +556,8 @@ int atrex_agg_stats(atrex_agg_t* h, atrex_stats_t* out, void* stream) {
     }
     out->table_slots = h->L.n_slots;
     out->hot_slots = c->hot_n;
+    out->n_spilled = c->n_spilled;
+    out->n_overflow = c->n_overflow;
     return device_status_to_error(c);
 }
 

@@ -1,14 +1,19 @@
 // Device-side data layout and helpers shared by the library's kernels.
 //
 // HBM layout
-//   key table   : open addressing, power-of-two capacity >= 2 * max_keys, one 32-byte slot
-//                 (= one L2 sector) per key:
-//                   skey  = ~key, so that 0 means EMPTY and reset is a memset
-//                   lo    = low 64 bits of the weighted time (wraps; wraps are counted)
-//                   cnthi = count in bits 0..39, number of wraps of `lo` plus merged high
-//                           words in bits 40..63  (count < 2^40, weighted time < 2^88)
-//                   spare
-//   work table  : same scheme keyed by op_id << 32 | shape_id, holding flops, bytes, dtype
+//   key table   : P partitions (power of two) of C slots each, structure of arrays:
+//                   keys[P*C]  ~key, so that 0 means EMPTY and reset is a memset
+//                   vals[P*C]  {lo, cnthi}: lo = low 64 bits of the weighted time (wraps; wraps
+//                              are counted), cnthi = count in bits 0..39, number of wraps of
+//                              `lo` plus merged high words in bits 40..63
+//                              (count < 2^40, weighted time < 2^88)
+//                 A key lives in partition hash >> (64 - log2 P), at a slot found by linear
+//                 probing inside that partition only.  C is chosen so that one partition's
+//                 keys and per-launch accumulators fit in one SM's shared memory: the
+//                 aggregation pass owns a partition per CTA and needs no global atomics.
+//   spill bufs  : [P][G][cap] 16-byte {key, weighted duration} entries and [P][G] counts,
+//                 written by CTA g of the scatter pass, read by CTA p of the partition pass
+//   work table  : open addressing keyed by op_id << 32 | shape_id, holding flops, bytes, dtype
 //   control     : counters, per-phase totals, top-k histogram
 #pragma once
 #include <cstdint>
@@ -19,14 +24,6 @@
 namespace atrex {
 
 typedef unsigned long long ull;
-
-struct Slot {
-    ull skey;
-    ull lo;
-    ull cnthi;
-    ull spare;
-};
-static_assert(sizeof(Slot) == 32, "one slot per 32-byte sector");
 
 struct WorkSlot {
     ull skey;      // ~(op_id << 32 | shape_id), 0 = EMPTY
@@ -58,7 +55,10 @@ struct Control {
     ull sel_count;             // top-k: selected candidates
     ull hot_n;                 // keys in the hot directory
     ull work_status;           // ST_WORK_* bits of the last work-table load
-    ull pad0;
+    ull hot_skew;              // 1 if one key dominates the sample: combine equal lanes per warp
+    ull n_spilled;             // records routed through the spill buffers
+    ull n_overflow;            // records that found their spill buffer full (slow exact path)
+    ull pad1[6];
     ull total_lo[ATREX_MAX_PHASES];
     ull total_hi[ATREX_MAX_PHASES];
     ull keys_per_phase[ATREX_MAX_PHASES];
@@ -66,7 +66,19 @@ struct Control {
     uint32_t hist[TOPK_BINS];
 };
 
-// 64-bit mixer for slot selection: multiply, fold, multiply; the top bits index the table.
+// 32-bit mixer of a packed key for the key table, the spill partitions and the hot directory:
+// two multiplicative hashes of the key's words, folded and multiplied once more.  The top
+// bits pick the partition, the bits below them the start slot inside it.
+__device__ __forceinline__ uint32_t hash32(uint32_t key_hi, uint32_t key_lo) {
+    uint32_t h = (key_lo * 0x9E3779B1u) ^ (key_hi * 0x85EBCA77u);
+    h ^= h >> 15;
+    h *= 0x2C1B3C6Du;
+    h ^= h >> 13;
+    return h;
+}
+__device__ __forceinline__ uint32_t hash32(ull key) { return hash32((uint32_t)(key >> 32), (uint32_t)key); }
+
+// 64-bit mixer for the work table: multiply, fold, multiply; the top bits index the table.
 __device__ __forceinline__ ull hash_key(ull key) {
     ull h = key * 0x9E3779B97F4A7C15ull;
     h ^= h >> 32;
@@ -84,52 +96,62 @@ __device__ __forceinline__ ull ld_relaxed(const ull* p) {
     return v;
 }
 
-// Find (or claim) the slot of `key`.  Returns nullptr after `max_probe` steps (table full).
-__device__ __forceinline__ Slot* find_or_claim(Slot* table, ull mask, int shift, uint32_t max_probe,
-                                               ull key, ull h) {
+struct TableRef {
+    ull* keys;            // [P * C]
+    ulonglong2* vals;     // [P * C] {lo, cnthi}
+    uint32_t lp;          // log2(P)
+    uint32_t C;           // slots per partition
+    Control* ctl;
+};
+
+constexpr ull NO_INDEX = ~0ull;
+
+__device__ __forceinline__ uint32_t part_of(uint32_t h, uint32_t lp) { return h >> (32 - lp); }  // lp >= 1
+
+// start slot inside the partition, from the hash bits below the partition bits
+__device__ __forceinline__ uint32_t local_of(uint32_t h, uint32_t lp, uint32_t C) { return __umulhi(h << lp, C); }
+
+// Find (or claim) the slot of `key` directly in HBM.  Returns NO_INDEX when the key's
+// partition has no free slot.  Used off the hot path: directory flush, buffer overflow,
+// merge.
+__device__ __forceinline__ ull find_or_claim(const TableRef& t, ull key, uint32_t h) {
     const ull skey = ~key;
-    ull s = h >> shift;
-    for (uint32_t probe = 0; probe < max_probe; ++probe) {
-        Slot* e = table + s;
-        ull k = ld_relaxed(&e->skey);
-        if (k == skey) return e;
+    const ull base = (ull)part_of(h, t.lp) * t.C;
+    uint32_t s = local_of(h, t.lp, t.C);
+    for (uint32_t probe = 0; probe < t.C; ++probe) {
+        ull* kp = t.keys + base + s;
+        ull k = ld_relaxed(kp);
+        if (k == skey) return base + s;
         if (k == 0) {
-            ull old = atomicCAS(&e->skey, 0ull, skey);
-            if (old == 0 || old == skey) return e;
+            ull old = atomicCAS(kp, 0ull, skey);
+            if (old == 0 || old == skey) return base + s;
         }
-        s = (s + 1) & mask;
+        s = (s + 1 == t.C) ? 0u : s + 1;
     }
-    return nullptr;
+    return NO_INDEX;
 }
 
 // Exact, order-independent accumulation of (count, v_hi * 2^64 + v_lo) into a slot: the
 // thread whose add wraps `lo` is unique, and it alone adds the carry.
-__device__ __forceinline__ void slot_add(Slot* e, ull v_lo, ull v_hi, ull count) {
+__device__ __forceinline__ void slot_add(const TableRef& t, ull idx, ull v_lo, ull v_hi, ull count) {
+    ull* v = reinterpret_cast<ull*>(t.vals + idx);
     ull carry = 0;
     if (v_lo != 0) {
-        ull old = atomicAdd(&e->lo, v_lo);
+        ull old = atomicAdd(v, v_lo);
         carry = (old + v_lo < old) ? 1ull : 0ull;
     }
     ull inc = count + ((v_hi + carry) << HI_SHIFT);
-    if (inc != 0) atomicAdd(&e->cnthi, inc);
+    if (inc != 0) atomicAdd(v + 1, inc);
 }
 
-struct TableRef {
-    Slot* table;
-    ull mask;
-    int shift;            // 64 - log2(capacity)
-    uint32_t max_probe;
-    Control* ctl;
-};
-
-__device__ __forceinline__ void table_accumulate(const TableRef& t, ull key, ull h, ull v_lo, ull v_hi, ull count) {
-    Slot* e = find_or_claim(t.table, t.mask, t.shift, t.max_probe, key, h);
-    if (e == nullptr) {
+__device__ __forceinline__ void table_accumulate(const TableRef& t, ull key, uint32_t h, ull v_lo, ull v_hi, ull count) {
+    ull idx = find_or_claim(t, key, h);
+    if (idx == NO_INDEX) {
         atomicOr(&t.ctl->status, ST_TABLE_FULL);
         atomicAdd(&t.ctl->n_dropped, count);
         return;
     }
-    slot_add(e, v_lo, v_hi, count);
+    slot_add(t, idx, v_lo, v_hi, count);
 }
 
 // One round-to-nearest-even conversion of hi * 2^64 + lo to binary64.  The top 64

@@ -17,22 +17,26 @@ struct SlotView {
     bool live;
 };
 
-__device__ __forceinline__ SlotView load_slot(const Slot* s) {
-    const ulonglong2* q = reinterpret_cast<const ulonglong2*>(s);
-    ulonglong2 a = q[0], b = q[1];
+__device__ __forceinline__ SlotView load_slot(const TableRef& t, ull i) {
     SlotView v;
-    v.live = a.x != 0;
-    v.key = ~a.x;
-    v.lo = a.y;
-    v.count = b.x & COUNT_MASK;
-    v.hi = b.x >> HI_SHIFT;
+    ull sk = t.keys[i];
+    v.live = sk != 0;
+    v.key = ~sk;
+    v.lo = v.count = v.hi = 0;
+    if (v.live) {
+        ulonglong2 x = t.vals[i];
+        v.lo = x.x;
+        v.count = x.y & COUNT_MASK;
+        v.hi = x.y >> HI_SHIFT;
+    }
     return v;
 }
 
 // ---- per-phase totals -------------------------------------------------------------------
 // Each thread keeps private per-phase 128-bit sums in its own shared-memory column; columns
 // are added per CTA and folded into the control block with a carry-aware pair of atomics.
-__global__ void __launch_bounds__(TOT_THREADS) totals_kernel(const Slot* table, ull n_slots, Control* ctl) {
+__global__ void __launch_bounds__(TOT_THREADS) totals_kernel(TableRef tab, ull n_slots) {
+    Control* ctl = tab.ctl;
     __shared__ ull s_lo[ATREX_MAX_PHASES][TOT_THREADS];
     __shared__ ull s_hi[ATREX_MAX_PHASES][TOT_THREADS];
     __shared__ ull s_cnt[ATREX_MAX_PHASES][TOT_THREADS];
@@ -43,7 +47,7 @@ __global__ void __launch_bounds__(TOT_THREADS) totals_kernel(const Slot* table, 
         s_lo[p][t] = 0; s_hi[p][t] = 0; s_cnt[p][t] = 0; s_nk[p][t] = 0;
     }
     for (ull i = (ull)blockIdx.x * blockDim.x + t; i < n_slots; i += (ull)gridDim.x * blockDim.x) {
-        SlotView v = load_slot(table + i);
+        SlotView v = load_slot(tab, i);
         if (!v.live) continue;
         int p = (int)(v.key >> 48) & (ATREX_MAX_PHASES - 1);
         ull o = s_lo[p][t], n = o + v.lo;
@@ -132,7 +136,7 @@ __global__ void __launch_bounds__(FIN_THREADS) emit_kernel(FinalizeParams p) {
         ull i = r * stride + (ull)blockIdx.x * blockDim.x + threadIdx.x;
         SlotView v;
         v.live = false;
-        if (i < p.n_slots) v = load_slot(p.table + i);
+        if (i < p.n_slots) v = load_slot(p.t, i);
         unsigned live = __ballot_sync(0xFFFFFFFFu, v.live);
         if (live == 0) continue;
         ull base = 0;
@@ -215,7 +219,7 @@ __global__ void __launch_bounds__(FIN_THREADS) topk_hist_kernel(TopkParams p) {
     for (int i = threadIdx.x; i < TOPK_BINS; i += blockDim.x) h[i] = 0;
     __syncthreads();
     for (ull i = (ull)blockIdx.x * blockDim.x + threadIdx.x; i < p.n_slots; i += (ull)gridDim.x * blockDim.x) {
-        SlotView v = load_slot(p.table + i);
+        SlotView v = load_slot(p.t, i);
         if (!v.live || (uint32_t)(v.key >> 48) != p.phase) continue;
         Composite x = composite_of(v);
         if (compare_prefix(x, p) != 0) continue;
@@ -228,7 +232,7 @@ __global__ void __launch_bounds__(FIN_THREADS) topk_hist_kernel(TopkParams p) {
 
 __global__ void __launch_bounds__(FIN_THREADS) topk_collect_kernel(TopkParams p) {
     for (ull i = (ull)blockIdx.x * blockDim.x + threadIdx.x; i < p.n_slots; i += (ull)gridDim.x * blockDim.x) {
-        SlotView v = load_slot(p.table + i);
+        SlotView v = load_slot(p.t, i);
         if (!v.live || (uint32_t)(v.key >> 48) != p.phase) continue;
         Composite x = composite_of(v);
         if (!p.collect_all && compare_prefix(x, p) < 0) continue;
@@ -276,7 +280,7 @@ __global__ void __launch_bounds__(FIN_THREADS) topk_emit_kernel(FinalizeParams p
     __shared__ bool zeroT[ATREX_MAX_PHASES];
     load_phase_totals(p.ctl, dT, zeroT);
     for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-        SlotView v = load_slot(p.table + sel[(ull)i * 4 + 3]);
+        SlotView v = load_slot(p.t, sel[(ull)i * 4 + 3]);
         store_entry(p.out + i, make_entry(v, dT, zeroT, p));
     }
 }
@@ -284,8 +288,8 @@ __global__ void __launch_bounds__(FIN_THREADS) topk_emit_kernel(FinalizeParams p
 // ---- launchers ----------------------------------------------------------------------------
 cudaError_t finalize_prepare() { return cudaSuccess; }
 
-cudaError_t launch_totals(const Slot* table, ull n_slots, Control* ctl, int grid, cudaStream_t stream) {
-    totals_kernel<<<grid, TOT_THREADS, 0, stream>>>(table, n_slots, ctl);
+cudaError_t launch_totals(const TableRef& t, ull n_slots, int grid, cudaStream_t stream) {
+    totals_kernel<<<grid, TOT_THREADS, 0, stream>>>(t, n_slots);
     return cudaGetLastError();
 }
 

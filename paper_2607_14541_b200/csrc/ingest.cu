@@ -1,31 +1,41 @@
-// Ingest: Eq. 2's group-by sum, streamed.
+// Ingest: Eq. 2's group-by sum, streamed, as a two-pass radix-partitioned aggregation.
 //
-// One persistent CTA per SM.  Each thread pulls records with 32-byte vector loads (two
-// 16-byte records per load, several loads in flight, streaming cache policy), packs the
-// key, multiplies the application's card-hour weight by the duration, and adds
-// (1, product) to the key's accumulators:
-//   * keys found in the shared-memory HOT DIRECTORY (the most frequent keys of a sample of
-//     the trace, identical in every CTA, read-only during the pass) are accumulated with
-//     32-bit shared-memory atomics in three limbs with explicit carries; lanes of a warp
-//     that hit the same slot are first combined with warp reductions;
-//   * every other record goes to the global open-addressing table with one 64-bit
-//     returning atomic (low limb, detects the wrap) and one 64-bit reduction
-//     (count + carries), after locating / claiming the slot.
-// At the end each CTA flushes its directory accumulators into the global table, so after
-// the kernel the global table alone holds exact sums.  All sums are integers, so the result
-// does not depend on which path a record took, on scheduling, or on chunking.
+// Random read-modify-write into a table far larger than L2 is bound by DRAM latency and by
+// the L2's atomic rate, not by bandwidth, so the hot path avoids global atomics altogether:
+//
+// Pass 1  SCATTER  (one persistent CTA per SM).  Each thread pulls records with 32-byte
+//   vector loads (two 16-byte records per load, several loads in flight, streaming cache
+//   policy), packs the key and multiplies the application's card-hour weight by the duration.
+//   * Keys found in the shared-memory HOT DIRECTORY (the most frequent keys of a sample of the
+//     trace, identical in every CTA, read-only during the pass) are accumulated on the spot
+//     with 32-bit shared-memory atomics in limbs with explicit carries; lanes of a warp that
+//     hit the same slot are first combined with warp reductions.
+//   * Every other record becomes a 16-byte {key, product} entry appended to the CTA's private
+//     buffer for the key's partition.  Appends of one (CTA, partition) pair are sequential in
+//     memory, so L2 merges them into full lines before they reach HBM.
+//   At the end the CTA flushes its directory accumulators into the table (these few thousand
+//   slots stay L2-resident) and publishes its per-partition entry counts.
+//
+// Pass 2  PARTITION  (one CTA per partition).  The CTA copies its partition's keys from HBM
+//   into shared memory, streams the partition's entries from all scatter CTAs, finds or
+//   claims each key's slot in shared memory and accumulates there, then adds the per-slot
+//   deltas back to the HBM table with coalesced read-modify-writes.  The CTA is the only
+//   writer of its partition, so no global atomics are involved.
+//
+// All sums are integers, so the result does not depend on which route a record took, on
+// scheduling, or on chunking.  Entries that do not fit a spill buffer, directory wraps and
+// merges fall back to exact atomic updates of the HBM table.
 #include "atrex_dev.cuh"
 #include "kernels.h"
 
 namespace atrex {
 
 constexpr int INGEST_THREADS = 1024;
-constexpr int LOADS_PER_ITER = 2;                 // 32-byte loads in flight per thread
-constexpr int RECS_PER_ITER = 2 * LOADS_PER_ITER;  // records per thread per iteration
 constexpr uint32_t NO_SLOT = 0xFFFFFFFFu;
+constexpr uint32_t NEW_KEY_FLAG = 0x80000000u;     // partition pass: slot claimed in this launch
 
-__device__ __forceinline__ uint32_t dir_bucket(ull h, uint32_t n_buckets) {
-    return __umulhi((uint32_t)(h >> 20), n_buckets);
+__device__ __forceinline__ uint32_t dir_bucket(uint32_t h, uint32_t n_buckets) {
+    return __umulhi(h * 0xC2B2AE35u, n_buckets);
 }
 
 __device__ __forceinline__ void ld_stream_256(const void* p, uint32_t (&w)[8]) {
@@ -36,43 +46,67 @@ __device__ __forceinline__ void ld_stream_256(const void* p, uint32_t (&w)[8]) {
 
 struct SmemDir {
     ull* keys;        // [slots], ~key, 0 = empty
-    uint32_t* cnt;    // [slots]
-    uint32_t* a0;     // [slots] bits 0..31 of the slot's sum
-    uint32_t* a1;     // [slots] bits 32..63
+    uint32_t* a0;     // [slots] this launch's weighted time of the slot: bits 0..31 ...
+    uint32_t* a1;     // [slots] ... and bits 32..63 (carries of a0 are added here by the adder)
+    uint32_t* cnt;    // [slots] this launch's record count of the slot
+    uint32_t* cursor; // [P] entries appended to this CTA's buffer of each partition
     const uint32_t* appw;
 };
 
-// Add (count, v) to a directory slot.  v < 2^53.  A wrap of the 64-bit (a1:a0) pair is rare
-// and is forwarded to the global table as one unit of the high word.
-__device__ __forceinline__ void dir_add(const SmemDir& d, uint32_t slot, ull v, uint32_t count,
-                                        const TableRef& t, ull key, ull h) {
-    atomicAdd(&d.cnt[slot], count);
+// Shared-memory accumulation uses native 32-bit atomics only (64-bit shared atomics are
+// compare-and-swap loops).  A slot's weighted time is kept in two limbs: the returning add on
+// the low limb tells the adder whether it wrapped, and the adder then adds the carry, with
+// the value's high word, to the high limb.  The high limb grows by less than 2^16 per record,
+// so it is drained every 2^14 counted records (the returning count add elects the drainer):
+// 2^14 records plus the adds that can slip in before the drain (at most one warp's worth per
+// thread of the CTA, 2^15 records) stay below 2^32.
+constexpr uint32_t DRAIN_SHIFT = 14;
+
+__device__ __forceinline__ bool limbs_add(uint32_t* a0, uint32_t* a1, uint32_t* cnt, ull v, uint32_t count) {
     uint32_t v0 = (uint32_t)v;
-    uint32_t o0 = atomicAdd(&d.a0[slot], v0);
+    uint32_t o0 = atomicAdd(a0, v0);
     uint32_t x = (uint32_t)(v >> 32) + ((o0 + v0 < o0) ? 1u : 0u);
-    if (x != 0) {
-        uint32_t o1 = atomicAdd(&d.a1[slot], x);
-        if (o1 + x < o1) table_accumulate(t, key, h, 0, 1, 0);
+    if (x != 0) atomicAdd(a1, x);
+    uint32_t c = atomicAdd(cnt, count) & 0x7FFFFFFFu;
+    return ((c + count) >> DRAIN_SHIFT) != (c >> DRAIN_SHIFT);  // true: the caller must drain
+}
+
+__device__ __forceinline__ ull limbs_drain(uint32_t* a0, uint32_t* a1, ull* hi_out) {
+    // the two exchanges need not be simultaneous: whatever lands between them stays in the
+    // limbs for the next drain or the final flush
+    ull lo = atomicExch(a0, 0u);
+    ull hi = atomicExch(a1, 0u);
+    ull v = lo + (hi << 32);
+    *hi_out = (hi >> 32) + (v < lo ? 1ull : 0ull);
+    return v;
+}
+
+// Add (count, v) to a directory slot, v < 2^53, count <= 32.
+__device__ __forceinline__ void dir_add(const SmemDir& d, uint32_t slot, ull v, uint32_t count, const TableRef& t,
+                                        uint32_t h) {
+    if (limbs_add(&d.a0[slot], &d.a1[slot], &d.cnt[slot], v, count)) {
+        ull hi, lo = limbs_drain(&d.a0[slot], &d.a1[slot], &hi);
+        table_accumulate(t, ~d.keys[slot], h, lo, hi, 0);
     }
 }
 
-// Process R records held in registers by every lane of the warp (lane-invalid ones masked).
-template <bool HOT, int R>
+// Process R records held in registers by every lane of the warp (absent ones masked).
+// Written in stages over the R records so that their shared-memory round trips overlap.
+template <bool HOT, bool DEDUPE, int R>
 __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&present)[R], const IngestParams& p,
                                         const SmemDir& d, uint32_t& rejected) {
-    ull key[R], prod[R], h[R];
-    bool todo[R];  // still has to go to the global table
+    uint32_t khi[R], h[R];
+    ull prod[R];
+    bool todo[R];  // valid and not yet accumulated
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         uint32_t app = w[r][0];
-        uint32_t op = w[r][1] & 0xFFFFu;
-        uint32_t phase = (w[r][1] >> 16) & 0xFFu;
-        bool ok = present[r] && app < p.n_apps && phase < p.n_phases;
+        khi[r] = w[r][1] & 0x00FFFFFFu;                 // phase << 16 | op_id: the key's high word
+        bool ok = present[r] && app < p.n_apps && (khi[r] >> 16) < p.n_phases;
         rejected += (present[r] && !ok) ? 1u : 0u;
-        uint32_t wgt = ok ? d.appw[app] : 0u;
-        key[r] = pack_key(phase, op, w[r][2]);
+        uint32_t wgt = d.appw[ok ? app : 0u];
         prod[r] = (ull)wgt * (ull)w[r][3];
-        h[r] = hash_key(key[r]);
+        h[r] = hash32(khi[r], w[r][2]);
         todo[r] = ok;
     }
     if (HOT) {
@@ -81,79 +115,127 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
         for (int r = 0; r < R; ++r) {
             uint32_t b = dir_bucket(h[r], p.hot_buckets) * 2;
             ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(d.keys + b);
-            ull skey = ~key[r];
+            ull skey = ~(((ull)khi[r] << 32) | w[r][2]);
             slot[r] = !todo[r] ? NO_SLOT : (kk.x == skey ? b : (kk.y == skey ? b + 1 : NO_SLOT));
         }
-        const unsigned lane = threadIdx.x & 31u;
+        if (DEDUPE) {
+            // one key dominates the trace: combine the lanes that share the first hitting lane's slot
+            const unsigned lane = threadIdx.x & 31u;
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-            // combine the lanes that share the first hitting lane's slot (dominant-key case)
-            unsigned hits = __ballot_sync(0xFFFFFFFFu, slot[r] != NO_SLOT);
-            if (hits != 0) {
+            for (int r = 0; r < R; ++r) {
+                unsigned hits = __ballot_sync(0xFFFFFFFFu, slot[r] != NO_SLOT);
+                if (hits == 0) continue;
                 int lead = __ffs(hits) - 1;
                 uint32_t ls = __shfl_sync(0xFFFFFFFFu, slot[r], lead);
                 unsigned same = __ballot_sync(0xFFFFFFFFu, slot[r] == ls);
-                if (__popc(same) >= 2) {
-                    if (slot[r] == ls) {
-                        uint32_t s_lo = __reduce_add_sync(same, (uint32_t)prod[r] & 0xFFFFFFu);
-                        uint32_t s_hi = __reduce_add_sync(same, (uint32_t)(prod[r] >> 24));
-                        if (lane == (unsigned)lead)
-                            dir_add(d, ls, (ull)s_lo + ((ull)s_hi << 24), (uint32_t)__popc(same), p.t, key[r], h[r]);
-                        slot[r] = NO_SLOT;
-                        todo[r] = false;
-                    }
+                if (__popc(same) >= 2 && slot[r] == ls) {
+                    uint32_t s_lo = __reduce_add_sync(same, (uint32_t)prod[r] & 0xFFFFFFu);
+                    uint32_t s_hi = __reduce_add_sync(same, (uint32_t)(prod[r] >> 24));
+                    if (lane == (unsigned)lead)
+                        dir_add(d, ls, (ull)s_lo + ((ull)s_hi << 24), (uint32_t)__popc(same), p.t, h[r]);
+                    slot[r] = NO_SLOT;
+                    todo[r] = false;
                 }
             }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
             if (slot[r] != NO_SLOT) {
-                dir_add(d, slot[r], prod[r], 1u, p.t, key[r], h[r]);
+                dir_add(d, slot[r], prod[r], 1u, p.t, h[r]);
                 todo[r] = false;
             }
         }
     }
-    // global table: issue the first-probe key loads together, then resolve, then the adds
-    Slot* e[R];
-    ull k0[R];
+    // spill: append {key, product} to this CTA's buffer of the key's partition
+    uint32_t pos[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) {
-        e[r] = p.t.table + (h[r] >> p.t.shift);
-        k0[r] = todo[r] ? ld_relaxed(&e[r]->skey) : 0ull;
-    }
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        if (todo[r] && k0[r] != ~key[r]) {
-            e[r] = find_or_claim(p.t.table, p.t.mask, p.t.shift, p.t.max_probe, key[r], h[r]);
-            if (e[r] == nullptr) {
-                atomicOr(&p.t.ctl->status, ST_TABLE_FULL);
-                atomicAdd(&p.t.ctl->n_dropped, 1ull);
-                todo[r] = false;
-            }
-        }
-    }
-    ull old[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) old[r] = (todo[r] && prod[r] != 0) ? atomicAdd(&e[r]->lo, prod[r]) : 0ull;
+    for (int r = 0; r < R; ++r) pos[r] = todo[r] ? atomicAdd(&d.cursor[part_of(h[r], p.t.lp)], 1u) : 0u;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         if (todo[r]) {
-            ull carry = (old[r] + prod[r] < old[r]) ? 1ull : 0ull;
-            atomicAdd(&e[r]->cnthi, 1ull + (carry << HI_SHIFT));
+            ull key = ((ull)khi[r] << 32) | w[r][2];
+            if (pos[r] < p.cap) {
+                uint32_t idx = part_of(h[r], p.t.lp) * (p.n_groups * p.cap) + blockIdx.x * p.cap + pos[r];
+                *reinterpret_cast<ulonglong2*>(p.spill + (ull)idx * 16ull) = make_ulonglong2(key, prod[r]);
+            } else {
+                table_accumulate(p.t, key, h[r], prod[r], 0, 1);  // buffer full: exact slow path
+            }
         }
     }
 }
 
+template <bool HOT, bool DEDUPE>
+__device__ __forceinline__ void scatter_body(const IngestParams& p, const SmemDir& d, uint32_t& rejected) {
+    // two 32-byte loads (four records) in flight per thread: the next pair is requested before
+    // the current one is processed
+    const unsigned char* body = reinterpret_cast<const unsigned char*>(p.body);
+    const ull stride = (ull)gridDim.x * INGEST_THREADS;
+    uint32_t rawA[8], rawB[8];
+    auto fetch = [&](ull i, uint32_t (&raw)[8]) {
+        if (i < p.n_pairs) {
+            ld_stream_256(body + i * 32, raw);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) raw[j] = 0;
+        }
+    };
+    auto consume = [&](ull i, const uint32_t (&raw)[8]) {
+        uint32_t w[2][4];
+        bool present[2];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            w[0][j] = raw[j];
+            w[1][j] = raw[4 + j];
+        }
+        present[0] = present[1] = i < p.n_pairs;
+        process<HOT, DEDUPE, 2>(w, present, p, d, rejected);
+    };
+    const ull first = (ull)blockIdx.x * INGEST_THREADS;
+    fetch(first + threadIdx.x, rawA);
+    fetch(first + stride + threadIdx.x, rawB);
+    for (ull base = first; base < p.n_pairs; base += 2 * stride) {  // CTA-uniform trip count
+        ull i = base + threadIdx.x;
+        uint32_t cur[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cur[j] = rawA[j];
+        fetch(i + 2 * stride, rawA);
+        consume(i, cur);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cur[j] = rawB[j];
+        fetch(i + 3 * stride, rawB);
+        consume(i + stride, cur);
+    }
+    // records that do not form an aligned pair (at most one before and one after the body)
+    if (blockIdx.x == 0 && threadIdx.x < 32) {
+        uint32_t w1[1][4] = {{0, 0, 0, 0}};
+        bool pr[1] = {false};
+        const void* src = threadIdx.x == 0 ? p.single[0] : p.single[1];
+        if (threadIdx.x < p.n_single) {
+            uint4 v = *reinterpret_cast<const uint4*>(src);
+            w1[0][0] = v.x; w1[0][1] = v.y; w1[0][2] = v.z; w1[0][3] = v.w;
+            pr[0] = true;
+        }
+        process<HOT, DEDUPE, 1>(w1, pr, p, d, rejected);
+    }
+}
+
 template <bool HOT>
-__global__ void __launch_bounds__(INGEST_THREADS, 1) ingest_kernel(IngestParams p) {
+__global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     SmemDir d;
     unsigned char* sp = smem_raw;
     d.keys = reinterpret_cast<ull*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 8 : 0;
-    d.cnt = reinterpret_cast<uint32_t*>(sp);
-    sp += HOT ? (size_t)p.hot_slots * 4 : 0;
     d.a0 = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
     d.a1 = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
+    d.cnt = reinterpret_cast<uint32_t*>(sp);
+    sp += HOT ? (size_t)p.hot_slots * 4 : 0;
+    const uint32_t n_parts = 1u << p.t.lp;
+    d.cursor = reinterpret_cast<uint32_t*>(sp);
+    sp += (size_t)n_parts * 4;
+    for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) d.cursor[i] = 0;
     if (p.appw_in_smem) {
         uint32_t* s_appw = reinterpret_cast<uint32_t*>(sp);
         for (uint32_t i = threadIdx.x; i < p.n_apps; i += blockDim.x) s_appw[i] = p.app_w[i];
@@ -164,66 +246,143 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) ingest_kernel(IngestParams 
     if (HOT) {
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
             d.keys[i] = p.hot_keys[i];
-            d.cnt[i] = 0;
             d.a0[i] = 0;
             d.a1[i] = 0;
+            d.cnt[i] = 0;
         }
     }
     __syncthreads();
 
     uint32_t rejected = 0;
-    const ull tile = (ull)INGEST_THREADS * LOADS_PER_ITER;  // pairs per CTA iteration
-    const unsigned char* body = reinterpret_cast<const unsigned char*>(p.body);
-    for (ull base = (ull)blockIdx.x * tile; base < p.n_pairs; base += (ull)gridDim.x * tile) {
-        uint32_t w[RECS_PER_ITER][4];
-        bool present[RECS_PER_ITER];
-        uint32_t raw[LOADS_PER_ITER][8];
-#pragma unroll
-        for (int u = 0; u < LOADS_PER_ITER; ++u) {
-            ull i = base + (ull)u * INGEST_THREADS + threadIdx.x;
-            bool in = i < p.n_pairs;
-            if (in) {
-                ld_stream_256(body + i * 32, raw[u]);
-            } else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) raw[u][j] = 0;
-            }
-            present[2 * u] = in;
-            present[2 * u + 1] = in;
-        }
-#pragma unroll
-        for (int u = 0; u < LOADS_PER_ITER; ++u)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                w[2 * u][j] = raw[u][j];
-                w[2 * u + 1][j] = raw[u][4 + j];
-            }
-        process<HOT, RECS_PER_ITER>(w, present, p, d, rejected);
-    }
-    // records that do not form an aligned pair (at most one before and one after the body)
-    if (blockIdx.x == 0 && threadIdx.x < 32) {
-        uint32_t w1[1][4] = {{0, 0, 0, 0}};
-        bool pr[1] = {false};
-        if (threadIdx.x < p.n_single) {
-            uint4 v = *reinterpret_cast<const uint4*>(p.single[threadIdx.x]);
-            w1[0][0] = v.x; w1[0][1] = v.y; w1[0][2] = v.z; w1[0][3] = v.w;
-            pr[0] = true;
-        }
-        process<HOT, 1>(w1, pr, p, d, rejected);
-    }
+    if (HOT && p.t.ctl->hot_skew != 0)
+        scatter_body<HOT, true>(p, d, rejected);
+    else
+        scatter_body<HOT, false>(p, d, rejected);
+
     // rejected counter: one atomic per warp
     uint32_t rsum = __reduce_add_sync(0xFFFFFFFFu, rejected);
     if ((threadIdx.x & 31u) == 0 && rsum != 0) atomicAdd(&p.t.ctl->n_rejected, (ull)rsum);
 
+    __syncthreads();
+    uint32_t spilled = 0, overflow = 0;
+    for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) {
+        uint32_t c = d.cursor[i];
+        p.spill_cnt[(ull)i * p.n_groups + blockIdx.x] = min(c, p.cap);
+        spilled += min(c, p.cap);
+        overflow += c > p.cap ? c - p.cap : 0u;
+    }
+    spilled = __reduce_add_sync(0xFFFFFFFFu, spilled);
+    overflow = __reduce_add_sync(0xFFFFFFFFu, overflow);
+    if ((threadIdx.x & 31u) == 0) {
+        if (spilled) atomicAdd(&p.t.ctl->n_spilled, (ull)spilled);
+        if (overflow) atomicAdd(&p.t.ctl->n_overflow, (ull)overflow);
+    }
     if (HOT) {
-        __syncthreads();
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
             uint32_t c = d.cnt[i], lo = d.a0[i], hi = d.a1[i];
             if ((c | lo | hi) != 0) {
                 ull key = ~d.keys[i];
-                table_accumulate(p.t, key, hash_key(key), (ull)lo | ((ull)hi << 32), 0, (ull)c);
+                table_accumulate(p.t, key, hash32(key), (ull)lo | ((ull)hi << 32), 0, (ull)c);
             }
         }
+    }
+}
+
+// --------------------------------------------------------------------------------------
+// Pass 2: one CTA aggregates one partition entirely in shared memory.
+__global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionParams q) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t C = q.t.C;
+    ull* s_keys = reinterpret_cast<ull*>(smem_raw);
+    uint32_t* s_a0 = reinterpret_cast<uint32_t*>(s_keys + C);
+    uint32_t* s_a1 = s_a0 + C;
+    uint32_t* s_cnt = s_a1 + C;
+    __shared__ uint32_t s_total;
+    const uint32_t part = blockIdx.x;
+    const uint32_t* my_cnt = q.spill_cnt + (ull)part * q.n_groups;
+    if (threadIdx.x == 0) s_total = 0;
+    __syncthreads();
+    uint32_t local_total = 0;
+    for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) local_total += my_cnt[g];
+    local_total = __reduce_add_sync(0xFFFFFFFFu, local_total);
+    if ((threadIdx.x & 31u) == 0 && local_total) atomicAdd(&s_total, local_total);
+    __syncthreads();
+    if (s_total == 0) return;  // nothing was spilled to this partition
+
+    const ull base = (ull)part * C;
+    for (uint32_t i = threadIdx.x; i < C; i += blockDim.x) {
+        s_keys[i] = q.t.keys[base + i];
+        s_a0[i] = 0;
+        s_a1[i] = 0;
+        s_cnt[i] = 0;
+    }
+    __syncthreads();
+
+    const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
+    for (uint32_t g = warp; g < q.n_used; g += n_warps) {
+        const uint32_t n_e = my_cnt[g];
+        const ulonglong2* src = reinterpret_cast<const ulonglong2*>(q.spill) + ((ull)part * q.n_groups + g) * q.cap;
+        for (uint32_t e0 = 0; e0 < n_e; e0 += 128) {
+            ulonglong2 ent[4];
+            bool have[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                uint32_t e = e0 + u * 32 + lane;
+                have[u] = e < n_e;
+                if (have[u]) ent[u] = __ldcs(src + e);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const ull key = ent[u].x, v = ent[u].y, skey = ~key;
+                uint32_t s = local_of(hash32(key), q.t.lp, C);
+                // warp-convergent probe: every lane steps until all lanes have their slot
+                bool searching = have[u], ok = have[u];
+                uint32_t steps = 0;
+                while (__any_sync(0xFFFFFFFFu, searching)) {
+                    if (searching) {
+                        ull k = s_keys[s];
+                        if (k == 0) {
+                            k = atomicCAS(&s_keys[s], 0ull, skey);
+                            if (k == 0) {
+                                atomicOr(&s_cnt[s], NEW_KEY_FLAG);
+                                k = skey;
+                            }
+                        }
+                        if (k == skey) {
+                            searching = false;
+                        } else {
+                            s = (s + 1 == C) ? 0u : s + 1;
+                            if (++steps >= C) {  // partition full
+                                searching = false;
+                                ok = false;
+                                atomicOr(&q.t.ctl->status, ST_TABLE_FULL);
+                                atomicAdd(&q.t.ctl->n_dropped, 1ull);
+                            }
+                        }
+                    }
+                }
+                if (ok && limbs_add(&s_a0[s], &s_a1[s], &s_cnt[s], v, 1u)) {
+                    // drain: this CTA owns the slot, so adds into HBM are exact; the write-back
+                    // below adds on top of them
+                    ull hi, lo = limbs_drain(&s_a0[s], &s_a1[s], &hi);
+                    ull* vp = reinterpret_cast<ull*>(q.t.vals + base + s);
+                    ull old = atomicAdd(vp, lo);
+                    hi += (old + lo < old) ? 1ull : 0ull;
+                    if (hi) atomicAdd(vp + 1, hi << HI_SHIFT);
+                }
+            }
+        }
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < C; i += blockDim.x) {
+        uint32_t c = s_cnt[i];
+        if (c == 0) continue;
+        ull* vp = reinterpret_cast<ull*>(q.t.vals + base + i);
+        ull lo = ld_relaxed(vp), cnthi = ld_relaxed(vp + 1);
+        ull nlo = lo + ((ull)s_a0[i] | ((ull)s_a1[i] << 32));
+        cnthi += (ull)(c & ~NEW_KEY_FLAG) + ((nlo < lo ? 1ull : 0ull) << HI_SHIFT);
+        *reinterpret_cast<ulonglong2*>(vp) = make_ulonglong2(nlo, cnthi);
+        if (c & NEW_KEY_FLAG) q.t.keys[base + i] = s_keys[i];
     }
 }
 
@@ -256,10 +415,13 @@ __global__ void __launch_bounds__(1024, 1) hot_build_kernel(HotBuildParams p) {
         if (v.x >= p.n_apps || phase >= p.n_phases) continue;
         ull key = pack_key(phase, v.y & 0xFFFFu, v.z);
         ull skey = ~key;
-        uint32_t s = (uint32_t)(hash_key(key) >> 50);  // 14 bits
+        uint32_t s = hash32(key) >> 18;  // 14 bits
         for (uint32_t probe = 0; probe < SAMPLE_PROBES; ++probe) {
             ull k = skeys[s];
-            if (k == 0) k = atomicCAS(&skeys[s], 0ull, skey), k = (k == 0) ? skey : k;
+            if (k == 0) {
+                k = atomicCAS(&skeys[s], 0ull, skey);
+                if (k == 0) k = skey;
+            }
             if (k == skey) {
                 atomicAdd(&scnt[s], 1u);
                 break;
@@ -280,6 +442,11 @@ __global__ void __launch_bounds__(1024, 1) hot_build_kernel(HotBuildParams p) {
             thr = (uint32_t)c;
         }
         s_thr = thr;
+        // a key holding more than 1/32 of the sample makes same-slot collisions inside a warp
+        // common: tell the scatter pass to combine equal lanes first
+        uint32_t top = 255;
+        while (top > 0 && hist[top] == 0) --top;
+        p.ctl->hot_skew = (top >= 255 || top * 32u >= p.n_sample) ? 1ull : 0ull;
     }
     __syncthreads();
     const uint32_t thr = s_thr;
@@ -291,7 +458,7 @@ __global__ void __launch_bounds__(1024, 1) hot_build_kernel(HotBuildParams p) {
                 uint32_t c = scnt[i];
                 if (c >= lo && c < hi) {
                     ull skey = skeys[i];
-                    uint32_t b = dir_bucket(hash_key(~skey), p.hot_slots / 2) * 2;
+                    uint32_t b = dir_bucket(hash32(~skey), p.hot_slots / 2) * 2;
                     if (atomicCAS(&p.hot_keys[b], 0ull, skey) == 0 || atomicCAS(&p.hot_keys[b + 1], 0ull, skey) == 0)
                         atomicAdd(&s_inserted, 1u);
                 }
@@ -307,31 +474,34 @@ __global__ void __launch_bounds__(1024, 1) hot_build_kernel(HotBuildParams p) {
 __global__ void __launch_bounds__(256) merge_kernel(const atrex_entry_t* in, ull n, TableRef t) {
     for (ull i = (ull)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (ull)gridDim.x * blockDim.x) {
         atrex_entry_t e = in[i];
-        table_accumulate(t, e.key, hash_key(e.key), e.wt_lo, e.wt_hi, e.count);
+        table_accumulate(t, e.key, hash32(e.key), e.wt_lo, e.wt_hi, e.count);
     }
 }
 
 // --------------------------------------------------------------------------------------
 // host launchers
 
-size_t ingest_smem_bytes(bool hot, uint32_t hot_slots, uint32_t n_apps, bool appw_in_smem) {
-    return (hot ? (size_t)hot_slots * 20 : 0) + (appw_in_smem ? (size_t)n_apps * 4 : 0);
-}
-
 cudaError_t ingest_prepare() {
-    cudaError_t e = cudaFuncSetAttribute(ingest_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+    cudaError_t e = cudaFuncSetAttribute(scatter_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(ingest_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+    e = cudaFuncSetAttribute(scatter_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(partition_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(hot_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SAMPLE_SLOTS * 12);
 }
 
-cudaError_t launch_ingest(const IngestParams& p, bool hot, int grid, cudaStream_t stream) {
-    size_t smem = ingest_smem_bytes(hot, p.hot_slots, p.n_apps, p.appw_in_smem != 0);
+cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream) {
+    size_t smem = (hot ? (size_t)p.hot_slots * 20 : 0) + ((size_t)4 << p.t.lp) + (p.appw_in_smem ? (size_t)p.n_apps * 4 : 0);
     if (hot)
-        ingest_kernel<true><<<grid, INGEST_THREADS, smem, stream>>>(p);
+        scatter_kernel<true><<<grid, INGEST_THREADS, smem, stream>>>(p);
     else
-        ingest_kernel<false><<<grid, INGEST_THREADS, smem, stream>>>(p);
+        scatter_kernel<false><<<grid, INGEST_THREADS, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_partition(const PartitionParams& q, cudaStream_t stream) {
+    partition_kernel<<<1u << q.t.lp, INGEST_THREADS, (size_t)q.t.C * 20, stream>>>(q);
     return cudaGetLastError();
 }
 

@@ -16,6 +16,20 @@ struct IngestParams {
     uint32_t hot_slots;        // even
     uint32_t hot_buckets;      // hot_slots / 2
     TableRef t;
+    // spill buffers: entry (p, g, i) at spill + ((p * n_groups + g) * cap + i) * 16 bytes
+    unsigned char* spill;
+    uint32_t* spill_cnt;       // [P][n_groups]
+    uint32_t n_groups;         // G, row pitch of the buffers (= CTAs of the widest scatter launch)
+    uint32_t cap;              // entries per (partition, CTA) buffer
+};
+
+struct PartitionParams {
+    TableRef t;
+    const unsigned char* spill;
+    const uint32_t* spill_cnt;
+    uint32_t n_groups;         // row pitch G
+    uint32_t n_used;           // CTAs of the scatter launch that fed this pass (<= G)
+    uint32_t cap;
 };
 
 struct HotBuildParams {
@@ -36,7 +50,7 @@ struct WorkRef {
 };
 
 struct FinalizeParams {
-    const Slot* table;
+    TableRef t;
     ull n_slots;
     Control* ctl;
     WorkRef work;
@@ -46,7 +60,7 @@ struct FinalizeParams {
 };
 
 struct TopkParams {
-    const Slot* table;
+    TableRef t;
     ull n_slots;
     Control* ctl;
     uint32_t phase;
@@ -57,14 +71,14 @@ struct TopkParams {
     uint32_t sel_cap;
 };
 
-size_t ingest_smem_bytes(bool hot, uint32_t hot_slots, uint32_t n_apps, bool appw_in_smem);
 cudaError_t ingest_prepare();
-cudaError_t launch_ingest(const IngestParams& p, bool hot, int grid, cudaStream_t stream);
+cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream);
+cudaError_t launch_partition(const PartitionParams& p, cudaStream_t stream);
 cudaError_t launch_hot_build(const HotBuildParams& p, cudaStream_t stream);
 cudaError_t launch_merge(const atrex_entry_t* in, ull n, const TableRef& t, int grid, cudaStream_t stream);
 
 cudaError_t finalize_prepare();
-cudaError_t launch_totals(const Slot* table, ull n_slots, Control* ctl, int grid, cudaStream_t stream);
+cudaError_t launch_totals(const TableRef& t, ull n_slots, int grid, cudaStream_t stream);
 cudaError_t launch_emit(const FinalizeParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_work_insert(const atrex_work_t* rows, ull n, const WorkRef& w, Control* ctl, int grid,
                                cudaStream_t stream);
