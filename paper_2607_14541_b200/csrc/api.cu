@@ -18,7 +18,9 @@ constexpr uint32_t LP_MIN = 8, LP_MAX = 12;             // 256 .. 4096 partition
 constexpr ull MAX_KEYS = 1ull << 25;
 constexpr ull MAX_RECORDS_TOTAL = 1ull << 40;
 constexpr uint32_t HOT_MIN_RECORDS = 32768;             // smaller calls run without a directory
-constexpr uint32_t HOT_SAMPLE = 131072;
+constexpr uint32_t HOT_SAMPLE = 1u << 20;
+constexpr uint32_t CAND_BITS = 16;                     // candidate table of the directory build
+constexpr size_t HOT_SCRATCH_BYTES = (65536 * 4) + ((size_t)12 << CAND_BITS);
 constexpr uint32_t APPW_SMEM_MAX = 4096;
 constexpr uint32_t MAX_PROBE = 4096;                   // work-table probe bound
 constexpr uint32_t SEL_CAP = ATREX_MAX_TOPK + TOPK_CAND_CAP;
@@ -39,7 +41,7 @@ int log2_of(ull p) {
 
 struct Layout {
     size_t off_ctl, off_keys, off_vals, off_work, off_appw, off_hot, off_staging[2], off_sel, off_topk_out,
-        off_spill_cnt, off_spill, total;
+        off_spill_cnt, off_spill, off_hot_scratch, total;
     ull n_slots, work_slots;
     uint32_t lp, C;              // partitions = 1 << lp, slots per partition
     uint32_t n_groups, cap;      // spill buffers: [P][n_groups][cap] entries
@@ -91,8 +93,9 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     L->off_staging[1] = o;     o += STAGING_BYTES;
     L->off_sel = o;            o += round_up((size_t)SEL_CAP * 32, ALIGN);
     L->off_topk_out = o;       o += round_up((size_t)ATREX_MAX_TOPK * sizeof(atrex_entry_t), ALIGN);
+    L->off_hot_scratch = o;    o += round_up(HOT_SCRATCH_BYTES, ALIGN);
     L->off_spill_cnt = o;      o += round_up(((size_t)L->n_groups << L->lp) * 4, ALIGN);
-    L->off_spill = o;          o += round_up(((size_t)L->n_groups << L->lp) * L->cap * 16, ALIGN);
+    L->off_spill = o;          o += round_up(((size_t)L->n_groups << L->lp) * L->cap * 16, ALIGN) + ALIGN;  // + prefetch overrun
     L->total = o;
 }
 
@@ -120,6 +123,7 @@ struct atrex_agg {
     ulonglong2* vals = nullptr;
     uint32_t* spill_cnt = nullptr;
     unsigned char* spill = nullptr;
+    unsigned char* hot_scratch = nullptr;
     WorkSlot* work = nullptr;
     uint32_t* d_appw = nullptr;
     ull* hot_keys = nullptr;
@@ -240,6 +244,7 @@ int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out) {
         h->vals = (ulonglong2*)(h->ws + L.off_vals);
         h->spill_cnt = (uint32_t*)(h->ws + L.off_spill_cnt);
         h->spill = h->ws + L.off_spill;
+        h->hot_scratch = h->ws + L.off_hot_scratch;
         h->work = (WorkSlot*)(h->ws + L.off_work);
         h->d_appw = (uint32_t*)(h->ws + L.off_appw);
         h->hot_keys = (ull*)(h->ws + L.off_hot);
@@ -334,8 +339,13 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
         b.hot_keys = h->hot_keys;
         b.hot_slots = h->L.hot_slots;
         b.ctl = h->ctl;
-        CU(h, launch_hot_build(b, s));
-        h->launches++;
+        b.sketch = (uint32_t*)h->hot_scratch;
+        b.cand_keys = (ull*)(h->hot_scratch + 65536 * 4);
+        b.cand_cnt = (uint32_t*)(h->hot_scratch + 65536 * 4 + ((size_t)8 << CAND_BITS));
+        b.cand_bits = CAND_BITS;
+        CU(h, cudaMemsetAsync(h->hot_scratch, 0, HOT_SCRATCH_BYTES, s));
+        CU(h, launch_hot_build(b, h->n_sms, s));
+        h->launches += 3;
         h->hot_ready = true;
     }
     IngestParams p;

@@ -11,8 +11,10 @@
 //                 probing inside that partition only.  C is chosen so that one partition's
 //                 keys and per-launch accumulators fit in one SM's shared memory: the
 //                 aggregation pass owns a partition per CTA and needs no global atomics.
-//   spill bufs  : [P][G][cap] 16-byte {key, weighted duration} entries and [P][G] counts,
-//                 written by CTA g of the scatter pass, read by CTA p of the partition pass
+//   spill bufs  : [G][P][cap] 16-byte {key, weighted duration} entries and [G][P] counts,
+//                 written by CTA g of the scatter pass (its buffers are contiguous, which keeps
+//                 the scattered 16-byte appends within a few pages), read by CTA p of the
+//                 partition pass
 //   work table  : open addressing keyed by op_id << 32 | shape_id, holding flops, bytes, dtype
 //   control     : counters, per-phase totals, top-k histogram
 #pragma once

@@ -155,8 +155,12 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
         if (todo[r]) {
             ull key = ((ull)khi[r] << 32) | w[r][2];
             if (pos[r] < p.cap) {
-                uint32_t idx = part_of(h[r], p.t.lp) * (p.n_groups * p.cap) + blockIdx.x * p.cap + pos[r];
-                *reinterpret_cast<ulonglong2*>(p.spill + (ull)idx * 16ull) = make_ulonglong2(key, prod[r]);
+                uint32_t idx = ((blockIdx.x << p.t.lp) + part_of(h[r], p.t.lp)) * p.cap + pos[r];
+                unsigned char* at = p.spill + (ull)idx * 16ull;
+                *reinterpret_cast<ulonglong2*>(at) = make_ulonglong2(key, prod[r]);
+                // a 16-byte store into a line that is not in L2 stalls on a write-miss fill; two
+                // entries before this buffer moves on to its next 128-byte line, pull that line in
+                if ((pos[r] & 7u) == 6) asm volatile("prefetch.global.L2 [%0];" ::"l"(at + 32));
             } else {
                 table_accumulate(p.t, key, h[r], prod[r], 0, 1);  // buffer full: exact slow path
             }
@@ -267,7 +271,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     uint32_t spilled = 0, overflow = 0;
     for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) {
         uint32_t c = d.cursor[i];
-        p.spill_cnt[(ull)i * p.n_groups + blockIdx.x] = min(c, p.cap);
+        p.spill_cnt[((ull)blockIdx.x << p.t.lp) + i] = min(c, p.cap);
         spilled += min(c, p.cap);
         overflow += c > p.cap ? c - p.cap : 0u;
     }
@@ -299,11 +303,10 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     uint32_t* s_cnt = s_a1 + C;
     __shared__ uint32_t s_total;
     const uint32_t part = blockIdx.x;
-    const uint32_t* my_cnt = q.spill_cnt + (ull)part * q.n_groups;
     if (threadIdx.x == 0) s_total = 0;
     __syncthreads();
     uint32_t local_total = 0;
-    for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) local_total += my_cnt[g];
+    for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) local_total += q.spill_cnt[((ull)g << q.t.lp) + part];
     local_total = __reduce_add_sync(0xFFFFFFFFu, local_total);
     if ((threadIdx.x & 31u) == 0 && local_total) atomicAdd(&s_total, local_total);
     __syncthreads();
@@ -320,8 +323,8 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
 
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
     for (uint32_t g = warp; g < q.n_used; g += n_warps) {
-        const uint32_t n_e = my_cnt[g];
-        const ulonglong2* src = reinterpret_cast<const ulonglong2*>(q.spill) + ((ull)part * q.n_groups + g) * q.cap;
+        const uint32_t n_e = q.spill_cnt[((ull)g << q.t.lp) + part];
+        const ulonglong2* src = reinterpret_cast<const ulonglong2*>(q.spill) + (((ull)g << q.t.lp) + part) * q.cap;
         for (uint32_t e0 = 0; e0 < n_e; e0 += 128) {
             ulonglong2 ent[4];
             bool have[4];
@@ -387,56 +390,92 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
 }
 
 // --------------------------------------------------------------------------------------
-// Hot-directory construction: one CTA counts the keys of a strided sample of the records in
-// a shared-memory table, picks the count threshold that fills the directory, and installs the
-// selected keys, most frequent classes first, into 2-slot buckets.  Which keys end up in the
-// directory only affects speed, never results.
-constexpr uint32_t SAMPLE_SLOTS = 16384;
-constexpr uint32_t SAMPLE_PROBES = 8;
+// Hot-directory construction, three small kernels over a strided sample of the records:
+//   1. count   every sampled key bumps one of 65536 counters chosen by its hash;
+//   2. admit   sampled keys whose counter reached ADMIT_MIN are inserted, with exact counts,
+//              into a candidate table (colliding cold keys may slip in; harmless);
+//   3. select  one CTA picks the count threshold that fills the directory and installs the
+//              candidates, most frequent classes first, into 2-slot buckets.
+// Which keys end up in the directory only affects speed, never results.
+constexpr uint32_t SKETCH_BITS = 16;
+constexpr uint32_t ADMIT_MIN = 3;
+constexpr uint32_t CAND_PROBES = 16;
 
-__global__ void __launch_bounds__(1024, 1) hot_build_kernel(HotBuildParams p) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    ull* skeys = reinterpret_cast<ull*>(smem_raw);
-    uint32_t* scnt = reinterpret_cast<uint32_t*>(smem_raw + (size_t)SAMPLE_SLOTS * 8);
-    __shared__ uint32_t hist[256];
-    __shared__ uint32_t s_thr, s_inserted;
-    for (uint32_t i = threadIdx.x; i < SAMPLE_SLOTS; i += blockDim.x) {
-        skeys[i] = 0;
-        scnt[i] = 0;
+__device__ __forceinline__ bool sample_key(const HotBuildParams& p, uint32_t j, ull* key) {
+    uint4 v = p.recs[(ull)j * p.stride];
+    uint32_t khi = v.y & 0x00FFFFFFu;
+    *key = ((ull)khi << 32) | v.z;
+    return v.x < p.n_apps && (khi >> 16) < p.n_phases;
+}
+
+// Lanes of a warp that target the same counter are combined first, so that a trace dominated
+// by one key does not serialise on one address.
+__device__ __forceinline__ void combined_count(uint32_t* counters, uint32_t index, bool active) {
+    unsigned act = __ballot_sync(0xFFFFFFFFu, active);
+    if (!active) return;
+    unsigned same = __match_any_sync(act, index);
+    if ((threadIdx.x & 31u) == (unsigned)(__ffs(same) - 1)) atomicAdd(&counters[index], (uint32_t)__popc(same));
+}
+
+__global__ void __launch_bounds__(256) hot_count_kernel(HotBuildParams p) {
+    const uint32_t stride = gridDim.x * blockDim.x;
+    const uint32_t rounds = (p.n_sample + stride - 1) / stride;  // uniform trip count: warp collectives inside
+    for (uint32_t r = 0; r < rounds; ++r) {
+        uint32_t j = r * stride + blockIdx.x * blockDim.x + threadIdx.x;
+        ull key = 0;
+        bool ok = j < p.n_sample && sample_key(p, j, &key);
+        combined_count(p.sketch, hash32(key) >> (32 - SKETCH_BITS), ok);
     }
+}
+
+__global__ void __launch_bounds__(256) hot_admit_kernel(HotBuildParams p) {
+    const uint32_t stride = gridDim.x * blockDim.x;
+    const uint32_t rounds = (p.n_sample + stride - 1) / stride;
+    for (uint32_t r = 0; r < rounds; ++r) {
+        uint32_t j = r * stride + blockIdx.x * blockDim.x + threadIdx.x;
+        ull key = 0;
+        bool ok = j < p.n_sample && sample_key(p, j, &key);
+        uint32_t h = hash32(key);
+        ok = ok && p.sketch[h >> (32 - SKETCH_BITS)] >= ADMIT_MIN;
+        const ull skey = ~key;
+        uint32_t s = (h * 0x9E3779B1u) >> (32 - p.cand_bits);
+        bool found = false;
+        if (ok) {
+            for (uint32_t probe = 0; probe < CAND_PROBES && !found; ++probe) {
+                ull k = ld_relaxed(&p.cand_keys[s]);
+                if (k == 0) {
+                    k = atomicCAS(&p.cand_keys[s], 0ull, skey);
+                    if (k == 0) k = skey;
+                }
+                if (k == skey)
+                    found = true;
+                else
+                    s = (s + 1) & ((1u << p.cand_bits) - 1);
+            }
+        }
+        combined_count(p.cand_cnt, s, found);
+    }
+}
+
+__global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
+    __shared__ uint32_t hist[1024];
+    __shared__ uint32_t s_thr, s_inserted, s_max;
+    const uint32_t n_cand = 1u << p.cand_bits;
+    hist[threadIdx.x] = 0;
+    if (threadIdx.x == 0) s_max = 0;
     for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) p.hot_keys[i] = 0;
-    if (threadIdx.x < 256) hist[threadIdx.x] = 0;
     if (threadIdx.x == 0) s_inserted = 0;
     __syncthreads();
-
-    for (uint32_t j = threadIdx.x; j < p.n_sample; j += blockDim.x) {
-        uint4 v = p.recs[(ull)j * p.stride];
-        uint32_t phase = (v.y >> 16) & 0xFFu;
-        if (v.x >= p.n_apps || phase >= p.n_phases) continue;
-        ull key = pack_key(phase, v.y & 0xFFFFu, v.z);
-        ull skey = ~key;
-        uint32_t s = hash32(key) >> 18;  // 14 bits
-        for (uint32_t probe = 0; probe < SAMPLE_PROBES; ++probe) {
-            ull k = skeys[s];
-            if (k == 0) {
-                k = atomicCAS(&skeys[s], 0ull, skey);
-                if (k == 0) k = skey;
-            }
-            if (k == skey) {
-                atomicAdd(&scnt[s], 1u);
-                break;
-            }
-            s = (s + 1) & (SAMPLE_SLOTS - 1);
-        }
+    for (uint32_t i = threadIdx.x; i < n_cand; i += blockDim.x) {
+        uint32_t c = p.cand_cnt[i];
+        if (c != 0) atomicAdd(&hist[min(c, 1023u)], 1u);
+        if (c >= 1023u) atomicMax(&s_max, c);
     }
-    __syncthreads();
-    for (uint32_t i = threadIdx.x; i < SAMPLE_SLOTS; i += blockDim.x)
-        if (scnt[i] != 0) atomicAdd(&hist[min(scnt[i], 255u)], 1u);
     __syncthreads();
     if (threadIdx.x == 0) {
         // smallest threshold >= 2 whose class fits the directory with some over-subscription
-        uint32_t budget = p.hot_slots + p.hot_slots / 4, cum = 0, thr = 256;
-        for (int c = 255; c >= 2; --c) {
+        uint32_t budget = p.hot_slots + p.hot_slots / 4, cum = 0, thr = 1024;
+        for (int c = 1023; c >= 2; --c) {
             if (cum + hist[c] > budget) break;
             cum += hist[c];
             thr = (uint32_t)c;
@@ -444,20 +483,18 @@ __global__ void __launch_bounds__(1024, 1) hot_build_kernel(HotBuildParams p) {
         s_thr = thr;
         // a key holding more than 1/32 of the sample makes same-slot collisions inside a warp
         // common: tell the scatter pass to combine equal lanes first
-        uint32_t top = 255;
-        while (top > 0 && hist[top] == 0) --top;
-        p.ctl->hot_skew = (top >= 255 || top * 32u >= p.n_sample) ? 1ull : 0ull;
+        p.ctl->hot_skew = ((ull)s_max * 32u >= p.n_sample) ? 1ull : 0ull;
     }
     __syncthreads();
     const uint32_t thr = s_thr;
-    const uint32_t bounds[5] = {0xFFFFFFFFu, 128u, 32u, 8u, 2u};
-    for (int round = 0; round < 4; ++round) {
+    const uint32_t bounds[6] = {0xFFFFFFFFu, 512u, 128u, 32u, 8u, 2u};
+    for (int round = 0; round < 5; ++round) {
         uint32_t hi = bounds[round], lo = max(bounds[round + 1], thr);
         if (lo < hi) {
-            for (uint32_t i = threadIdx.x; i < SAMPLE_SLOTS; i += blockDim.x) {
-                uint32_t c = scnt[i];
+            for (uint32_t i = threadIdx.x; i < n_cand; i += blockDim.x) {
+                uint32_t c = p.cand_cnt[i];
                 if (c >= lo && c < hi) {
-                    ull skey = skeys[i];
+                    ull skey = p.cand_keys[i];
                     uint32_t b = dir_bucket(hash32(~skey), p.hot_slots / 2) * 2;
                     if (atomicCAS(&p.hot_keys[b], 0ull, skey) == 0 || atomicCAS(&p.hot_keys[b + 1], 0ull, skey) == 0)
                         atomicAdd(&s_inserted, 1u);
@@ -488,7 +525,7 @@ cudaError_t ingest_prepare() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(partition_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(hot_build_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SAMPLE_SLOTS * 12);
+    return cudaSuccess;
 }
 
 cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream) {
@@ -505,8 +542,13 @@ cudaError_t launch_partition(const PartitionParams& q, cudaStream_t stream) {
     return cudaGetLastError();
 }
 
-cudaError_t launch_hot_build(const HotBuildParams& p, cudaStream_t stream) {
-    hot_build_kernel<<<1, 1024, SAMPLE_SLOTS * 12, stream>>>(p);
+cudaError_t launch_hot_build(const HotBuildParams& p, int n_sms, cudaStream_t stream) {
+    // the caller has zeroed the sketch and the candidate table on this stream
+    int grid = (int)((p.n_sample + 255) / 256);
+    if (grid > n_sms * 8) grid = n_sms * 8;
+    hot_count_kernel<<<grid, 256, 0, stream>>>(p);
+    hot_admit_kernel<<<grid, 256, 0, stream>>>(p);
+    hot_select_kernel<<<1, 1024, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

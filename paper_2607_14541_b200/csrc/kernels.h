@@ -16,9 +16,9 @@ struct IngestParams {
     uint32_t hot_slots;        // even
     uint32_t hot_buckets;      // hot_slots / 2
     TableRef t;
-    // spill buffers: entry (p, g, i) at spill + ((p * n_groups + g) * cap + i) * 16 bytes
+    // spill buffers: entry i of scatter CTA g for partition p at spill + ((g * P + p) * cap + i) * 16 bytes
     unsigned char* spill;
-    uint32_t* spill_cnt;       // [P][n_groups]
+    uint32_t* spill_cnt;       // [n_groups][P]
     uint32_t n_groups;         // G, row pitch of the buffers (= CTAs of the widest scatter launch)
     uint32_t cap;              // entries per (partition, CTA) buffer
 };
@@ -39,6 +39,10 @@ struct HotBuildParams {
     uint32_t n_apps, n_phases;
     ull* hot_keys;
     uint32_t hot_slots;
+    uint32_t* sketch;          // [65536] sample counters by hash
+    ull* cand_keys;            // [1 << cand_bits] candidate table: ~key, 0 = empty
+    uint32_t* cand_cnt;        // [1 << cand_bits] exact sample counts of the candidates
+    uint32_t cand_bits;
     Control* ctl;
 };
 
@@ -74,7 +78,7 @@ struct TopkParams {
 cudaError_t ingest_prepare();
 cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream);
 cudaError_t launch_partition(const PartitionParams& p, cudaStream_t stream);
-cudaError_t launch_hot_build(const HotBuildParams& p, cudaStream_t stream);
+cudaError_t launch_hot_build(const HotBuildParams& p, int n_sms, cudaStream_t stream);
 cudaError_t launch_merge(const atrex_entry_t* in, ull n, const TableRef& t, int grid, cudaStream_t stream);
 
 cudaError_t finalize_prepare();
