@@ -66,7 +66,7 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     L->lp = LP_MIN;
     while (L->lp < LP_MAX && (need + (1ull << L->lp) - 1) / (1ull << L->lp) > c_max) ++L->lp;
     ull per = (need + (1ull << L->lp) - 1) >> L->lp;
-    if (per > c_max) per = c_max;
+    if (per > c_max || L->lp > LP_MIN) per = c_max;  // big tables: use all of shared memory, lower load factor
     if (per < 128) per = 128;
     L->C = (uint32_t)((per + 31) / 32 * 32);
     L->n_slots = (ull)L->C << L->lp;
@@ -381,7 +381,7 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
     q.n_groups = h->L.n_groups;
     q.n_used = (uint32_t)grid;
     q.cap = h->L.cap;
-    CU(h, launch_partition(q, s));
+    CU(h, launch_partition(q, h->n_sms, s));
     h->launches += 2;
     return ATREX_OK;
 }

@@ -112,6 +112,7 @@ __device__ __forceinline__ uint32_t part_of(uint32_t h, uint32_t lp) { return h 
 
 // start slot inside the partition, from the hash bits below the partition bits
 __device__ __forceinline__ uint32_t local_of(uint32_t h, uint32_t lp, uint32_t C) { return __umulhi(h << lp, C); }
+// (probe sequences start at the even slot at or below this one and then visit consecutive slots)
 
 // Find (or claim) the slot of `key` directly in HBM.  Returns NO_INDEX when the key's
 // partition has no free slot.  Used off the hot path: directory flush, buffer overflow,
@@ -119,7 +120,7 @@ __device__ __forceinline__ uint32_t local_of(uint32_t h, uint32_t lp, uint32_t C
 __device__ __forceinline__ ull find_or_claim(const TableRef& t, ull key, uint32_t h) {
     const ull skey = ~key;
     const ull base = (ull)part_of(h, t.lp) * t.C;
-    uint32_t s = local_of(h, t.lp, t.C);
+    uint32_t s = local_of(h, t.lp, t.C) & ~1u;
     for (uint32_t probe = 0; probe < t.C; ++probe) {
         ull* kp = t.keys + base + s;
         ull k = ld_relaxed(kp);

@@ -25,6 +25,8 @@
 // All sums are integers, so the result does not depend on which route a record took, on
 // scheduling, or on chunking.  Entries that do not fit a spill buffer, directory wraps and
 // merges fall back to exact atomic updates of the HBM table.
+#include <type_traits>
+
 #include "atrex_dev.cuh"
 #include "kernels.h"
 
@@ -50,7 +52,9 @@ struct SmemDir {
     uint32_t* a1;     // [slots] ... and bits 32..63 (carries of a0 are added here by the adder)
     uint32_t* cnt;    // [slots] this launch's record count of the slot
     uint32_t* cursor; // [P] entries appended to this CTA's buffer of each partition
-    const uint32_t* appw;
+    const uint32_t* appw_s;  // card-hour weights in shared memory (when they fit) ...
+    const uint32_t* appw_g;  // ... else in global memory
+    bool appw_shared;
 };
 
 // Shared-memory accumulation uses native 32-bit atomics only (64-bit shared atomics are
@@ -92,7 +96,7 @@ __device__ __forceinline__ void dir_add(const SmemDir& d, uint32_t slot, ull v, 
 
 // Process R records held in registers by every lane of the warp (absent ones masked).
 // Written in stages over the R records so that their shared-memory round trips overlap.
-template <bool HOT, bool DEDUPE, int R>
+template <bool HOT, bool DEDUPE, bool FULL, int R>
 __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&present)[R], const IngestParams& p,
                                         const SmemDir& d, uint32_t& rejected) {
     uint32_t khi[R], h[R];
@@ -102,9 +106,10 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
     for (int r = 0; r < R; ++r) {
         uint32_t app = w[r][0];
         khi[r] = w[r][1] & 0x00FFFFFFu;                 // phase << 16 | op_id: the key's high word
-        bool ok = present[r] && app < p.n_apps && (khi[r] >> 16) < p.n_phases;
-        rejected += (present[r] && !ok) ? 1u : 0u;
-        uint32_t wgt = d.appw[ok ? app : 0u];
+        bool ok = (FULL || present[r]) && app < p.n_apps && (khi[r] >> 16) < p.n_phases;
+        rejected += ((FULL || present[r]) && !ok) ? 1u : 0u;
+        // card-hour weight: from shared memory when the table fits there, else from global
+        uint32_t wgt = d.appw_shared ? d.appw_s[ok ? app : 0u] : __ldg(d.appw_g + (ok ? app : 0u));
         prod[r] = (ull)wgt * (ull)w[r][3];
         h[r] = hash32(khi[r], w[r][2]);
         todo[r] = ok;
@@ -170,20 +175,27 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
 
 template <bool HOT, bool DEDUPE>
 __device__ __forceinline__ void scatter_body(const IngestParams& p, const SmemDir& d, uint32_t& rejected) {
-    // two 32-byte loads (four records) in flight per thread: the next pair is requested before
-    // the current one is processed
+    // Each thread keeps two 32-byte loads (four records) in flight: the pair after next is
+    // requested before the current pair is processed.  CTA b handles pairs
+    // (b + k * gridDim) * 1024 + tid; rounds in which every CTA's tile is complete need no
+    // bounds checks, the last (ragged) ones are predicated.
     const unsigned char* body = reinterpret_cast<const unsigned char*>(p.body);
     const ull stride = (ull)gridDim.x * INGEST_THREADS;
+    const ull full_rounds = p.n_pairs / stride;                    // rounds complete for every CTA
+    const ull rounds = (p.n_pairs + stride - 1) / stride;
+    const ull first = (ull)blockIdx.x * INGEST_THREADS + threadIdx.x;
     uint32_t rawA[8], rawB[8];
-    auto fetch = [&](ull i, uint32_t (&raw)[8]) {
-        if (i < p.n_pairs) {
+    auto fetch = [&](ull round, uint32_t (&raw)[8]) {
+        ull i = first + round * stride;
+        if (round < full_rounds || (round < rounds && i < p.n_pairs)) {
             ld_stream_256(body + i * 32, raw);
         } else {
 #pragma unroll
             for (int j = 0; j < 8; ++j) raw[j] = 0;
         }
     };
-    auto consume = [&](ull i, const uint32_t (&raw)[8]) {
+    auto consume = [&](ull round, const uint32_t (&raw)[8], auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
         uint32_t w[2][4];
         bool present[2];
 #pragma unroll
@@ -191,23 +203,35 @@ __device__ __forceinline__ void scatter_body(const IngestParams& p, const SmemDi
             w[0][j] = raw[j];
             w[1][j] = raw[4 + j];
         }
-        present[0] = present[1] = i < p.n_pairs;
-        process<HOT, DEDUPE, 2>(w, present, p, d, rejected);
+        present[0] = present[1] = FULL || (first + round * stride) < p.n_pairs;
+        process<HOT, DEDUPE, FULL, 2>(w, present, p, d, rejected);
     };
-    const ull first = (ull)blockIdx.x * INGEST_THREADS;
-    fetch(first + threadIdx.x, rawA);
-    fetch(first + stride + threadIdx.x, rawB);
-    for (ull base = first; base < p.n_pairs; base += 2 * stride) {  // CTA-uniform trip count
-        ull i = base + threadIdx.x;
+    using True = std::integral_constant<bool, true>;
+    using False = std::integral_constant<bool, false>;
+    fetch(0, rawA);
+    fetch(1, rawB);
+    ull round = 0;
+    for (; round + 2 <= full_rounds; round += 2) {
         uint32_t cur[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) cur[j] = rawA[j];
-        fetch(i + 2 * stride, rawA);
-        consume(i, cur);
+        fetch(round + 2, rawA);
+        consume(round, cur, True{});
 #pragma unroll
         for (int j = 0; j < 8; ++j) cur[j] = rawB[j];
-        fetch(i + 3 * stride, rawB);
-        consume(i + stride, cur);
+        fetch(round + 3, rawB);
+        consume(round + 1, cur, True{});
+    }
+    for (; round < rounds; round += 2) {  // ragged tail, predicated
+        uint32_t cur[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cur[j] = rawA[j];
+        fetch(round + 2, rawA);
+        consume(round, cur, False{});
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cur[j] = rawB[j];
+        fetch(round + 3, rawB);
+        consume(round + 1, cur, False{});
     }
     // records that do not form an aligned pair (at most one before and one after the body)
     if (blockIdx.x == 0 && threadIdx.x < 32) {
@@ -219,7 +243,7 @@ __device__ __forceinline__ void scatter_body(const IngestParams& p, const SmemDi
             w1[0][0] = v.x; w1[0][1] = v.y; w1[0][2] = v.z; w1[0][3] = v.w;
             pr[0] = true;
         }
-        process<HOT, DEDUPE, 1>(w1, pr, p, d, rejected);
+        process<HOT, DEDUPE, false, 1>(w1, pr, p, d, rejected);
     }
 }
 
@@ -243,10 +267,12 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     if (p.appw_in_smem) {
         uint32_t* s_appw = reinterpret_cast<uint32_t*>(sp);
         for (uint32_t i = threadIdx.x; i < p.n_apps; i += blockDim.x) s_appw[i] = p.app_w[i];
-        d.appw = s_appw;
+        d.appw_s = s_appw;
     } else {
-        d.appw = p.app_w;
+        d.appw_s = reinterpret_cast<uint32_t*>(sp);
     }
+    d.appw_g = p.app_w;
+    d.appw_shared = p.appw_in_smem != 0;
     if (HOT) {
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
             d.keys[i] = p.hot_keys[i];
@@ -293,7 +319,11 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
 }
 
 // --------------------------------------------------------------------------------------
-// Pass 2: one CTA aggregates one partition entirely in shared memory.
+// Pass 2: a CTA aggregates one partition at a time entirely in shared memory.  CTAs are
+// persistent and take partitions blockIdx.x, blockIdx.x + gridDim.x, ...; while one partition
+// is processed, the next one's keys and spill entries are pulled into L2.
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
 __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionParams q) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t C = q.t.C;
@@ -302,90 +332,131 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     uint32_t* s_a1 = s_a0 + C;
     uint32_t* s_cnt = s_a1 + C;
     __shared__ uint32_t s_total;
-    const uint32_t part = blockIdx.x;
-    if (threadIdx.x == 0) s_total = 0;
-    __syncthreads();
-    uint32_t local_total = 0;
-    for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) local_total += q.spill_cnt[((ull)g << q.t.lp) + part];
-    local_total = __reduce_add_sync(0xFFFFFFFFu, local_total);
-    if ((threadIdx.x & 31u) == 0 && local_total) atomicAdd(&s_total, local_total);
-    __syncthreads();
-    if (s_total == 0) return;  // nothing was spilled to this partition
-
-    const ull base = (ull)part * C;
-    for (uint32_t i = threadIdx.x; i < C; i += blockDim.x) {
-        s_keys[i] = q.t.keys[base + i];
-        s_a0[i] = 0;
-        s_a1[i] = 0;
-        s_cnt[i] = 0;
-    }
-    __syncthreads();
-
+    const uint32_t n_parts = 1u << q.t.lp;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
-    for (uint32_t g = warp; g < q.n_used; g += n_warps) {
-        const uint32_t n_e = q.spill_cnt[((ull)g << q.t.lp) + part];
-        const ulonglong2* src = reinterpret_cast<const ulonglong2*>(q.spill) + (((ull)g << q.t.lp) + part) * q.cap;
-        for (uint32_t e0 = 0; e0 < n_e; e0 += 128) {
-            ulonglong2 ent[4];
-            bool have[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                uint32_t e = e0 + u * 32 + lane;
-                have[u] = e < n_e;
-                if (have[u]) ent[u] = __ldcs(src + e);
+
+    for (uint32_t part = blockIdx.x; part < n_parts; part += gridDim.x) {
+        if (threadIdx.x == 0) s_total = 0;
+        __syncthreads();  // also: the previous partition's write-back has finished reading shared memory
+        uint32_t local_total = 0;
+        for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) local_total += q.spill_cnt[((ull)g << q.t.lp) + part];
+        local_total = __reduce_add_sync(0xFFFFFFFFu, local_total);
+        if (lane == 0 && local_total) atomicAdd(&s_total, local_total);
+
+        __syncthreads();
+        if (s_total == 0) continue;  // nothing was spilled to this partition (uniform)
+
+        const ull base = (ull)part * C;
+        for (uint32_t i = threadIdx.x; i < C; i += blockDim.x) {
+            s_keys[i] = q.t.keys[base + i];
+            s_a0[i] = 0;
+            s_a1[i] = 0;
+            s_cnt[i] = 0;
+        }
+        __syncthreads();
+
+        for (uint32_t g = warp; g < q.n_used; g += n_warps) {
+            const ull sb = ((ull)g << q.t.lp) + part;
+            const uint32_t n_e = q.spill_cnt[sb];
+            const ulonglong2* src = reinterpret_cast<const ulonglong2*>(q.spill) + sb * q.cap;
+            if (g + n_warps < q.n_used) {  // short-distance prefetch: this warp's next sub-buffer
+                const ull nb = ((ull)(g + n_warps) << q.t.lp) + part;
+                const uint32_t bytes = q.spill_cnt[nb] * 16u;
+                const unsigned char* nsrc = q.spill + nb * q.cap * 16ull;
+                for (uint32_t off = lane * 128u; off < bytes; off += 32u * 128u) prefetch_l2(nsrc + off);
             }
+            for (uint32_t e0 = 0; e0 < n_e; e0 += 128) {
+                ull skey[4], v[4];
+                uint32_t slot[4];
+                bool searching[4], ok[4];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const ull key = ent[u].x, v = ent[u].y, skey = ~key;
-                uint32_t s = local_of(hash32(key), q.t.lp, C);
-                // warp-convergent probe: every lane steps until all lanes have their slot
-                bool searching = have[u], ok = have[u];
+                for (int u = 0; u < 4; ++u) {
+                    uint32_t e = e0 + u * 32 + lane;
+                    ok[u] = e < n_e;
+                    ulonglong2 ent = ok[u] ? __ldcs(src + e) : make_ulonglong2(0, 0);
+                    skey[u] = ~ent.x;
+                    v[u] = ent.y;
+                    slot[u] = local_of(hash32(ent.x), q.t.lp, C) & ~1u;  // probe sequence starts at an even slot
+                    searching[u] = ok[u];
+                }
+                // warp-convergent probe of all four entries, two slots per 16-byte load
                 uint32_t steps = 0;
-                while (__any_sync(0xFFFFFFFFu, searching)) {
-                    if (searching) {
-                        ull k = s_keys[s];
-                        if (k == 0) {
-                            k = atomicCAS(&s_keys[s], 0ull, skey);
-                            if (k == 0) {
-                                atomicOr(&s_cnt[s], NEW_KEY_FLAG);
-                                k = skey;
+                while (__any_sync(0xFFFFFFFFu, searching[0] | searching[1] | searching[2] | searching[3])) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (!searching[u]) continue;
+                        const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(s_keys + slot[u]);
+                        if (kk.x == skey[u]) {
+                            searching[u] = false;
+                        } else if (kk.x == 0) {
+                            ull old = atomicCAS(&s_keys[slot[u]], 0ull, skey[u]);  // lost races re-read the pair
+                            if (old == 0) atomicOr(&s_cnt[slot[u]], NEW_KEY_FLAG);
+                            if (old == 0 || old == skey[u]) searching[u] = false;
+                        } else if (kk.y == skey[u]) {
+                            slot[u] += 1;
+                            searching[u] = false;
+                        } else if (kk.y == 0) {
+                            ull old = atomicCAS(&s_keys[slot[u] + 1], 0ull, skey[u]);
+                            if (old == 0) atomicOr(&s_cnt[slot[u] + 1], NEW_KEY_FLAG);
+                            if (old == 0 || old == skey[u]) {
+                                slot[u] += 1;
+                                searching[u] = false;
                             }
-                        }
-                        if (k == skey) {
-                            searching = false;
                         } else {
-                            s = (s + 1 == C) ? 0u : s + 1;
-                            if (++steps >= C) {  // partition full
-                                searching = false;
-                                ok = false;
+                            slot[u] = (slot[u] + 2 >= C) ? 0u : slot[u] + 2;
+                        }
+                    }
+                    if (++steps > 2 * C) {  // partition full (bounded; counts lost races too)
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (searching[u]) {
+                                searching[u] = false;
+                                ok[u] = false;
                                 atomicOr(&q.t.ctl->status, ST_TABLE_FULL);
                                 atomicAdd(&q.t.ctl->n_dropped, 1ull);
                             }
                         }
                     }
                 }
-                if (ok && limbs_add(&s_a0[s], &s_a1[s], &s_cnt[s], v, 1u)) {
-                    // drain: this CTA owns the slot, so adds into HBM are exact; the write-back
-                    // below adds on top of them
-                    ull hi, lo = limbs_drain(&s_a0[s], &s_a1[s], &hi);
-                    ull* vp = reinterpret_cast<ull*>(q.t.vals + base + s);
-                    ull old = atomicAdd(vp, lo);
-                    hi += (old + lo < old) ? 1ull : 0ull;
-                    if (hi) atomicAdd(vp + 1, hi << HI_SHIFT);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (ok[u] && limbs_add(&s_a0[slot[u]], &s_a1[slot[u]], &s_cnt[slot[u]], v[u], 1u)) {
+                        // drain: this CTA owns the slot, so adds into HBM are exact; the write-back
+                        // below adds on top of them
+                        ull hi, lo = limbs_drain(&s_a0[slot[u]], &s_a1[slot[u]], &hi);
+                        ull* vp = reinterpret_cast<ull*>(q.t.vals + base + slot[u]);
+                        ull old = atomicAdd(vp, lo);
+                        hi += (old + lo < old) ? 1ull : 0ull;
+                        if (hi) atomicAdd(vp + 1, hi << HI_SHIFT);
+                    }
                 }
             }
         }
-    }
-    __syncthreads();
-    for (uint32_t i = threadIdx.x; i < C; i += blockDim.x) {
-        uint32_t c = s_cnt[i];
-        if (c == 0) continue;
-        ull* vp = reinterpret_cast<ull*>(q.t.vals + base + i);
-        ull lo = ld_relaxed(vp), cnthi = ld_relaxed(vp + 1);
-        ull nlo = lo + ((ull)s_a0[i] | ((ull)s_a1[i] << 32));
-        cnthi += (ull)(c & ~NEW_KEY_FLAG) + ((nlo < lo ? 1ull : 0ull) << HI_SHIFT);
-        *reinterpret_cast<ulonglong2*>(vp) = make_ulonglong2(nlo, cnthi);
-        if (c & NEW_KEY_FLAG) q.t.keys[base + i] = s_keys[i];
+        __syncthreads();
+        {   // while the deltas are written back, pull the next partition's keys and each warp's
+            // first sub-buffer towards L2 (used within microseconds, so they are still there)
+            const uint32_t next = part + gridDim.x;
+            if (next < n_parts) {
+                const unsigned char* nk = reinterpret_cast<const unsigned char*>(q.t.keys + (ull)next * C);
+                for (uint32_t off = threadIdx.x * 128u; off < C * 8u; off += blockDim.x * 128u) prefetch_l2(nk + off);
+                if (warp < q.n_used) {
+                    const ull nb = ((ull)warp << q.t.lp) + next;
+                    const uint32_t bytes = q.spill_cnt[nb] * 16u;
+                    const unsigned char* nsrc = q.spill + nb * q.cap * 16ull;
+                    for (uint32_t off = lane * 128u; off < bytes; off += 32u * 128u) prefetch_l2(nsrc + off);
+                }
+            }
+        }
+        for (uint32_t i = threadIdx.x; i < C; i += blockDim.x) {
+            uint32_t c = s_cnt[i];
+            if (c == 0) continue;
+            ull* vp = reinterpret_cast<ull*>(q.t.vals + base + i);
+            ull lo = ld_relaxed(vp), cnthi = ld_relaxed(vp + 1);
+            ull nlo = lo + ((ull)s_a0[i] | ((ull)s_a1[i] << 32));
+            cnthi += (ull)(c & ~NEW_KEY_FLAG) + ((nlo < lo ? 1ull : 0ull) << HI_SHIFT);
+            *reinterpret_cast<ulonglong2*>(vp) = make_ulonglong2(nlo, cnthi);
+            if (c & NEW_KEY_FLAG) q.t.keys[base + i] = s_keys[i];
+        }
     }
 }
 
@@ -537,8 +608,9 @@ cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream
     return cudaGetLastError();
 }
 
-cudaError_t launch_partition(const PartitionParams& q, cudaStream_t stream) {
-    partition_kernel<<<1u << q.t.lp, INGEST_THREADS, (size_t)q.t.C * 20, stream>>>(q);
+cudaError_t launch_partition(const PartitionParams& q, int n_sms, cudaStream_t stream) {
+    int grid = (int)(1u << q.t.lp) < n_sms ? (int)(1u << q.t.lp) : n_sms;
+    partition_kernel<<<grid, INGEST_THREADS, (size_t)q.t.C * 20, stream>>>(q);
     return cudaGetLastError();
 }
 

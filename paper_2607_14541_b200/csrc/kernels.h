@@ -77,7 +77,7 @@ struct TopkParams {
 
 cudaError_t ingest_prepare();
 cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream);
-cudaError_t launch_partition(const PartitionParams& p, cudaStream_t stream);
+cudaError_t launch_partition(const PartitionParams& p, int n_sms, cudaStream_t stream);
 cudaError_t launch_hot_build(const HotBuildParams& p, int n_sms, cudaStream_t stream);
 cudaError_t launch_merge(const atrex_entry_t* in, ull n, const TableRef& t, int grid, cudaStream_t stream);
 
