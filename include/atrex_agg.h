@@ -57,7 +57,8 @@ typedef enum {
     ATREX_ERR_CUDA = -4,           /* a CUDA runtime call failed (see atrex_agg_last_cuda_error)        */
     ATREX_ERR_TIMEOUT = -5,        /* a bounded device-side wait gave up                                */
     ATREX_ERR_STATE = -6,          /* call order: topk before finalize, or > 2^40 records               */
-    ATREX_ERR_NOMEM = -7           /* workspace too small / allocation failed                           */
+    ATREX_ERR_NOMEM = -7,          /* workspace too small / allocation failed                           */
+    ATREX_ERR_TOO_LARGE = -8       /* input larger than a fixed-size internal buffer can take           */
 } atrex_status_t;
 
 /* One observed device-kernel invocation (Sec. 3.1; the d_{a,phi,r,l} of Eq. 2). 16 bytes. */
@@ -186,6 +187,36 @@ int atrex_agg_last_cuda_error(const atrex_agg_t*);
 
 /* Number of kernels this handle has launched so far (for launch accounting in benchmarks). */
 uint64_t atrex_agg_launch_count(const atrex_agg_t*);
+
+/* Ranked top-k over an array of entries, for callers that cannot allocate device memory.
+ *
+ * (The paper has no counterpart to this call; it exists for deployment reasons only.)
+ *
+ * Who this is for: code that runs where nobody may call cudaMalloc -- a service whose device
+ * memory was divided up at start-up, a plugin that receives buffers but no allocator, a process
+ * whose memory pool belongs to another component.  atrex_agg_topk ranks out of a handle's
+ * workspace, and that workspace had to be allocated by someone.  This call takes no handle: it
+ * ranks `n` entries the caller already holds on the device (for instance atrex_agg_finalize's
+ * output, or entries received from elsewhere) and keeps its selection buffer in a fixed array
+ * inside the library image.  It calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   d_entries  DEVICE, n entries (8-byte aligned); key, wt_lo, wt_hi decide the ranking, the
+ *              whole 48-byte entry is copied to the output unchanged
+ *   n, k       at most ATREX_STATIC_TOPK_MAX_ENTRIES each; larger values are refused with
+ *              ATREX_ERR_TOO_LARGE and nothing runs
+ *   d_out      DEVICE, capacity k entries: the min(k, entries of `phase`) best entries of that
+ *              phase, by weighted time descending (exact 128-bit compare), then key ascending
+ *   h_n_out    HOST, number of entries written
+ *
+ * The fixed array costs 2 MiB + 256 bytes of device memory on every GPU that loads the library,
+ * until the process exits.  All calls on a device share it and it keeps the previous call's
+ * contents, so the call clears it first; two calls whose GPU work overlaps (different streams
+ * or threads) would race on it -- keep them ordered.  The first call on each device also looks
+ * up the array's device address; make that first call outside any stream capture.  The call
+ * synchronises `stream` before returning. */
+#define ATREX_STATIC_TOPK_MAX_ENTRIES 65536u
+int atrex_topk_entries_static(const atrex_entry_t* d_entries, uint64_t n, uint32_t phase, uint32_t k,
+                              atrex_entry_t* d_out, uint32_t* h_n_out, void* stream);
 
 #ifdef __cplusplus
 }

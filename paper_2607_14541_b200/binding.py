@@ -27,6 +27,8 @@ ATREX_ERR_CUDA = -4
 ATREX_ERR_TIMEOUT = -5
 ATREX_ERR_STATE = -6
 ATREX_ERR_NOMEM = -7
+ATREX_ERR_TOO_LARGE = -8
+ATREX_STATIC_TOPK_MAX_ENTRIES = 65536
 
 RECORD_DTYPE = np.dtype([("app_id", "<u4"), ("op_id", "<u2"), ("phase", "u1"), ("pad", "u1"),
                          ("shape_id", "<u4"), ("duration_ns", "<u4")])
@@ -38,7 +40,7 @@ EXPORTED_SYMBOLS = [
     "atrex_agg_workspace_bytes", "atrex_agg_create", "atrex_agg_set_work_table", "atrex_agg_ingest",
     "atrex_agg_ingest_host", "atrex_agg_merge", "atrex_agg_finalize", "atrex_agg_topk", "atrex_agg_stats",
     "atrex_agg_reset", "atrex_agg_destroy", "atrex_strerror", "atrex_agg_last_cuda_error",
-    "atrex_agg_launch_count",
+    "atrex_agg_launch_count", "atrex_topk_entries_static",
 ]
 
 
@@ -84,6 +86,7 @@ def _load():
     L.atrex_agg_last_cuda_error.argtypes = [vp]
     L.atrex_agg_launch_count.restype = u64
     L.atrex_agg_launch_count.argtypes = [vp]
+    L.atrex_topk_entries_static.argtypes = [vp, u64, u32, u32, vp, C.POINTER(u32), vp]
     return L
 
 
@@ -104,6 +107,7 @@ atrex_agg_destroy = lib.atrex_agg_destroy
 atrex_strerror = lib.atrex_strerror
 atrex_agg_last_cuda_error = lib.atrex_agg_last_cuda_error
 atrex_agg_launch_count = lib.atrex_agg_launch_count
+atrex_topk_entries_static = lib.atrex_topk_entries_static
 
 
 class AtrexError(RuntimeError):
@@ -122,6 +126,22 @@ def make_peaks(peak_bw: float, peak_flops) -> atrex_hw_peaks_t:
     for i in range(ATREX_MAX_DTYPES):
         pk.peak_flops[i] = float(pf[i])
     return pk
+
+
+def topk_entries_static(entries, n: int, phase: int, k: int, out, stream=None) -> int:
+    """Rank ``n`` entries held in the CUDA tensor ``entries`` without any device allocation.
+
+    For callers that cannot allocate on the device: the selection buffer is a fixed array inside
+    the library, so ``n`` and ``k`` may be at most ATREX_STATIC_TOPK_MAX_ENTRIES.  ``out`` is a
+    caller-provided CUDA tensor with room for ``k`` 48-byte entries; returns how many were written.
+    """
+    n_out = C.c_uint32(0)
+    s = None if stream is None else (stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+    rc = atrex_topk_entries_static(entries.data_ptr() if n else None, int(n), int(phase), int(k),
+                                   out.data_ptr() if k else None, C.byref(n_out), s)
+    if rc != ATREX_OK:
+        raise AtrexError(rc, "atrex_topk_entries_static")
+    return int(n_out.value)
 
 
 class Aggregator:

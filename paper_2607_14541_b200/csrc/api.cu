@@ -581,6 +581,7 @@ const char* atrex_strerror(int status) {
         case ATREX_ERR_TIMEOUT: return "bounded device wait gave up";
         case ATREX_ERR_STATE: return "call not valid in this state";
         case ATREX_ERR_NOMEM: return "workspace too small or allocation failed";
+        case ATREX_ERR_TOO_LARGE: return "input larger than the fixed internal buffer";
         default: return "unknown status";
     }
 }

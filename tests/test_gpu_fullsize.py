@@ -1,0 +1,76 @@
+"""Parity at the benchmark's full size and launch configuration (2^30 records in 8 chunks of
+2^27, the workload bench.py times): sampled outputs the oracle computes one by one from the
+very same bytes, plus properties that hold at any size."""
+import numpy as np
+import pytest
+
+import oracle
+from tracegen.configs import make_spec
+from tracegen.layout import RECORD_DTYPE
+from tests.helpers import entry_wt, f64_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def test_full_size_chunked_trace_sampled_keys_and_invariants():
+    import torch
+    import paper_2607_14541_b200 as p
+    from tracegen.gpu import GpuSampler
+
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 << 30:
+        pytest.skip("needs ~30 GB of device memory")
+    spec = make_spec(3)
+    n, chunk = spec.n, spec.chunk_records
+    work = spec.work_table()
+    agg = p.Aggregator(spec.app_weights, spec.n_phases, spec.max_keys, max_work_rows=len(work))
+    agg.set_work_table(work)
+    sampler = GpuSampler(spec)
+    records = torch.empty(n * 16, dtype=torch.uint8, device="cuda:0")
+    sampler.fill(records, 0, n)
+    for c in range(spec.n_chunks):
+        agg.ingest(records[c * chunk * 16:(c + 1) * chunk * 16], n=chunk)
+    ent = agg.finalize_numpy(spec.peak_bw, spec.peak_flops)
+    st = agg.stats()
+
+    # properties that hold at any size
+    assert st["n_valid"] == n and st["n_rejected"] == 0 and st["n_dropped"] == 0 and st["n_overflow"] == 0
+    assert int(ent["count"].sum()) == n and len(ent) == st["n_keys"] == len(np.unique(ent["key"]))
+    for ph in range(spec.n_phases):
+        sel = ent[(ent["key"] >> np.uint64(48)) == ph]
+        tot = int(sel["wt_lo"].astype(object).sum()) + (int(sel["wt_hi"].astype(object).sum()) << 64)
+        assert tot == st["totals"][ph]
+        assert abs(float(np.sum(sel["phase_weight"], dtype=np.longdouble)) - 1.0) < 3 * len(sel) * 2.0**-53
+
+    # sampled keys: hottest, coldest and a spread in between, recomputed by the oracle from
+    # the same bytes (chunk by chunk), together with the per-phase totals as a plain sum
+    order = np.argsort(ent["count"], kind="stable")
+    pick = np.unique(np.concatenate([order[:40], order[-40:], order[:: max(1, len(order) // 120)]]))
+    keys = ent["key"][pick]
+    o = oracle.Oracle(spec.app_weights, spec.n_phases)
+    o.set_work(work)
+    acc, valid = np.zeros(16, dtype=np.uint64), np.zeros(2, dtype=np.uint64)
+    for c in range(spec.n_chunks):
+        host = records[c * chunk * 16:(c + 1) * chunk * 16].cpu().numpy().view(RECORD_DTYPE)
+        o.ingest_filtered(host, keys)
+        o.direct_totals(host, acc, valid)
+    assert int(valid[0]) == n and int(valid[1]) == 0
+    totals = [int(acc[2 * q]) | (int(acc[2 * q + 1]) << 64) for q in range(8)]
+    assert totals == st["totals"]
+    exp = o.finalize(spec.peak_bw, spec.peak_flops)          # weights here are relative to the sample only
+    got = ent[pick][np.argsort(ent["key"][pick], kind="stable")]
+    assert np.array_equal(exp["key"], got["key"])
+    assert np.array_equal(exp["count"], got["count"])
+    assert np.array_equal(exp["wt_lo"], got["wt_lo"]) and np.array_equal(exp["wt_hi"], got["wt_hi"])
+    assert np.array_equal(exp["roofline_s"].view(np.uint64), got["roofline_s"].view(np.uint64))
+    for e in got:                                            # Eq. 3 against the independently summed totals
+        t = totals[int(e["key"]) >> 48]
+        assert f64_bits(float(e["phase_weight"])) == f64_bits(oracle.u128_to_f64(entry_wt(e)) / oracle.u128_to_f64(t))
+
+    # the ranking: top-k must be the k largest (wt, then smaller key) of the phase's entries
+    for ph in range(spec.n_phases):
+        sel = ent[(ent["key"] >> np.uint64(48)) == ph]
+        wt = sel["wt_hi"].astype(object) * (1 << 64) + sel["wt_lo"].astype(object)
+        best = sorted(zip((-wt).tolist(), sel["key"].tolist()))[: spec.topk]
+        top = agg.topk(ph, spec.topk)
+        assert [int(k) for k in top["key"]] == [k for _, k in best]
