@@ -122,6 +122,9 @@ typedef struct {
     uint64_t hot_slots;                   /* keys currently in the shared-memory hot directory */
     uint64_t n_spilled;                   /* records that went through the partition spill buffers */
     uint64_t n_overflow;                  /* records that found their spill buffer full (slow exact path) */
+    uint64_t max_spill_fill;              /* fullest spill buffer seen since reset, in entries */
+    uint64_t spill_cap;                   /* capacity of one spill buffer, in entries */
+    uint64_t n_drains;                    /* partition passes that ran since reset */
 } atrex_stats_t;
 
 typedef struct atrex_agg atrex_agg_t;
@@ -174,6 +177,11 @@ int atrex_agg_topk(atrex_agg_t*, uint32_t phase, uint32_t k, atrex_entry_t* h_ou
 
 /* Counters and per-phase totals (HOST output).  Synchronises `stream`. */
 int atrex_agg_stats(atrex_agg_t*, atrex_stats_t* h_out, void* stream);
+
+/* Diagnostic: copy the keys currently in the shared-memory hot directory (built from a sample of
+ * the first large ingest after create/reset) to `h_keys` (HOST, capacity `cap` keys, any order).
+ * *n_out = number of keys in the directory, which may exceed `cap`.  Synchronises `stream`. */
+int atrex_agg_hot_directory(atrex_agg_t*, uint64_t* h_keys, uint32_t cap, uint32_t* n_out, void* stream);
 
 /* Forget all records (the work table and weights are kept).  Asynchronous on `stream`. */
 int atrex_agg_reset(atrex_agg_t*, void* stream);

@@ -40,7 +40,7 @@ EXPORTED_SYMBOLS = [
     "atrex_agg_workspace_bytes", "atrex_agg_create", "atrex_agg_set_work_table", "atrex_agg_ingest",
     "atrex_agg_ingest_host", "atrex_agg_merge", "atrex_agg_finalize", "atrex_agg_topk", "atrex_agg_stats",
     "atrex_agg_reset", "atrex_agg_destroy", "atrex_strerror", "atrex_agg_last_cuda_error",
-    "atrex_agg_launch_count", "atrex_topk_entries_static",
+    "atrex_agg_launch_count", "atrex_topk_entries_static", "atrex_agg_hot_directory",
 ]
 
 
@@ -59,7 +59,8 @@ class atrex_stats_t(C.Structure):
                 ("n_keys", C.c_uint64), ("total_lo", C.c_uint64 * ATREX_MAX_PHASES),
                 ("total_hi", C.c_uint64 * ATREX_MAX_PHASES), ("keys_per_phase", C.c_uint64 * ATREX_MAX_PHASES),
                 ("table_slots", C.c_uint64), ("hot_slots", C.c_uint64), ("n_spilled", C.c_uint64),
-                ("n_overflow", C.c_uint64)]
+                ("n_overflow", C.c_uint64), ("max_spill_fill", C.c_uint64), ("spill_cap", C.c_uint64),
+                ("n_drains", C.c_uint64)]
 
 
 def _load():
@@ -79,6 +80,7 @@ def _load():
     L.atrex_agg_topk.argtypes = [vp, u32, u32, vp, C.POINTER(u32), vp]
     L.atrex_agg_stats.argtypes = [vp, C.POINTER(atrex_stats_t), vp]
     L.atrex_agg_reset.argtypes = [vp, vp]
+    L.atrex_agg_hot_directory.argtypes = [vp, vp, u32, C.POINTER(u32), vp]
     L.atrex_agg_destroy.argtypes = [vp]
     L.atrex_agg_destroy.restype = None
     L.atrex_strerror.restype = C.c_char_p
@@ -103,6 +105,7 @@ atrex_agg_finalize = lib.atrex_agg_finalize
 atrex_agg_topk = lib.atrex_agg_topk
 atrex_agg_stats = lib.atrex_agg_stats
 atrex_agg_reset = lib.atrex_agg_reset
+atrex_agg_hot_directory = lib.atrex_agg_hot_directory
 atrex_agg_destroy = lib.atrex_agg_destroy
 atrex_strerror = lib.atrex_strerror
 atrex_agg_last_cuda_error = lib.atrex_agg_last_cuda_error
@@ -263,7 +266,16 @@ class Aggregator:
                 "n_keys": st.n_keys,
                 "totals": [int(st.total_lo[p]) | (int(st.total_hi[p]) << 64) for p in range(ATREX_MAX_PHASES)],
                 "keys_per_phase": [int(x) for x in st.keys_per_phase], "table_slots": st.table_slots,
-                "hot_slots": st.hot_slots, "n_spilled": st.n_spilled, "n_overflow": st.n_overflow}
+                "hot_slots": st.hot_slots, "n_spilled": st.n_spilled, "n_overflow": st.n_overflow,
+                "max_spill_fill": st.max_spill_fill, "spill_cap": st.spill_cap, "n_drains": st.n_drains}
+
+    def hot_directory(self, stream=None) -> np.ndarray:
+        """Keys currently in the shared-memory hot directory (diagnostic)."""
+        out = np.zeros(16384, dtype=np.uint64)
+        n = C.c_uint32(0)
+        self._check(atrex_agg_hot_directory(self._h, out.ctypes.data, out.shape[0], C.byref(n), self._stream(stream)),
+                    "atrex_agg_hot_directory")
+        return out[: min(n.value, out.shape[0])].copy()
 
     def reset(self, stream=None):
         self._check(atrex_agg_reset(self._h, self._stream(stream)), "atrex_agg_reset")

@@ -19,8 +19,9 @@ constexpr ull MAX_KEYS = 1ull << 25;
 constexpr ull MAX_RECORDS_TOTAL = 1ull << 40;
 constexpr uint32_t HOT_MIN_RECORDS = 32768;             // smaller calls run without a directory
 constexpr uint32_t HOT_SAMPLE = 1u << 20;
-constexpr uint32_t CAND_BITS = 16;                     // candidate table of the directory build
-constexpr size_t HOT_SCRATCH_BYTES = (65536 * 4) + ((size_t)12 << CAND_BITS);
+constexpr uint32_t CAND_BITS = 17;                     // candidate table of the directory build
+constexpr size_t SKETCH_BYTES = (size_t)4 << 20;        // 2^20 counters (ingest.cu SKETCH_BITS)
+constexpr size_t HOT_SCRATCH_BYTES = SKETCH_BYTES + ((size_t)12 << CAND_BITS);
 constexpr uint32_t APPW_SMEM_MAX = 4096;
 constexpr uint32_t MAX_PROBE = 4096;                   // work-table probe bound
 constexpr uint32_t SEL_CAP = ATREX_MAX_TOPK + TOPK_CAND_CAP;
@@ -80,7 +81,7 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     size_t appw_smem = L->appw_in_smem ? (size_t)c->n_apps * 4 : 0;
     size_t fixed = appw_smem + 2048 + ((size_t)4 << L->lp);
     size_t budget = smem_optin > fixed ? smem_optin - fixed : 0;
-    L->hot_slots = (uint32_t)(budget / 20) & ~1u;
+    L->hot_slots = (uint32_t)(budget / 20) & ~3u;   // whole 4-slot buckets
     if (c->flags & ATREX_FLAG_NO_HOT_DIRECTORY) L->hot_slots = 0;
     size_t o = 0;
     L->off_ctl = o;            o += round_up(sizeof(Control), ALIGN);
@@ -133,6 +134,8 @@ struct atrex_agg {
     Control* h_ctl = nullptr;  // pinned mirror
     bool hot_ready = false;
     bool finalized = false;
+    bool spill_pending = false;   // entries may sit in the spill buffers
+    ull scatter_seq = 0;          // sequence number of the last scatter launch
     atrex_hw_peaks_t peaks;
     ull n_records = 0;
     cudaStream_t copy_stream = nullptr;
@@ -256,6 +259,7 @@ int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out) {
         if (e == cudaSuccess) e = cudaMemset(h->ws + L.off_ctl, 0, L.off_appw - L.off_ctl);  // control, table, work
         if (e == cudaSuccess) e = cudaMemcpy(h->d_appw, cfg->app_weights, (size_t)cfg->n_apps * 4, cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = cudaMemset(h->hot_keys, 0, (size_t)(L.hot_slots ? L.hot_slots : 2) * 8);
+        if (e == cudaSuccess) e = cudaMemset(h->spill_cnt, 0, ((size_t)L.n_groups << L.lp) * 4);
         if (e == cudaSuccess) e = cudaHostAlloc((void**)&h->h_ctl, sizeof(Control), cudaHostAllocDefault);
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
         for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
@@ -295,6 +299,8 @@ int atrex_agg_reset(atrex_agg_t* h, void* stream) {
     cudaStream_t s = (cudaStream_t)stream;
     CU(h, cudaMemsetAsync(h->ctl, 0, sizeof(Control), s));
     CU(h, cudaMemsetAsync(h->keys, 0, h->L.off_work - h->L.off_keys, s));  // keys and vals
+    CU(h, cudaMemsetAsync(h->spill_cnt, 0, ((size_t)h->L.n_groups << h->L.lp) * 4, s));  // discard undrained entries
+    h->spill_pending = false;
     h->hot_ready = false;
     h->finalized = false;
     h->n_records = 0;
@@ -327,6 +333,26 @@ int atrex_agg_set_work_table(atrex_agg_t* h, const atrex_work_t* rows, uint64_t 
     return ATREX_OK;
 }
 
+// Partition pass over the spill buffers.  Unforced, the kernel exits at once unless the scatter
+// launch just before it saw a buffer more than 5/8 full; forced (before results are read), it
+// drains whatever is there.
+static int drain_spill(atrex_agg* h, bool force, cudaStream_t s) {
+    if (force && !h->spill_pending) return ATREX_OK;
+    PartitionParams q;
+    q.t = h->table_ref();
+    q.spill = h->spill;
+    q.spill_cnt = h->spill_cnt;
+    q.n_groups = h->L.n_groups;
+    q.n_used = h->L.n_groups;
+    q.cap = h->L.cap;
+    q.force = force ? 1u : 0u;
+    q.seq = h->scatter_seq;
+    CU(h, launch_partition(q, h->n_sms, s));
+    h->launches++;
+    if (force) h->spill_pending = false;
+    return ATREX_OK;
+}
+
 static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, cudaStream_t s) {
     // hot directory from a sample of the first sufficiently large call after create/reset
     if (h->L.hot_slots && !h->hot_ready && n >= HOT_MIN_RECORDS) {
@@ -340,8 +366,8 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
         b.hot_slots = h->L.hot_slots;
         b.ctl = h->ctl;
         b.sketch = (uint32_t*)h->hot_scratch;
-        b.cand_keys = (ull*)(h->hot_scratch + 65536 * 4);
-        b.cand_cnt = (uint32_t*)(h->hot_scratch + 65536 * 4 + ((size_t)8 << CAND_BITS));
+        b.cand_keys = (ull*)(h->hot_scratch + SKETCH_BYTES);
+        b.cand_cnt = (uint32_t*)(h->hot_scratch + SKETCH_BYTES + ((size_t)8 << CAND_BITS));
         b.cand_bits = CAND_BITS;
         CU(h, cudaMemsetAsync(h->hot_scratch, 0, HOT_SCRATCH_BYTES, s));
         CU(h, launch_hot_build(b, h->n_sms, s));
@@ -364,7 +390,7 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
     p.app_w = h->d_appw;
     p.hot_keys = h->hot_keys;
     p.hot_slots = h->L.hot_slots;
-    p.hot_buckets = h->L.hot_slots / 2;
+    p.hot_buckets = h->L.hot_slots / 4;
     p.t = h->table_ref();
     p.spill = h->spill;
     p.spill_cnt = h->spill_cnt;
@@ -373,17 +399,12 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
     const ull pairs_per_cta_iter = 2048;
     ull want = (p.n_pairs + pairs_per_cta_iter - 1) / pairs_per_cta_iter;
     int grid = (int)(want < 1 ? 1 : (want > (ull)h->n_sms ? (ull)h->n_sms : want));
+    p.drain_above = h->L.cap / 8 * 5;
+    p.seq = ++h->scatter_seq;
     CU(h, launch_scatter(p, h->hot_ready, grid, s));
-    PartitionParams q;
-    q.t = p.t;
-    q.spill = h->spill;
-    q.spill_cnt = h->spill_cnt;
-    q.n_groups = h->L.n_groups;
-    q.n_used = (uint32_t)grid;
-    q.cap = h->L.cap;
-    CU(h, launch_partition(q, h->n_sms, s));
-    h->launches += 2;
-    return ATREX_OK;
+    h->spill_pending = true;
+    h->launches++;
+    return drain_spill(h, /*force=*/false, s);
 }
 
 int atrex_agg_ingest(atrex_agg_t* h, const atrex_record_t* d_records, uint64_t n, void* stream) {
@@ -469,7 +490,9 @@ int atrex_agg_finalize(atrex_agg_t* h, const atrex_hw_peaks_t* peaks, atrex_entr
     DeviceGuard guard(h->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
     h->peaks = *peaks;
-    int rc = run_totals(h, s);
+    int rc = drain_spill(h, /*force=*/true, s);
+    if (rc != ATREX_OK) return rc;
+    rc = run_totals(h, s);
     if (rc != ATREX_OK) return rc;
     CU(h, cudaMemsetAsync(&h->ctl->n_out, 0, sizeof(ull), s));
     CU(h, launch_emit(finalize_params(h, d_out, out_cap), h->scan_grid(h->L.n_slots, 256 * 4), s));
@@ -508,7 +531,14 @@ int atrex_agg_topk(atrex_agg_t* h, uint32_t phase, uint32_t k, atrex_entry_t* h_
         p.collect_all = 1;
         total = n_phase;
     } else {
-        // most-significant-digit radix select on the ranking composite
+        // most-significant-digit radix select on the ranking composite; digits start at the
+        // highest bit the phase total has (no key's weighted time exceeds it)
+        {
+            ull hi = h->h_ctl->total_hi[phase], lo = h->h_ctl->total_lo[phase];
+            int top_bit = hi ? 64 + (63 - __builtin_clzll(hi)) : (lo ? 63 - __builtin_clzll(lo) : 0);
+            p.shift = (uint32_t)(143 - (top_bit + 56));
+        }
+        const uint32_t n_digits = (144 - p.shift + 11) / 12;
         ull need = k, cand = 0;
         uint32_t* hist = h->h_ctl->hist;
         while (true) {
@@ -526,7 +556,7 @@ int atrex_agg_topk(atrex_agg_t* h, uint32_t phase, uint32_t k, atrex_entry_t* h_
             need -= above;
             cand = hist[bin];
             p.prefix_digit[p.n_prefix_digits++] = (uint16_t)bin;
-            if (cand <= TOPK_CAND_CAP || p.n_prefix_digits == (uint32_t)TOPK_DIGITS) break;
+            if (cand <= TOPK_CAND_CAP || p.n_prefix_digits == n_digits) break;
         }
         total = (k - need) + cand;
     }
@@ -549,7 +579,9 @@ int atrex_agg_stats(atrex_agg_t* h, atrex_stats_t* out, void* stream) {
     if (!h || !out) return ATREX_ERR_INVALID;
     DeviceGuard guard(h->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
-    int rc = run_totals(h, s);
+    int rc = drain_spill(h, /*force=*/true, s);
+    if (rc != ATREX_OK) return rc;
+    rc = run_totals(h, s);
     if (rc != ATREX_OK) return rc;
     CU(h, cudaMemcpyAsync(h->h_ctl, h->ctl, offsetof(Control, hist), cudaMemcpyDeviceToHost, s));
     CU(h, cudaStreamSynchronize(s));
@@ -568,7 +600,36 @@ int atrex_agg_stats(atrex_agg_t* h, atrex_stats_t* out, void* stream) {
     out->hot_slots = c->hot_n;
     out->n_spilled = c->n_spilled;
     out->n_overflow = c->n_overflow;
+    out->max_spill_fill = c->max_fill;
+    out->spill_cap = h->L.cap;
+    out->n_drains = c->n_drains;
     return device_status_to_error(c);
+}
+
+int atrex_agg_hot_directory(atrex_agg_t* h, uint64_t* h_keys, uint32_t cap, uint32_t* n_out, void* stream) {
+    if (!h || !n_out || (cap && !h_keys)) return ATREX_ERR_INVALID;
+    *n_out = 0;
+    if (!h->hot_ready || h->L.hot_slots == 0) return ATREX_OK;
+    DeviceGuard guard(h->cfg.device);
+    cudaStream_t s = (cudaStream_t)stream;
+    ull* image = (ull*)malloc((size_t)h->L.hot_slots * 8);
+    if (!image) return ATREX_ERR_NOMEM;
+    cudaError_t e = cudaMemcpyAsync(image, h->hot_keys, (size_t)h->L.hot_slots * 8, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        free(image);
+        h->last_cuda_error = (int)e;
+        return ATREX_ERR_CUDA;
+    }
+    uint32_t n = 0;
+    for (uint32_t i = 0; i < h->L.hot_slots; ++i) {
+        if (image[i] == 0) continue;
+        if (n < cap) h_keys[n] = ~image[i];
+        ++n;
+    }
+    free(image);
+    *n_out = n;
+    return ATREX_OK;
 }
 
 const char* atrex_strerror(int status) {

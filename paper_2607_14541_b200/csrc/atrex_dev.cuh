@@ -60,7 +60,11 @@ struct Control {
     ull hot_skew;              // 1 if one key dominates the sample: combine equal lanes per warp
     ull n_spilled;             // records routed through the spill buffers
     ull n_overflow;            // records that found their spill buffer full (slow exact path)
-    ull pad1[6];
+    ull drain_seq;             // sequence number of the last scatter launch that asked for a drain
+    ull max_fill;              // fullest spill buffer seen since reset (entries)
+    ull n_drains;              // partition passes that actually ran
+    ull dir_mult;              // multiplier of the hot directory's bucket hash chosen at build time
+    ull pad1[2];
     ull total_lo[ATREX_MAX_PHASES];
     ull total_hi[ATREX_MAX_PHASES];
     ull keys_per_phase[ATREX_MAX_PHASES];

@@ -125,26 +125,44 @@ __device__ __forceinline__ void load_phase_totals(const Control* ctl, double* dT
     __syncthreads();
 }
 
+// Four slots per thread per round: their table loads and work-table probes are independent, so
+// the dependent-load latency of the probes overlaps.
+constexpr int EMIT_ILP = 4;
+
 __global__ void __launch_bounds__(FIN_THREADS) emit_kernel(FinalizeParams p) {
     __shared__ double dT[ATREX_MAX_PHASES];
     __shared__ bool zeroT[ATREX_MAX_PHASES];
     load_phase_totals(p.ctl, dT, zeroT);
     const unsigned lane = threadIdx.x & 31u;
     const ull stride = (ull)gridDim.x * blockDim.x;
-    const ull rounds = (p.n_slots + stride - 1) / stride;  // uniform trip count keeps warps converged
+    const ull rounds = (p.n_slots + stride * EMIT_ILP - 1) / (stride * EMIT_ILP);  // uniform: warps stay converged
     for (ull r = 0; r < rounds; ++r) {
-        ull i = r * stride + (ull)blockIdx.x * blockDim.x + threadIdx.x;
-        SlotView v;
-        v.live = false;
-        if (i < p.n_slots) v = load_slot(p.t, i);
-        unsigned live = __ballot_sync(0xFFFFFFFFu, v.live);
-        if (live == 0) continue;
+        SlotView v[EMIT_ILP];
+        unsigned live[EMIT_ILP];
+        int total = 0;
+#pragma unroll
+        for (int u = 0; u < EMIT_ILP; ++u) {
+            ull i = (r * EMIT_ILP + u) * stride + (ull)blockIdx.x * blockDim.x + threadIdx.x;
+            v[u].live = false;
+            if (i < p.n_slots) v[u] = load_slot(p.t, i);
+            live[u] = __ballot_sync(0xFFFFFFFFu, v[u].live);
+            total += __popc(live[u]);
+        }
+        if (total == 0) continue;
         ull base = 0;
-        if (lane == (unsigned)(__ffs(live) - 1)) base = atomicAdd(&p.ctl->n_out, (ull)__popc(live));
-        base = __shfl_sync(0xFFFFFFFFu, base, __ffs(live) - 1);
-        if (v.live) {
-            ull pos = base + __popc(live & ((1u << lane) - 1u));
-            if (pos < p.out_cap) store_entry(p.out + pos, make_entry(v, dT, zeroT, p));
+        if (lane == 0) base = atomicAdd(&p.ctl->n_out, (ull)total);
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        atrex_entry_t e[EMIT_ILP];
+#pragma unroll
+        for (int u = 0; u < EMIT_ILP; ++u)
+            if (v[u].live) e[u] = make_entry(v[u], dT, zeroT, p);
+#pragma unroll
+        for (int u = 0; u < EMIT_ILP; ++u) {
+            if (v[u].live) {
+                ull pos = base + __popc(live[u] & ((1u << lane) - 1u));
+                if (pos < p.out_cap) store_entry(p.out + pos, e[u]);
+            }
+            base += __popc(live[u]);
         }
     }
 }
@@ -197,8 +215,12 @@ __device__ __forceinline__ Composite composite_of(const SlotView& v) {
     return x;
 }
 
-__device__ __forceinline__ uint32_t digit_of(const Composite& x, int d) {
-    int off = 144 - 12 * (d + 1);
+// Digit d (most significant first) of the composite shifted left by `shift` bits.  The shift
+// drops the leading zero bits that every key of the phase shares (no weighted time exceeds the
+// phase total), so that the first digit already separates the top of the ranking.
+__device__ __forceinline__ uint32_t digit_of(const Composite& x, int d, int shift) {
+    int off = 144 - 12 * (d + 1) - shift;
+    if (off < 0) return (uint32_t)(x.c[0] << (-off)) & 0xFFFu;  // last, partial digit
     int wi = off >> 6, sh = off & 63;
     ull v = x.c[wi] >> sh;
     if (sh > 52 && wi < 2) v |= x.c[wi + 1] << (64 - sh);
@@ -208,7 +230,7 @@ __device__ __forceinline__ uint32_t digit_of(const Composite& x, int d) {
 // -1: below the prefix, 0: equal on all fixed digits, +1: above
 __device__ __forceinline__ int compare_prefix(const Composite& x, const TopkParams& p) {
     for (uint32_t d = 0; d < p.n_prefix_digits; ++d) {
-        uint32_t a = digit_of(x, (int)d), b = p.prefix_digit[d];
+        uint32_t a = digit_of(x, (int)d, (int)p.shift), b = p.prefix_digit[d];
         if (a != b) return a > b ? 1 : -1;
     }
     return 0;
@@ -223,7 +245,7 @@ __global__ void __launch_bounds__(FIN_THREADS) topk_hist_kernel(TopkParams p) {
         if (!v.live || (uint32_t)(v.key >> 48) != p.phase) continue;
         Composite x = composite_of(v);
         if (compare_prefix(x, p) != 0) continue;
-        atomicAdd(&h[digit_of(x, (int)p.n_prefix_digits)], 1u);
+        atomicAdd(&h[digit_of(x, (int)p.n_prefix_digits, (int)p.shift)], 1u);
     }
     __syncthreads();
     for (int i = threadIdx.x; i < TOPK_BINS; i += blockDim.x)

@@ -34,11 +34,16 @@ namespace atrex {
 
 constexpr int INGEST_THREADS = 1024;
 constexpr uint32_t NO_SLOT = 0xFFFFFFFFu;
+constexpr uint32_t DIR_WAYS = 4;                   // slots per hot-directory bucket (32 bytes of keys)
 constexpr uint32_t NEW_KEY_FLAG = 0x80000000u;     // partition pass: slot claimed in this launch
 
-__device__ __forceinline__ uint32_t dir_bucket(uint32_t h, uint32_t n_buckets) {
-    return __umulhi(h * 0xC2B2AE35u, n_buckets);
+// Bucket of the hot directory.  The odd multiplier is picked per build among DIR_MULTS so that
+// as little sampled weight as possible is lost to buckets that more than two hot keys map to.
+__device__ __forceinline__ uint32_t dir_bucket(uint32_t h, uint32_t mult, uint32_t n_buckets) {
+    return __umulhi(h * mult, n_buckets);
 }
+__constant__ uint32_t DIR_MULTS[8] = {0xC2B2AE35u, 0x27D4EB2Fu, 0x165667B1u, 0x9E3779B9u,
+                                      0x85EBCA6Bu, 0xD3A2646Du, 0xFD7046C5u, 0xB55A4F09u};
 
 __device__ __forceinline__ void ld_stream_256(const void* p, uint32_t (&w)[8]) {
     asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
@@ -52,6 +57,7 @@ struct SmemDir {
     uint32_t* a1;     // [slots] ... and bits 32..63 (carries of a0 are added here by the adder)
     uint32_t* cnt;    // [slots] this launch's record count of the slot
     uint32_t* cursor; // [P] entries appended to this CTA's buffer of each partition
+    uint32_t mult;    // bucket-hash multiplier of this directory image
     const uint32_t* appw_s;  // card-hour weights in shared memory (when they fit) ...
     const uint32_t* appw_g;  // ... else in global memory
     bool appw_shared;
@@ -118,10 +124,12 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
         uint32_t slot[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            uint32_t b = dir_bucket(h[r], p.hot_buckets) * 2;
-            ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(d.keys + b);
-            ull skey = ~(((ull)khi[r] << 32) | w[r][2]);
-            slot[r] = !todo[r] ? NO_SLOT : (kk.x == skey ? b : (kk.y == skey ? b + 1 : NO_SLOT));
+            uint32_t b = dir_bucket(h[r], d.mult, p.hot_buckets) * DIR_WAYS;
+            const ulonglong2 k01 = *reinterpret_cast<const ulonglong2*>(d.keys + b);
+            const ulonglong2 k23 = *reinterpret_cast<const ulonglong2*>(d.keys + b + 2);
+            const ull skey = ~(((ull)khi[r] << 32) | w[r][2]);
+            uint32_t way = k01.x == skey ? 0u : (k01.y == skey ? 1u : (k23.x == skey ? 2u : (k23.y == skey ? 3u : DIR_WAYS)));
+            slot[r] = (!todo[r] || way == DIR_WAYS) ? NO_SLOT : b + way;
         }
         if (DEDUPE) {
             // one key dominates the trace: combine the lanes that share the first hitting lane's slot
@@ -260,10 +268,12 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
     d.cnt = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
+    d.mult = HOT ? (uint32_t)p.t.ctl->dir_mult : 1u;
     const uint32_t n_parts = 1u << p.t.lp;
     d.cursor = reinterpret_cast<uint32_t*>(sp);
     sp += (size_t)n_parts * 4;
-    for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) d.cursor[i] = 0;
+    // the buffers persist across launches until the partition pass drains them: resume the cursors
+    for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) d.cursor[i] = p.spill_cnt[((ull)blockIdx.x << p.t.lp) + i];
     if (p.appw_in_smem) {
         uint32_t* s_appw = reinterpret_cast<uint32_t*>(sp);
         for (uint32_t i = threadIdx.x; i < p.n_apps; i += blockDim.x) s_appw[i] = p.app_w[i];
@@ -294,18 +304,27 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     if ((threadIdx.x & 31u) == 0 && rsum != 0) atomicAdd(&p.t.ctl->n_rejected, (ull)rsum);
 
     __syncthreads();
-    uint32_t spilled = 0, overflow = 0;
+    uint32_t spilled = 0, overflow = 0, fullest = 0;
+    bool crowded = false;
     for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) {
-        uint32_t c = d.cursor[i];
-        p.spill_cnt[((ull)blockIdx.x << p.t.lp) + i] = min(c, p.cap);
-        spilled += min(c, p.cap);
+        const ull at = ((ull)blockIdx.x << p.t.lp) + i;
+        uint32_t before = p.spill_cnt[at], c = d.cursor[i];
+        p.spill_cnt[at] = min(c, p.cap);
+        spilled += min(c, p.cap) - before;
         overflow += c > p.cap ? c - p.cap : 0u;
+        crowded |= c > p.drain_above;
+        fullest = max(fullest, c);
     }
+    fullest = __reduce_max_sync(0xFFFFFFFFu, fullest);
     spilled = __reduce_add_sync(0xFFFFFFFFu, spilled);
     overflow = __reduce_add_sync(0xFFFFFFFFu, overflow);
+    crowded = __any_sync(0xFFFFFFFFu, crowded);
     if ((threadIdx.x & 31u) == 0) {
         if (spilled) atomicAdd(&p.t.ctl->n_spilled, (ull)spilled);
         if (overflow) atomicAdd(&p.t.ctl->n_overflow, (ull)overflow);
+        // a buffer is filling up: have the partition pass that follows this launch drain them
+        if (crowded) atomicMax(&p.t.ctl->drain_seq, p.seq);
+        atomicMax(&p.t.ctl->max_fill, (ull)fullest);
     }
     if (HOT) {
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
@@ -334,6 +353,10 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     __shared__ uint32_t s_total;
     const uint32_t n_parts = 1u << q.t.lp;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
+    // the spill buffers are drained lazily: unless forced, only when the scatter launch just
+    // before this one found a buffer filling up
+    if (!q.force && ld_relaxed(&q.t.ctl->drain_seq) != q.seq) return;
+    if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(&q.t.ctl->n_drains, 1ull);
 
     for (uint32_t part = blockIdx.x; part < n_parts; part += gridDim.x) {
         if (threadIdx.x == 0) s_total = 0;
@@ -457,18 +480,20 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
             *reinterpret_cast<ulonglong2*>(vp) = make_ulonglong2(nlo, cnthi);
             if (c & NEW_KEY_FLAG) q.t.keys[base + i] = s_keys[i];
         }
+        // this partition's buffers are empty again
+        for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) q.spill_cnt[((ull)g << q.t.lp) + part] = 0;
     }
 }
 
 // --------------------------------------------------------------------------------------
 // Hot-directory construction, three small kernels over a strided sample of the records:
-//   1. count   every sampled key bumps one of 65536 counters chosen by its hash;
+//   1. count   every sampled key bumps one of 2^20 counters chosen by its hash;
 //   2. admit   sampled keys whose counter reached ADMIT_MIN are inserted, with exact counts,
 //              into a candidate table (colliding cold keys may slip in; harmless);
 //   3. select  one CTA picks the count threshold that fills the directory and installs the
-//              candidates, most frequent classes first, into 2-slot buckets.
+//              candidates, most frequent classes first, into 4-slot buckets.
 // Which keys end up in the directory only affects speed, never results.
-constexpr uint32_t SKETCH_BITS = 16;
+constexpr uint32_t SKETCH_BITS = 20;   // as many counters as samples, so that cold keys stay below ADMIT_MIN
 constexpr uint32_t ADMIT_MIN = 3;
 constexpr uint32_t CAND_PROBES = 16;
 
@@ -528,14 +553,18 @@ __global__ void __launch_bounds__(256) hot_admit_kernel(HotBuildParams p) {
     }
 }
 
+constexpr uint32_t SELECT_MAX = 14336;  // candidates kept for installation (directory <= 11.6K slots, x1.25)
+
 __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    ull* c_key = reinterpret_cast<ull*>(smem_raw);                        // [SELECT_MAX]
+    uint32_t* c_cnt = reinterpret_cast<uint32_t*>(c_key + SELECT_MAX);    // [SELECT_MAX]
     __shared__ uint32_t hist[1024];
-    __shared__ uint32_t s_thr, s_inserted, s_max;
+    __shared__ uint32_t s_thr, s_inserted, s_max, s_n;
     const uint32_t n_cand = 1u << p.cand_bits;
     hist[threadIdx.x] = 0;
-    if (threadIdx.x == 0) s_max = 0;
     for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) p.hot_keys[i] = 0;
-    if (threadIdx.x == 0) s_inserted = 0;
+    if (threadIdx.x == 0) s_inserted = s_max = s_n = 0;
     __syncthreads();
     for (uint32_t i = threadIdx.x; i < n_cand; i += blockDim.x) {
         uint32_t c = p.cand_cnt[i];
@@ -545,7 +574,7 @@ __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
     __syncthreads();
     if (threadIdx.x == 0) {
         // smallest threshold >= 2 whose class fits the directory with some over-subscription
-        uint32_t budget = p.hot_slots + p.hot_slots / 4, cum = 0, thr = 1024;
+        uint32_t budget = min(p.hot_slots + p.hot_slots / 4, SELECT_MAX), cum = 0, thr = 1024;
         for (int c = 1023; c >= 2; --c) {
             if (cum + hist[c] > budget) break;
             cum += hist[c];
@@ -558,17 +587,64 @@ __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
     }
     __syncthreads();
     const uint32_t thr = s_thr;
-    const uint32_t bounds[6] = {0xFFFFFFFFu, 512u, 128u, 32u, 8u, 2u};
-    for (int round = 0; round < 5; ++round) {
-        uint32_t hi = bounds[round], lo = max(bounds[round + 1], thr);
+    // compact the selected candidates into shared memory, then install them class by class
+    for (uint32_t i = threadIdx.x; i < n_cand; i += blockDim.x) {
+        uint32_t c = p.cand_cnt[i];
+        if (c >= thr) {
+            uint32_t at = atomicAdd(&s_n, 1u);
+            if (at < SELECT_MAX) {
+                c_key[at] = p.cand_keys[i];
+                c_cnt[at] = c;
+            }
+        }
+    }
+    __syncthreads();
+    const uint32_t n_sel = min(s_n, SELECT_MAX);
+    // pick the bucket-hash multiplier that loses the least sampled weight: a key is lost when
+    // its bucket's slots are already taken (approximated per class by
+    // arrival order, which is what the installation below does as well)
+    __shared__ uint32_t s_lost[8];
+    uint32_t* occupancy = hist;  // reuse: 1024 counters cover buckets modulo 1024 exactly when
+                                 // folded per pass below
+    if (threadIdx.x < 8) s_lost[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t n_buckets = p.hot_slots / DIR_WAYS;
+    for (uint32_t m = 0; m < 8; ++m) {
+        // buckets are examined in slices of 1024 so that the occupancy counters fit `hist`
+        for (uint32_t lo_b = 0; lo_b < n_buckets; lo_b += 1024) {
+            occupancy[threadIdx.x] = 0;
+            __syncthreads();
+            for (uint32_t i = threadIdx.x; i < n_sel; i += blockDim.x) {
+                uint32_t c = c_cnt[i];
+                if (c < 16) continue;  // only keys that matter
+                uint32_t b = dir_bucket(hash32(~c_key[i]), DIR_MULTS[m], n_buckets);
+                if (b >= lo_b && b < lo_b + 1024 && atomicAdd(&occupancy[b - lo_b], 1u) >= DIR_WAYS) atomicAdd(&s_lost[m], c);
+            }
+            __syncthreads();
+        }
+    }
+    if (threadIdx.x == 0) {
+        uint32_t best = 0;
+        for (uint32_t m = 1; m < 8; ++m)
+            if (s_lost[m] < s_lost[best]) best = m;
+        p.ctl->dir_mult = DIR_MULTS[best];
+        s_thr = DIR_MULTS[best];  // broadcast (the threshold is already in registers)
+    }
+    __syncthreads();
+    const uint32_t mult = s_thr;
+    // install from the most to the least frequent class (counts within a class differ < 2x), so
+    // that a key can only lose its bucket to keys about as frequent as itself
+    for (int round = 0; round < 11; ++round) {
+        uint32_t hi = round == 0 ? 0xFFFFFFFFu : (2048u >> round), lo = max(1024u >> round, thr);
         if (lo < hi) {
-            for (uint32_t i = threadIdx.x; i < n_cand; i += blockDim.x) {
-                uint32_t c = p.cand_cnt[i];
+            for (uint32_t i = threadIdx.x; i < n_sel; i += blockDim.x) {
+                uint32_t c = c_cnt[i];
                 if (c >= lo && c < hi) {
-                    ull skey = p.cand_keys[i];
-                    uint32_t b = dir_bucket(hash32(~skey), p.hot_slots / 2) * 2;
-                    if (atomicCAS(&p.hot_keys[b], 0ull, skey) == 0 || atomicCAS(&p.hot_keys[b + 1], 0ull, skey) == 0)
-                        atomicAdd(&s_inserted, 1u);
+                    ull skey = c_key[i];
+                    uint32_t b = dir_bucket(hash32(~skey), mult, n_buckets) * DIR_WAYS;
+                    bool placed = false;
+                    for (uint32_t way = 0; way < DIR_WAYS && !placed; ++way) placed = atomicCAS(&p.hot_keys[b + way], 0ull, skey) == 0;
+                    if (placed) atomicAdd(&s_inserted, 1u);
                 }
             }
         }
@@ -596,7 +672,7 @@ cudaError_t ingest_prepare() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(partition_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
     if (e != cudaSuccess) return e;
-    return cudaSuccess;
+    return cudaFuncSetAttribute(hot_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_MAX * 12);
 }
 
 cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream) {
@@ -620,7 +696,7 @@ cudaError_t launch_hot_build(const HotBuildParams& p, int n_sms, cudaStream_t st
     if (grid > n_sms * 8) grid = n_sms * 8;
     hot_count_kernel<<<grid, 256, 0, stream>>>(p);
     hot_admit_kernel<<<grid, 256, 0, stream>>>(p);
-    hot_select_kernel<<<1, 1024, 0, stream>>>(p);
+    hot_select_kernel<<<1, 1024, SELECT_MAX * 12, stream>>>(p);
     return cudaGetLastError();
 }
 

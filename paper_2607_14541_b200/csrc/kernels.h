@@ -13,23 +13,27 @@ struct IngestParams {
     uint32_t appw_in_smem;
     const uint32_t* app_w;     // device copy of the card-hour weights
     const ull* hot_keys;       // directory image, hot_slots entries of ~key (0 = empty)
-    uint32_t hot_slots;        // even
-    uint32_t hot_buckets;      // hot_slots / 2
+    uint32_t hot_slots;        // multiple of 4
+    uint32_t hot_buckets;      // hot_slots / 4
     TableRef t;
     // spill buffers: entry i of scatter CTA g for partition p at spill + ((g * P + p) * cap + i) * 16 bytes
     unsigned char* spill;
     uint32_t* spill_cnt;       // [n_groups][P]
     uint32_t n_groups;         // G, row pitch of the buffers (= CTAs of the widest scatter launch)
     uint32_t cap;              // entries per (partition, CTA) buffer
+    uint32_t drain_above;      // ask for a drain when a buffer holds more entries than this
+    ull seq;                   // sequence number of this launch
 };
 
 struct PartitionParams {
     TableRef t;
     const unsigned char* spill;
-    const uint32_t* spill_cnt;
+    uint32_t* spill_cnt;
     uint32_t n_groups;         // row pitch G
-    uint32_t n_used;           // CTAs of the scatter launch that fed this pass (<= G)
+    uint32_t n_used;           // scatter CTAs whose buffers are read (<= G)
     uint32_t cap;
+    uint32_t force;            // 1: drain unconditionally; 0: only if the scatter launch `seq` asked for it
+    ull seq;
 };
 
 struct HotBuildParams {
@@ -39,7 +43,7 @@ struct HotBuildParams {
     uint32_t n_apps, n_phases;
     ull* hot_keys;
     uint32_t hot_slots;
-    uint32_t* sketch;          // [65536] sample counters by hash
+    uint32_t* sketch;          // [2^20] sample counters by hash
     ull* cand_keys;            // [1 << cand_bits] candidate table: ~key, 0 = empty
     uint32_t* cand_cnt;        // [1 << cand_bits] exact sample counts of the candidates
     uint32_t cand_bits;
@@ -70,6 +74,7 @@ struct TopkParams {
     uint32_t phase;
     uint32_t n_prefix_digits;   // leading 12-bit digits of the ranking composite already fixed
     uint16_t prefix_digit[12];  // their values, most significant first
+    uint32_t shift;             // leading zero bits of the composite dropped before digit extraction
     int collect_all;
     ull* sel;                   // [sel_cap][4]: composite words 2,1,0 and the slot index
     uint32_t sel_cap;

@@ -33,7 +33,7 @@ def test_struct_layouts_match_the_header():
     assert p.RECORD_DTYPE.itemsize == 16 and p.WORK_DTYPE.itemsize == 24 and p.ENTRY_DTYPE.itemsize == 48
     assert C.sizeof(p.atrex_hw_peaks_t) == 72
     assert C.sizeof(p.atrex_agg_config_t) == 56
-    assert C.sizeof(p.atrex_stats_t) == 8 * (4 + 3 * 8 + 4)
+    assert C.sizeof(p.atrex_stats_t) == 8 * (4 + 3 * 8 + 7)
     assert p.RECORD_DTYPE.fields["shape_id"][1] == 8 and p.RECORD_DTYPE.fields["phase"][1] == 6
     assert p.WORK_DTYPE.fields["flops"][1] == 8 and p.ENTRY_DTYPE.fields["phase_weight"][1] == 32
 
