@@ -45,6 +45,7 @@ struct Layout {
         off_spill_cnt, off_spill, off_hot_scratch, total;
     ull n_slots, work_slots;
     uint32_t lp, C;              // partitions = 1 << lp, slots per partition
+    uint32_t Cw;                 // work-table slots per partition
     uint32_t n_groups, cap;      // spill buffers: [P][n_groups][cap] entries
     ull sub_launch;              // records per scatter + partition launch pair
     uint32_t hot_slots;
@@ -73,10 +74,14 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     L->n_slots = (ull)L->C << L->lp;
     L->n_groups = (uint32_t)n_sms;
     L->sub_launch = c->max_keys >= (1ull << 21) ? (1ull << 27) : (c->max_keys >= (1ull << 16) ? (1ull << 25) : (1ull << 24));
-    ull per_buf = (L->sub_launch * 5 / 2) / (((ull)n_sms) << L->lp);
+    // room for 3.5 launches' worth of entries if every record spilled: three launches can then
+    // accumulate before a drain, with slack for uneven partitions
+    ull per_buf = (L->sub_launch * 7 / 2) / (((ull)n_sms) << L->lp);
     if (per_buf < 64) per_buf = 64;
     L->cap = (uint32_t)((per_buf + 7) / 8 * 8);
-    L->work_slots = c->max_work_rows ? pow2_at_least(c->max_work_rows * 2 < 1024 ? 1024 : c->max_work_rows * 2) : 0;
+    // work table: same partitions as the key table, 1.5 slots per row plus slack for uneven partitions
+    L->Cw = c->max_work_rows ? (uint32_t)((((c->max_work_rows * 3 / 2) >> L->lp) + 64 + 31) / 32 * 32) : 0;
+    L->work_slots = (ull)L->Cw << L->lp;
     L->appw_in_smem = c->n_apps <= APPW_SMEM_MAX;
     size_t appw_smem = L->appw_in_smem ? (size_t)c->n_apps * 4 : 0;
     size_t fixed = appw_smem + 2048 + ((size_t)4 << L->lp);
@@ -155,9 +160,8 @@ struct atrex_agg {
     WorkRef work_ref() const {
         WorkRef w;
         w.table = L.work_slots ? work : nullptr;
-        w.mask = L.work_slots ? L.work_slots - 1 : 0;
-        w.shift = L.work_slots ? 64 - log2_of(L.work_slots) : 0;
-        w.max_probe = (uint32_t)(L.work_slots < MAX_PROBE ? L.work_slots : MAX_PROBE);
+        w.lp = L.lp;
+        w.Cw = L.Cw;
         return w;
     }
     int scan_grid(ull n_items, int threads) const {

@@ -15,7 +15,8 @@
 //                 written by CTA g of the scatter pass (its buffers are contiguous, which keeps
 //                 the scattered 16-byte appends within a few pages), read by CTA p of the
 //                 partition pass
-//   work table  : open addressing keyed by op_id << 32 | shape_id, holding flops, bytes, dtype
+//   work table  : the same P partitions (by the same hash of op_id and shape_id) of Cw 32-byte
+//                 slots {~(op_id << 32 | shape_id), flops, bytes, dtype}, probed inside the partition
 //   control     : counters, per-phase totals, top-k histogram
 #pragma once
 #include <cstdint>
@@ -72,25 +73,19 @@ struct Control {
     uint32_t hist[TOPK_BINS];
 };
 
-// 32-bit mixer of a packed key for the key table, the spill partitions and the hot directory:
-// two multiplicative hashes of the key's words, folded and multiplied once more.  The top
-// bits pick the partition, the bits below them the start slot inside it.
-__device__ __forceinline__ uint32_t hash32(uint32_t key_hi, uint32_t key_lo) {
-    uint32_t h = (key_lo * 0x9E3779B1u) ^ (key_hi * 0x85EBCA77u);
+// 32-bit mixer of (op_id, shape_id) for the key table, the spill partitions, the hot directory
+// and the work table: two multiplicative hashes of the two words, folded and multiplied once
+// more.  The top bits pick the partition, the bits below them the start slot inside it.  The
+// phase is deliberately left out: a key's partition is then also the partition of its
+// (operator, shape) row in the work table, which keeps the roofline pass's look-ups local.
+__device__ __forceinline__ uint32_t hash32(uint32_t op, uint32_t shape) {
+    uint32_t h = (shape * 0x9E3779B1u) ^ (op * 0x85EBCA77u);
     h ^= h >> 15;
     h *= 0x2C1B3C6Du;
     h ^= h >> 13;
     return h;
 }
-__device__ __forceinline__ uint32_t hash32(ull key) { return hash32((uint32_t)(key >> 32), (uint32_t)key); }
-
-// 64-bit mixer for the work table: multiply, fold, multiply; the top bits index the table.
-__device__ __forceinline__ ull hash_key(ull key) {
-    ull h = key * 0x9E3779B97F4A7C15ull;
-    h ^= h >> 32;
-    h *= 0xD6E8FEB86659FD93ull;
-    return h;
-}
+__device__ __forceinline__ uint32_t hash32(ull key) { return hash32((uint32_t)(key >> 32) & 0xFFFFu, (uint32_t)key); }
 
 __device__ __forceinline__ ull pack_key(uint32_t phase, uint32_t op, uint32_t shape) {
     return ((ull)phase << 48) | ((ull)op << 32) | (ull)shape;
@@ -114,9 +109,12 @@ constexpr ull NO_INDEX = ~0ull;
 
 __device__ __forceinline__ uint32_t part_of(uint32_t h, uint32_t lp) { return h >> (32 - lp); }  // lp >= 1
 
-// start slot inside the partition, from the hash bits below the partition bits
-__device__ __forceinline__ uint32_t local_of(uint32_t h, uint32_t lp, uint32_t C) { return __umulhi(h << lp, C); }
-// (probe sequences start at the even slot at or below this one and then visit consecutive slots)
+// Start slot inside the partition.  The phase, which the partition choice ignores, is mixed in
+// here so that the phases of one (operator, shape) do not pile up on the same slot.
+// (Probe sequences start at the even slot at or below this one and then visit consecutive slots.)
+__device__ __forceinline__ uint32_t local_of(uint32_t h, uint32_t phase, uint32_t C) {
+    return __umulhi((h ^ (phase * 0x9E3779B9u)) * 0x85EBCA6Bu, C);
+}
 
 // Find (or claim) the slot of `key` directly in HBM.  Returns NO_INDEX when the key's
 // partition has no free slot.  Used off the hot path: directory flush, buffer overflow,
@@ -124,7 +122,7 @@ __device__ __forceinline__ uint32_t local_of(uint32_t h, uint32_t lp, uint32_t C
 __device__ __forceinline__ ull find_or_claim(const TableRef& t, ull key, uint32_t h) {
     const ull skey = ~key;
     const ull base = (ull)part_of(h, t.lp) * t.C;
-    uint32_t s = local_of(h, t.lp, t.C) & ~1u;
+    uint32_t s = local_of(h, (uint32_t)(key >> 48), t.C) & ~1u;
     for (uint32_t probe = 0; probe < t.C; ++probe) {
         ull* kp = t.keys + base + s;
         ull k = ld_relaxed(kp);

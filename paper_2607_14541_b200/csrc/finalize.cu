@@ -81,9 +81,11 @@ __device__ __forceinline__ double roofline_time(const WorkRef& w, const atrex_hw
     if (w.table == nullptr) return qnan;
     ull pair = key & 0x0000FFFFFFFFFFFFull;
     ull skey = ~pair;
-    ull s = hash_key(pair) >> w.shift;
-    for (uint32_t probe = 0; probe < w.max_probe; ++probe) {
-        const WorkSlot* e = w.table + s;
+    const uint32_t h = hash32(pair);
+    const WorkSlot* part = w.table + (ull)part_of(h, w.lp) * w.Cw;
+    uint32_t s = local_of(h, 0u, w.Cw);
+    for (uint32_t probe = 0; probe < w.Cw; ++probe) {
+        const WorkSlot* e = part + s;
         ull k = e->skey;
         if (k == skey) {
             double t_compute = __ddiv_rn(__ull2double_rn(e->flops), pk.peak_flops[e->dtype & (ATREX_MAX_DTYPES - 1)]);
@@ -91,7 +93,7 @@ __device__ __forceinline__ double roofline_time(const WorkRef& w, const atrex_hw
             return fmax(t_compute, t_memory);
         }
         if (k == 0) break;
-        s = (s + 1) & w.mask;
+        s = (s + 1 == w.Cw) ? 0u : s + 1;
     }
     return qnan;
 }
@@ -177,10 +179,12 @@ __global__ void __launch_bounds__(256) work_insert_kernel(const atrex_work_t* ro
         }
         ull pair = ((ull)r.op_id << 32) | (ull)r.shape_id;
         ull skey = ~pair;
-        ull s = hash_key(pair) >> w.shift;
+        const uint32_t h = hash32(pair);
+        WorkSlot* part = w.table + (ull)part_of(h, w.lp) * w.Cw;
+        uint32_t s = local_of(h, 0u, w.Cw);
         bool done = false;
-        for (uint32_t probe = 0; probe < w.max_probe && !done; ++probe) {
-            WorkSlot* e = w.table + s;
+        for (uint32_t probe = 0; probe < w.Cw && !done; ++probe) {
+            WorkSlot* e = part + s;
             ull old = atomicCAS(&e->skey, 0ull, skey);
             if (old == 0) {
                 e->flops = r.flops;
@@ -191,7 +195,7 @@ __global__ void __launch_bounds__(256) work_insert_kernel(const atrex_work_t* ro
                 atomicOr(&ctl->work_status, ST_WORK_DUP);
                 done = true;
             } else {
-                s = (s + 1) & w.mask;
+                s = (s + 1 == w.Cw) ? 0u : s + 1;
             }
         }
         if (!done) atomicOr(&ctl->work_status, ST_WORK_FULL);

@@ -39,11 +39,15 @@ constexpr uint32_t NEW_KEY_FLAG = 0x80000000u;     // partition pass: slot claim
 
 // Bucket of the hot directory.  The odd multiplier is picked per build among DIR_MULTS so that
 // as little sampled weight as possible is lost to buckets that more than two hot keys map to.
-__device__ __forceinline__ uint32_t dir_bucket(uint32_t h, uint32_t mult, uint32_t n_buckets) {
-    return __umulhi(h * mult, n_buckets);
+// The table hash `h` leaves the phase out, the directory must not: the phases of a hot
+// (operator, shape) are usually all hot and would otherwise fight over one bucket.
+__device__ __forceinline__ uint32_t dir_bucket(uint32_t h, uint32_t phase, uint32_t mult, uint32_t n_buckets) {
+    return __umulhi((h + phase * 0x9E3779B9u) * mult, n_buckets);
 }
-__constant__ uint32_t DIR_MULTS[8] = {0xC2B2AE35u, 0x27D4EB2Fu, 0x165667B1u, 0x9E3779B9u,
-                                      0x85EBCA6Bu, 0xD3A2646Du, 0xFD7046C5u, 0xB55A4F09u};
+__device__ __forceinline__ uint32_t dir_bucket_of_key(ull key, uint32_t mult, uint32_t n_buckets) {
+    return dir_bucket(hash32(key), (uint32_t)(key >> 48), mult, n_buckets);
+}
+__constant__ uint32_t DIR_MULTS[4] = {0xC2B2AE35u, 0x27D4EB2Fu, 0x165667B1u, 0x9E3779B9u};
 
 __device__ __forceinline__ void ld_stream_256(const void* p, uint32_t (&w)[8]) {
     asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
@@ -117,14 +121,14 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
         // card-hour weight: from shared memory when the table fits there, else from global
         uint32_t wgt = d.appw_shared ? d.appw_s[ok ? app : 0u] : __ldg(d.appw_g + (ok ? app : 0u));
         prod[r] = (ull)wgt * (ull)w[r][3];
-        h[r] = hash32(khi[r], w[r][2]);
+        h[r] = hash32(khi[r] & 0xFFFFu, w[r][2]);
         todo[r] = ok;
     }
     if (HOT) {
         uint32_t slot[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            uint32_t b = dir_bucket(h[r], d.mult, p.hot_buckets) * DIR_WAYS;
+            uint32_t b = dir_bucket(h[r], khi[r] >> 16, d.mult, p.hot_buckets) * DIR_WAYS;
             const ulonglong2 k01 = *reinterpret_cast<const ulonglong2*>(d.keys + b);
             const ulonglong2 k23 = *reinterpret_cast<const ulonglong2*>(d.keys + b + 2);
             const ull skey = ~(((ull)khi[r] << 32) | w[r][2]);
@@ -399,7 +403,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                     ulonglong2 ent = ok[u] ? __ldcs(src + e) : make_ulonglong2(0, 0);
                     skey[u] = ~ent.x;
                     v[u] = ent.y;
-                    slot[u] = local_of(hash32(ent.x), q.t.lp, C) & ~1u;  // probe sequence starts at an even slot
+                    slot[u] = local_of(hash32(ent.x), (uint32_t)(ent.x >> 48), C) & ~1u;  // probe sequence starts at an even slot
                     searching[u] = ok[u];
                 }
                 // warp-convergent probe of all four entries, two slots per 16-byte load
@@ -554,6 +558,8 @@ __global__ void __launch_bounds__(256) hot_admit_kernel(HotBuildParams p) {
 }
 
 constexpr uint32_t SELECT_MAX = 14336;  // candidates kept for installation (directory <= 11.6K slots, x1.25)
+constexpr uint32_t OCC_MAX = 3072;      // directory buckets (<= 11.6K / 4)
+constexpr size_t SELECT_SMEM = (size_t)SELECT_MAX * 12 + (size_t)OCC_MAX * 4;
 
 __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -601,31 +607,26 @@ __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
     __syncthreads();
     const uint32_t n_sel = min(s_n, SELECT_MAX);
     // pick the bucket-hash multiplier that loses the least sampled weight: a key is lost when
-    // its bucket's slots are already taken (approximated per class by
-    // arrival order, which is what the installation below does as well)
-    __shared__ uint32_t s_lost[8];
-    uint32_t* occupancy = hist;  // reuse: 1024 counters cover buckets modulo 1024 exactly when
-                                 // folded per pass below
-    if (threadIdx.x < 8) s_lost[threadIdx.x] = 0;
-    __syncthreads();
+    // its bucket's slots are already taken (approximated by arrival order among the keys that
+    // matter, which is close to what the class-ordered installation below does)
+    __shared__ uint32_t s_lost[4];
+    uint32_t* occupancy = c_cnt + SELECT_MAX;  // [OCC_MAX] bucket counters behind the compact lists
     const uint32_t n_buckets = p.hot_slots / DIR_WAYS;
-    for (uint32_t m = 0; m < 8; ++m) {
-        // buckets are examined in slices of 1024 so that the occupancy counters fit `hist`
-        for (uint32_t lo_b = 0; lo_b < n_buckets; lo_b += 1024) {
-            occupancy[threadIdx.x] = 0;
-            __syncthreads();
-            for (uint32_t i = threadIdx.x; i < n_sel; i += blockDim.x) {
-                uint32_t c = c_cnt[i];
-                if (c < 16) continue;  // only keys that matter
-                uint32_t b = dir_bucket(hash32(~c_key[i]), DIR_MULTS[m], n_buckets);
-                if (b >= lo_b && b < lo_b + 1024 && atomicAdd(&occupancy[b - lo_b], 1u) >= DIR_WAYS) atomicAdd(&s_lost[m], c);
-            }
-            __syncthreads();
+    if (threadIdx.x < 4) s_lost[threadIdx.x] = 0;
+    for (uint32_t m = 0; m < 4; ++m) {
+        for (uint32_t i = threadIdx.x; i < n_buckets; i += blockDim.x) occupancy[i] = 0;
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < n_sel; i += blockDim.x) {
+            uint32_t c = c_cnt[i];
+            if (c < 16) continue;
+            uint32_t b = dir_bucket_of_key(~c_key[i], DIR_MULTS[m], n_buckets);
+            if (atomicAdd(&occupancy[b], 1u) >= DIR_WAYS) atomicAdd(&s_lost[m], c);
         }
+        __syncthreads();
     }
     if (threadIdx.x == 0) {
         uint32_t best = 0;
-        for (uint32_t m = 1; m < 8; ++m)
+        for (uint32_t m = 1; m < 4; ++m)
             if (s_lost[m] < s_lost[best]) best = m;
         p.ctl->dir_mult = DIR_MULTS[best];
         s_thr = DIR_MULTS[best];  // broadcast (the threshold is already in registers)
@@ -641,7 +642,7 @@ __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
                 uint32_t c = c_cnt[i];
                 if (c >= lo && c < hi) {
                     ull skey = c_key[i];
-                    uint32_t b = dir_bucket(hash32(~skey), mult, n_buckets) * DIR_WAYS;
+                    uint32_t b = dir_bucket_of_key(~skey, mult, n_buckets) * DIR_WAYS;
                     bool placed = false;
                     for (uint32_t way = 0; way < DIR_WAYS && !placed; ++way) placed = atomicCAS(&p.hot_keys[b + way], 0ull, skey) == 0;
                     if (placed) atomicAdd(&s_inserted, 1u);
@@ -672,7 +673,7 @@ cudaError_t ingest_prepare() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(partition_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(hot_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_MAX * 12);
+    return cudaFuncSetAttribute(hot_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM);
 }
 
 cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream) {
@@ -696,7 +697,7 @@ cudaError_t launch_hot_build(const HotBuildParams& p, int n_sms, cudaStream_t st
     if (grid > n_sms * 8) grid = n_sms * 8;
     hot_count_kernel<<<grid, 256, 0, stream>>>(p);
     hot_admit_kernel<<<grid, 256, 0, stream>>>(p);
-    hot_select_kernel<<<1, 1024, SELECT_MAX * 12, stream>>>(p);
+    hot_select_kernel<<<1, 1024, SELECT_SMEM, stream>>>(p);
     return cudaGetLastError();
 }
 

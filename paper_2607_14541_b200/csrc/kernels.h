@@ -51,10 +51,9 @@ struct HotBuildParams {
 };
 
 struct WorkRef {
-    WorkSlot* table;
-    ull mask;
-    int shift;
-    uint32_t max_probe;
+    WorkSlot* table;     // [P * Cw], nullptr when no work table was provisioned
+    uint32_t lp;         // log2(P), same partitioning as the key table
+    uint32_t Cw;         // slots per partition
 };
 
 struct FinalizeParams {
