@@ -30,6 +30,10 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "trace records aggregated/sec"
+# DRAM bytes (read + written) per 2^27-record ingest call of this workload, from the ncu captures
+# summarised in profiles/bench_launch_list_chunked_1B.md: scatter_kernel 4.41 GB per launch plus
+# the three partition drains of a step (12.15 GB) spread over its eight calls.
+NCU_DRAM_BYTES_PER_INGEST_CALL = 5.93e9
 UNIT = "records/s"
 WORKLOAD_INDEX = 3
 RECORD_BYTES = 16
@@ -253,13 +257,17 @@ def run_ours(args):
         peak, peak_src = measured_peak_hbm()
         mean_ingest_ms = statistics.mean(ingest_ms)
         achieved = chunk * RECORD_BYTES / (mean_ingest_ms * 1e-3) / 1e9
-        roofline = {"bound": "hbm", "kernel": "ingest_kernel<hot>", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "traffic": args.ncu_traffic_bytes,
+        traffic = args.ncu_traffic_bytes
+        if traffic is None and chunk == (1 << 27):
+            traffic = NCU_DRAM_BYTES_PER_INGEST_CALL
+        roofline = {"bound": "hbm", "kernel": "ingest pass: scatter_kernel (dominant) + partition_kernel drains",
+                    "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                     "algorithmic_bytes_per_launch": chunk * RECORD_BYTES, "launch_ms_mean": mean_ingest_ms,
                     "launch_ms_best": min(ingest_ms), "peak_source": peak_src,
                     "frac_of_nominal_8TBs": achieved / 8000.0,
-                    "note": "duration = CUDA events around each ingest call; call 0 of a step also holds the "
-                            "hot-directory build launch"}
+                    "note": "duration = CUDA events around each ingest call (scatter launch + partition launch, "
+                            "which drains the spill buffers every third call); call 0 of a step also holds the "
+                            "hot-directory build; achieved = 16 B x records / duration"}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "u64/u128 integer, f64 ratios", "data": "synthetic",
