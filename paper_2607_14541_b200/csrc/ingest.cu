@@ -55,52 +55,94 @@ __device__ __forceinline__ void ld_stream_256(const void* p, uint32_t (&w)[8]) {
                  : "l"(p));
 }
 
+// Shared memory is addressed explicitly through 32-bit shared-window addresses in the hot
+// loops: one integer add per access instead of generic 64-bit pointer arithmetic.
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ ulonglong2 lds_v2u64(uint32_t a) {
+    ulonglong2 v;
+    asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ ull lds_u64(uint32_t a) {
+    ull v;
+    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t atoms_add(uint32_t a, uint32_t v) {
+    uint32_t o;
+    asm volatile("atom.shared.add.u32 %0, [%1], %2;" : "=r"(o) : "r"(a), "r"(v) : "memory");
+    return o;
+}
+__device__ __forceinline__ void reds_add(uint32_t a, uint32_t v) {
+    asm volatile("red.shared.add.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+__device__ __forceinline__ void reds_or(uint32_t a, uint32_t v) {
+    asm volatile("red.shared.or.b32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t atoms_exch(uint32_t a, uint32_t v) {
+    uint32_t o;
+    asm volatile("atom.shared.exch.b32 %0, [%1], %2;" : "=r"(o) : "r"(a), "r"(v) : "memory");
+    return o;
+}
+__device__ __forceinline__ ull atoms_cas64(uint32_t a, ull expected, ull desired) {
+    ull o;
+    asm volatile("atom.shared.cas.b64 %0, [%1], %2, %3;" : "=l"(o) : "r"(a), "l"(expected), "l"(desired) : "memory");
+    return o;
+}
+
+// Shared-window byte addresses of the scatter pass's arrays.
 struct SmemDir {
-    ull* keys;        // [slots], ~key, 0 = empty
-    uint32_t* a0;     // [slots] this launch's weighted time of the slot: bits 0..31 ...
-    uint32_t* a1;     // [slots] ... and bits 32..63 (carries of a0 are added here by the adder)
-    uint32_t* cnt;    // [slots] this launch's record count of the slot
-    uint32_t* cursor; // [P] entries appended to this CTA's buffer of each partition
-    uint32_t mult;    // bucket-hash multiplier of this directory image
-    const uint32_t* appw_s;  // card-hour weights in shared memory (when they fit) ...
-    const uint32_t* appw_g;  // ... else in global memory
+    uint32_t keys;    // ull[slots], ~key, 0 = empty
+    uint32_t a0;      // u32[slots] this launch's weighted time of the slot: bits 0..31 ...
+    uint32_t a1;      // u32[slots] ... and bits 32.. (carries of a0 are added here by the adder)
+    uint32_t cnt;     // u32[slots] this launch's record count of the slot
+    uint32_t cursor;  // u32[P] entries appended to this CTA's buffer of each partition
+    uint32_t appw;    // u32[n_apps] card-hour weights, when they fit in shared memory ...
+    const uint32_t* appw_g;  // ... else they are read from global memory
     bool appw_shared;
+    uint32_t mult;    // bucket-hash multiplier of this directory image
 };
 
 // Shared-memory accumulation uses native 32-bit atomics only (64-bit shared atomics are
 // compare-and-swap loops).  A slot's weighted time is kept in two limbs: the returning add on
-// the low limb tells the adder whether it wrapped, and the adder then adds the carry, with
-// the value's high word, to the high limb.  The high limb grows by less than 2^16 per record,
-// so it is drained every 2^14 counted records (the returning count add elects the drainer):
-// 2^14 records plus the adds that can slip in before the drain (at most one warp's worth per
-// thread of the CTA, 2^15 records) stay below 2^32.
-constexpr uint32_t DRAIN_SHIFT = 14;
+// the low limb tells the adder whether it wrapped, and the adder then adds the carry, with the
+// value's high word, to the high limb.  One add raises the high limb by at most 2^21 (a warp's
+// combined 32 records of < 2^48 each), so the adder that takes it across 2^30 drains both
+// limbs; the adds that can slip in before its exchange (one per thread of the CTA) stay below
+// 2^31, so the high limb never wraps.
+constexpr uint32_t DRAIN_BIT = 0x40000000u;
 
-__device__ __forceinline__ bool limbs_add(uint32_t* a0, uint32_t* a1, uint32_t* cnt, ull v, uint32_t count) {
-    uint32_t v0 = (uint32_t)v;
-    uint32_t o0 = atomicAdd(a0, v0);
-    uint32_t x = (uint32_t)(v >> 32) + ((o0 + v0 < o0) ? 1u : 0u);
-    if (x != 0) atomicAdd(a1, x);
-    uint32_t c = atomicAdd(cnt, count) & 0x7FFFFFFFu;
-    return ((c + count) >> DRAIN_SHIFT) != (c >> DRAIN_SHIFT);  // true: the caller must drain
+// returns true when the caller must drain the slot
+__device__ __forceinline__ bool limbs_add(uint32_t a0, uint32_t a1, uint32_t cnt, ull v, uint32_t count) {
+    const uint32_t v0 = (uint32_t)v;
+    const uint32_t o0 = atoms_add(a0, v0);
+    const uint32_t x = (uint32_t)(v >> 32) + ((o0 + v0 < o0) ? 1u : 0u);
+    const uint32_t o1 = atoms_add(a1, x);
+    reds_add(cnt, count);
+    return ((o1 ^ (o1 + x)) & DRAIN_BIT) && !(o1 & DRAIN_BIT);
 }
 
-__device__ __forceinline__ ull limbs_drain(uint32_t* a0, uint32_t* a1, ull* hi_out) {
+__device__ __forceinline__ ull limbs_drain(uint32_t a0, uint32_t a1, ull* hi_out) {
     // the two exchanges need not be simultaneous: whatever lands between them stays in the
     // limbs for the next drain or the final flush
-    ull lo = atomicExch(a0, 0u);
-    ull hi = atomicExch(a1, 0u);
-    ull v = lo + (hi << 32);
-    *hi_out = (hi >> 32) + (v < lo ? 1ull : 0ull);
+    const ull lo = atoms_exch(a0, 0u);
+    const ull hi = atoms_exch(a1, 0u);
+    const ull v = lo + (hi << 32);
+    *hi_out = v < lo ? 1ull : 0ull;
     return v;
 }
 
 // Add (count, v) to a directory slot, v < 2^53, count <= 32.
 __device__ __forceinline__ void dir_add(const SmemDir& d, uint32_t slot, ull v, uint32_t count, const TableRef& t,
                                         uint32_t h) {
-    if (limbs_add(&d.a0[slot], &d.a1[slot], &d.cnt[slot], v, count)) {
-        ull hi, lo = limbs_drain(&d.a0[slot], &d.a1[slot], &hi);
-        table_accumulate(t, ~d.keys[slot], h, lo, hi, 0);
+    if (limbs_add(d.a0 + slot * 4, d.a1 + slot * 4, d.cnt + slot * 4, v, count)) {
+        ull hi, lo = limbs_drain(d.a0 + slot * 4, d.a1 + slot * 4, &hi);
+        table_accumulate(t, ~lds_u64(d.keys + slot * 8), h, lo, hi, 0);
     }
 }
 
@@ -116,10 +158,10 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
     for (int r = 0; r < R; ++r) {
         uint32_t app = w[r][0];
         khi[r] = w[r][1] & 0x00FFFFFFu;                 // phase << 16 | op_id: the key's high word
-        bool ok = (FULL || present[r]) && app < p.n_apps && (khi[r] >> 16) < p.n_phases;
+        bool ok = (FULL || present[r]) && app < p.n_apps && khi[r] < (p.n_phases << 16);
         rejected += ((FULL || present[r]) && !ok) ? 1u : 0u;
         // card-hour weight: from shared memory when the table fits there, else from global
-        uint32_t wgt = d.appw_shared ? d.appw_s[ok ? app : 0u] : __ldg(d.appw_g + (ok ? app : 0u));
+        uint32_t wgt = d.appw_shared ? lds_u32(d.appw + (ok ? app : 0u) * 4) : __ldg(d.appw_g + (ok ? app : 0u));
         prod[r] = (ull)wgt * (ull)w[r][3];
         h[r] = hash32(khi[r] & 0xFFFFu, w[r][2]);
         todo[r] = ok;
@@ -129,8 +171,8 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
 #pragma unroll
         for (int r = 0; r < R; ++r) {
             uint32_t b = dir_bucket(h[r], khi[r] >> 16, d.mult, p.hot_buckets) * DIR_WAYS;
-            const ulonglong2 k01 = *reinterpret_cast<const ulonglong2*>(d.keys + b);
-            const ulonglong2 k23 = *reinterpret_cast<const ulonglong2*>(d.keys + b + 2);
+            const ulonglong2 k01 = lds_v2u64(d.keys + b * 8);
+            const ulonglong2 k23 = lds_v2u64(d.keys + b * 8 + 16);
             const ull skey = ~(((ull)khi[r] << 32) | w[r][2]);
             uint32_t way = k01.x == skey ? 0u : (k01.y == skey ? 1u : (k23.x == skey ? 2u : (k23.y == skey ? 3u : DIR_WAYS)));
             slot[r] = (!todo[r] || way == DIR_WAYS) ? NO_SLOT : b + way;
@@ -166,7 +208,7 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
     // spill: append {key, product} to this CTA's buffer of the key's partition
     uint32_t pos[R];
 #pragma unroll
-    for (int r = 0; r < R; ++r) pos[r] = todo[r] ? atomicAdd(&d.cursor[part_of(h[r], p.t.lp)], 1u) : 0u;
+    for (int r = 0; r < R; ++r) pos[r] = todo[r] ? atoms_add(d.cursor + part_of(h[r], p.t.lp) * 4, 1u) : 0u;
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         if (todo[r]) {
@@ -262,37 +304,42 @@ __device__ __forceinline__ void scatter_body(const IngestParams& p, const SmemDi
 template <bool HOT>
 __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    SmemDir d;
+    // carve shared memory: directory (keys, limbs, counts), spill cursors, card-hour weights
     unsigned char* sp = smem_raw;
-    d.keys = reinterpret_cast<ull*>(sp);
+    ull* g_keys = reinterpret_cast<ull*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 8 : 0;
-    d.a0 = reinterpret_cast<uint32_t*>(sp);
+    uint32_t* g_a0 = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
-    d.a1 = reinterpret_cast<uint32_t*>(sp);
+    uint32_t* g_a1 = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
-    d.cnt = reinterpret_cast<uint32_t*>(sp);
+    uint32_t* g_cnt = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
-    d.mult = HOT ? (uint32_t)p.t.ctl->dir_mult : 1u;
     const uint32_t n_parts = 1u << p.t.lp;
-    d.cursor = reinterpret_cast<uint32_t*>(sp);
+    uint32_t* g_cursor = reinterpret_cast<uint32_t*>(sp);
     sp += (size_t)n_parts * 4;
-    // the buffers persist across launches until the partition pass drains them: resume the cursors
-    for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) d.cursor[i] = p.spill_cnt[((ull)blockIdx.x << p.t.lp) + i];
-    if (p.appw_in_smem) {
-        uint32_t* s_appw = reinterpret_cast<uint32_t*>(sp);
-        for (uint32_t i = threadIdx.x; i < p.n_apps; i += blockDim.x) s_appw[i] = p.app_w[i];
-        d.appw_s = s_appw;
-    } else {
-        d.appw_s = reinterpret_cast<uint32_t*>(sp);
-    }
+    uint32_t* g_appw = reinterpret_cast<uint32_t*>(sp);
+
+    SmemDir d;
+    d.keys = smem_addr(g_keys);
+    d.a0 = smem_addr(g_a0);
+    d.a1 = smem_addr(g_a1);
+    d.cnt = smem_addr(g_cnt);
+    d.cursor = smem_addr(g_cursor);
+    d.appw = smem_addr(g_appw);
     d.appw_g = p.app_w;
     d.appw_shared = p.appw_in_smem != 0;
+    d.mult = HOT ? (uint32_t)p.t.ctl->dir_mult : 1u;
+
+    // the buffers persist across launches until the partition pass drains them: resume the cursors
+    for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) g_cursor[i] = p.spill_cnt[((ull)blockIdx.x << p.t.lp) + i];
+    if (p.appw_in_smem)
+        for (uint32_t i = threadIdx.x; i < p.n_apps; i += blockDim.x) g_appw[i] = p.app_w[i];
     if (HOT) {
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
-            d.keys[i] = p.hot_keys[i];
-            d.a0[i] = 0;
-            d.a1[i] = 0;
-            d.cnt[i] = 0;
+            g_keys[i] = p.hot_keys[i];
+            g_a0[i] = 0;
+            g_a1[i] = 0;
+            g_cnt[i] = 0;
         }
     }
     __syncthreads();
@@ -312,7 +359,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     bool crowded = false;
     for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) {
         const ull at = ((ull)blockIdx.x << p.t.lp) + i;
-        uint32_t before = p.spill_cnt[at], c = d.cursor[i];
+        uint32_t before = p.spill_cnt[at], c = g_cursor[i];
         p.spill_cnt[at] = min(c, p.cap);
         spilled += min(c, p.cap) - before;
         overflow += c > p.cap ? c - p.cap : 0u;
@@ -332,9 +379,9 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     }
     if (HOT) {
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
-            uint32_t c = d.cnt[i], lo = d.a0[i], hi = d.a1[i];
+            uint32_t c = g_cnt[i], lo = g_a0[i], hi = g_a1[i];
             if ((c | lo | hi) != 0) {
-                ull key = ~d.keys[i];
+                ull key = ~g_keys[i];
                 table_accumulate(p.t, key, hash32(key), (ull)lo | ((ull)hi << 32), 0, (ull)c);
             }
         }
@@ -354,6 +401,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     uint32_t* s_a0 = reinterpret_cast<uint32_t*>(s_keys + C);
     uint32_t* s_a1 = s_a0 + C;
     uint32_t* s_cnt = s_a1 + C;
+    const uint32_t a_keys = smem_addr(s_keys), a_a0 = smem_addr(s_a0), a_a1 = smem_addr(s_a1), a_cnt = smem_addr(s_cnt);
     __shared__ uint32_t s_total;
     const uint32_t n_parts = 1u << q.t.lp;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
@@ -412,19 +460,19 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         if (!searching[u]) continue;
-                        const ulonglong2 kk = *reinterpret_cast<const ulonglong2*>(s_keys + slot[u]);
+                        const ulonglong2 kk = lds_v2u64(a_keys + slot[u] * 8);
                         if (kk.x == skey[u]) {
                             searching[u] = false;
                         } else if (kk.x == 0) {
-                            ull old = atomicCAS(&s_keys[slot[u]], 0ull, skey[u]);  // lost races re-read the pair
-                            if (old == 0) atomicOr(&s_cnt[slot[u]], NEW_KEY_FLAG);
+                            ull old = atoms_cas64(a_keys + slot[u] * 8, 0ull, skey[u]);  // lost races re-read the pair
+                            if (old == 0) reds_or(a_cnt + slot[u] * 4, NEW_KEY_FLAG);
                             if (old == 0 || old == skey[u]) searching[u] = false;
                         } else if (kk.y == skey[u]) {
                             slot[u] += 1;
                             searching[u] = false;
                         } else if (kk.y == 0) {
-                            ull old = atomicCAS(&s_keys[slot[u] + 1], 0ull, skey[u]);
-                            if (old == 0) atomicOr(&s_cnt[slot[u] + 1], NEW_KEY_FLAG);
+                            ull old = atoms_cas64(a_keys + slot[u] * 8 + 8, 0ull, skey[u]);
+                            if (old == 0) reds_or(a_cnt + slot[u] * 4 + 4, NEW_KEY_FLAG);
                             if (old == 0 || old == skey[u]) {
                                 slot[u] += 1;
                                 searching[u] = false;
@@ -447,10 +495,10 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    if (ok[u] && limbs_add(&s_a0[slot[u]], &s_a1[slot[u]], &s_cnt[slot[u]], v[u], 1u)) {
+                    if (ok[u] && limbs_add(a_a0 + slot[u] * 4, a_a1 + slot[u] * 4, a_cnt + slot[u] * 4, v[u], 1u)) {
                         // drain: this CTA owns the slot, so adds into HBM are exact; the write-back
                         // below adds on top of them
-                        ull hi, lo = limbs_drain(&s_a0[slot[u]], &s_a1[slot[u]], &hi);
+                        ull hi, lo = limbs_drain(a_a0 + slot[u] * 4, a_a1 + slot[u] * 4, &hi);
                         ull* vp = reinterpret_cast<ull*>(q.t.vals + base + slot[u]);
                         ull old = atomicAdd(vp, lo);
                         hi += (old + lo < old) ? 1ull : 0ull;
