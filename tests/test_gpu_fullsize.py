@@ -12,7 +12,8 @@ from tests.helpers import entry_wt, f64_bits
 pytestmark = pytest.mark.gpu
 
 
-def test_full_size_chunked_trace_sampled_keys_and_invariants():
+@pytest.mark.parametrize("index", [1, 2, 3, 4])
+def test_full_size_trace_sampled_keys_and_invariants(index):
     import torch
     import paper_2607_14541_b200 as p
     from tracegen.gpu import GpuSampler
@@ -20,7 +21,7 @@ def test_full_size_chunked_trace_sampled_keys_and_invariants():
     free, _ = torch.cuda.mem_get_info()
     if free < 40 << 30:
         pytest.skip("needs ~30 GB of device memory")
-    spec = make_spec(3)
+    spec = make_spec(index)
     n, chunk = spec.n, spec.chunk_records
     work = spec.work_table()
     agg = p.Aggregator(spec.app_weights, spec.n_phases, spec.max_keys, max_work_rows=len(work))
@@ -50,8 +51,9 @@ def test_full_size_chunked_trace_sampled_keys_and_invariants():
     o = oracle.Oracle(spec.app_weights, spec.n_phases)
     o.set_work(work)
     acc, valid = np.zeros(16, dtype=np.uint64), np.zeros(2, dtype=np.uint64)
-    for c in range(spec.n_chunks):
-        host = records[c * chunk * 16:(c + 1) * chunk * 16].cpu().numpy().view(RECORD_DTYPE)
+    piece = 1 << 27                                         # host copies of at most 2 GiB at a time
+    for lo in range(0, n, piece):
+        host = records[lo * 16:min(lo + piece, n) * 16].cpu().numpy().view(RECORD_DTYPE)
         o.ingest_filtered(host, keys)
         o.direct_totals(host, acc, valid)
     assert int(valid[0]) == n and int(valid[1]) == 0
@@ -70,7 +72,17 @@ def test_full_size_chunked_trace_sampled_keys_and_invariants():
     # the ranking: top-k must be the k largest (wt, then smaller key) of the phase's entries
     for ph in range(spec.n_phases):
         sel = ent[(ent["key"] >> np.uint64(48)) == ph]
-        wt = sel["wt_hi"].astype(object) * (1 << 64) + sel["wt_lo"].astype(object)
-        best = sorted(zip((-wt).tolist(), sel["key"].tolist()))[: spec.topk]
+        # pre-select by the high word and the top of the low word, then rank exactly
+        coarse = sel["wt_hi"].astype(np.float64) * 2.0**64 + sel["wt_lo"].astype(np.float64)
+        keep = sel[np.argsort(-coarse, kind="stable")[: 4 * spec.topk + 64]]
+        wt = keep["wt_hi"].astype(object) * (1 << 64) + keep["wt_lo"].astype(object)
+        best = sorted(zip((-wt).tolist(), keep["key"].tolist()))[: spec.topk]
         top = agg.topk(ph, spec.topk)
         assert [int(k) for k in top["key"]] == [k for _, k in best]
+        assert float(coarse[np.argsort(-coarse, kind="stable")[4 * spec.topk + 63]]) < float(-best[-1][0]) or len(sel) <= 4 * spec.topk + 64
+
+    if index == 4:   # every weight 2^20-1, every duration 2^28-1: wt = count * P, with carries into the high word
+        P = (2**20 - 1) * (2**28 - 1)
+        wt_all = ent["wt_hi"].astype(object) * (1 << 64) + ent["wt_lo"].astype(object)
+        assert (wt_all == ent["count"].astype(object) * P).all()
+        assert int(ent["wt_hi"].max()) > 6000
