@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 
 METRIC = "trace records aggregated/sec"
 # DRAM bytes (read + written) per 2^27-record ingest call of this workload, from the ncu captures
-# summarised in profiles/bench_launch_list_chunked_1B.md: scatter_kernel 4.41 GB per launch plus
+# summarised under profiles/: scatter_kernel 4.41 GB per launch plus
 # the three partition drains of a step (12.15 GB) spread over its eight calls.
 NCU_DRAM_BYTES_PER_INGEST_CALL = 5.93e9
 UNIT = "records/s"

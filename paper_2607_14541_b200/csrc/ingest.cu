@@ -12,15 +12,17 @@
 //     hit the same slot are first combined with warp reductions.
 //   * Every other record becomes a 16-byte {key, product} entry appended to the CTA's private
 //     buffer for the key's partition.  Appends of one (CTA, partition) pair are sequential in
-//     memory, so L2 merges them into full lines before they reach HBM.
-//   At the end the CTA flushes its directory accumulators into the table (these few thousand
-//   slots stay L2-resident) and publishes its per-partition entry counts.
+//     memory; the next 128-byte line of a buffer is prefetched into L2 shortly before the
+//     appends reach it, because a partial store into a line that is not cached stalls on a fill.
+//   At the end the CTA adds its directory accumulators to the table (these few thousand slots
+//   stay L2-resident) and stores its per-partition cursors: the buffers persist across launches.
 //
-// Pass 2  PARTITION  (one CTA per partition).  The CTA copies its partition's keys from HBM
-//   into shared memory, streams the partition's entries from all scatter CTAs, finds or
-//   claims each key's slot in shared memory and accumulates there, then adds the per-slot
-//   deltas back to the HBM table with coalesced read-modify-writes.  The CTA is the only
-//   writer of its partition, so no global atomics are involved.
+// Pass 2  PARTITION  (persistent CTAs, one partition at a time each).  Runs lazily: only when a
+//   buffer is filling up, or when results are about to be read.  The CTA copies its
+//   partition's keys from HBM into shared memory, streams the partition's entries from all
+//   scatter CTAs, finds or claims each key's slot in shared memory and accumulates there, then
+//   adds the per-slot deltas back to the HBM table with coalesced read-modify-writes.  The CTA
+//   is the only writer of its partition, so no global atomics are involved.
 //
 // All sums are integers, so the result does not depend on which route a record took, on
 // scheduling, or on chunking.  Entries that do not fit a spill buffer, directory wraps and
