@@ -168,6 +168,18 @@ int atrex_agg_merge(atrex_agg_t*, const atrex_entry_t* d_entries, uint64_t n, vo
 int atrex_agg_finalize(atrex_agg_t*, const atrex_hw_peaks_t* peaks, atrex_entry_t* d_out,
                        uint64_t out_cap, uint64_t* n_out, void* stream);
 
+/* atrex_agg_finalize for one shard of a trace that was split over several handles (GPUs).
+ * Eq. 3 normalises by the phase total over ALL records; when every handle holds only the keys it
+ * owns (after the partial aggregates were exchanged and folded with atrex_agg_merge), the caller
+ * adds the handles' per-phase totals (atrex_agg_stats, as 128-bit integers) and passes the sums
+ * here: total_lo / total_hi are HOST arrays of ATREX_MAX_PHASES low / high 64-bit words.  The
+ * entries written, and those atrex_agg_topk returns afterwards, then carry
+ * phase_weight = fl(fl(wt) / fl(global total)), bit-identical to a single handle that saw every
+ * record.  Everything else is as in atrex_agg_finalize. */
+int atrex_agg_finalize_with_totals(atrex_agg_t*, const atrex_hw_peaks_t* peaks, const uint64_t* total_lo,
+                                   const uint64_t* total_hi, atrex_entry_t* d_out, uint64_t out_cap,
+                                   uint64_t* n_out, void* stream);
+
 /* Table 2: the min(k, keys of `phase`) entries with the largest weighted time, compared as
  * exact 128-bit integers, ties broken by ascending key; written in that order to `h_out`
  * (HOST, capacity k).  k <= ATREX_MAX_TOPK.  Uses the totals and peaks of the last finalize

@@ -41,6 +41,7 @@ EXPORTED_SYMBOLS = [
     "atrex_agg_ingest_host", "atrex_agg_merge", "atrex_agg_finalize", "atrex_agg_topk", "atrex_agg_stats",
     "atrex_agg_reset", "atrex_agg_destroy", "atrex_strerror", "atrex_agg_last_cuda_error",
     "atrex_agg_launch_count", "atrex_topk_entries_static", "atrex_agg_hot_directory",
+    "atrex_agg_finalize_with_totals",
 ]
 
 
@@ -77,6 +78,7 @@ def _load():
     L.atrex_agg_ingest_host.argtypes = [vp, vp, u64, vp]
     L.atrex_agg_merge.argtypes = [vp, vp, u64, vp]
     L.atrex_agg_finalize.argtypes = [vp, C.POINTER(atrex_hw_peaks_t), vp, u64, C.POINTER(u64), vp]
+    L.atrex_agg_finalize_with_totals.argtypes = [vp, C.POINTER(atrex_hw_peaks_t), vp, vp, vp, u64, C.POINTER(u64), vp]
     L.atrex_agg_topk.argtypes = [vp, u32, u32, vp, C.POINTER(u32), vp]
     L.atrex_agg_stats.argtypes = [vp, C.POINTER(atrex_stats_t), vp]
     L.atrex_agg_reset.argtypes = [vp, vp]
@@ -103,6 +105,7 @@ atrex_agg_ingest_host = lib.atrex_agg_ingest_host
 atrex_agg_merge = lib.atrex_agg_merge
 atrex_agg_finalize = lib.atrex_agg_finalize
 atrex_agg_topk = lib.atrex_agg_topk
+atrex_agg_finalize_with_totals = lib.atrex_agg_finalize_with_totals
 atrex_agg_stats = lib.atrex_agg_stats
 atrex_agg_reset = lib.atrex_agg_reset
 atrex_agg_hot_directory = lib.atrex_agg_hot_directory
@@ -232,22 +235,36 @@ class Aggregator:
             n = entries.numel() * entries.element_size() // 48
         self._check(atrex_agg_merge(self._h, entries.data_ptr(), int(n), self._stream(stream)), "atrex_agg_merge")
 
-    def finalize(self, peak_bw: float, peak_flops, out=None, stream=None):
-        """Returns (entries, n): a CUDA uint8 tensor of 48-byte entries and the entry count."""
+    def finalize(self, peak_bw: float, peak_flops, out=None, stream=None, global_totals=None):
+        """Returns (entries, n): a CUDA uint8 tensor of 48-byte entries and the entry count.
+
+        ``global_totals`` (a list of per-phase 128-bit integers summed over all shards) switches to
+        ``atrex_agg_finalize_with_totals``."""
         torch = self._torch
         pk = make_peaks(peak_bw, peak_flops)
         n_out = C.c_uint64(0)
+        if global_totals is not None:
+            t = list(global_totals) + [0] * (ATREX_MAX_PHASES - len(global_totals))
+            lo = np.array([x & 0xFFFFFFFFFFFFFFFF for x in t[:ATREX_MAX_PHASES]], dtype=np.uint64)
+            hi = np.array([x >> 64 for x in t[:ATREX_MAX_PHASES]], dtype=np.uint64)
+
+            def call(ptr, cap):
+                return atrex_agg_finalize_with_totals(self._h, C.byref(pk), lo.ctypes.data, hi.ctypes.data, ptr, cap,
+                                                      C.byref(n_out), self._stream(stream))
+            name = "atrex_agg_finalize_with_totals"
+        else:
+            def call(ptr, cap):
+                return atrex_agg_finalize(self._h, C.byref(pk), ptr, cap, C.byref(n_out), self._stream(stream))
+            name = "atrex_agg_finalize"
         if out is None:
-            rc = atrex_agg_finalize(self._h, C.byref(pk), None, 0, C.byref(n_out), self._stream(stream))
-            self._check(rc, "atrex_agg_finalize")
+            self._check(call(None, 0), name)
             out = torch.empty(max(int(n_out.value), 1) * 48, dtype=torch.uint8, device=f"cuda:{self.device}")
         cap = out.numel() * out.element_size() // 48
-        rc = atrex_agg_finalize(self._h, C.byref(pk), out.data_ptr(), cap, C.byref(n_out), self._stream(stream))
-        self._check(rc, "atrex_agg_finalize")
+        self._check(call(out.data_ptr(), cap), name)
         return out, int(n_out.value)
 
-    def finalize_numpy(self, peak_bw: float, peak_flops, stream=None) -> np.ndarray:
-        out, n = self.finalize(peak_bw, peak_flops, stream=stream)
+    def finalize_numpy(self, peak_bw: float, peak_flops, stream=None, global_totals=None) -> np.ndarray:
+        out, n = self.finalize(peak_bw, peak_flops, stream=stream, global_totals=global_totals)
         return out[: n * 48].cpu().numpy().view(ENTRY_DTYPE).copy()
 
     def topk(self, phase: int, k: int, stream=None) -> np.ndarray:

@@ -483,8 +483,25 @@ static FinalizeParams finalize_params(const atrex_agg* h, atrex_entry_t* out, ui
     return p;
 }
 
+static int finalize_impl(atrex_agg_t* h, const atrex_hw_peaks_t* peaks, const uint64_t* total_lo,
+                         const uint64_t* total_hi, atrex_entry_t* d_out, uint64_t out_cap, uint64_t* n_out,
+                         void* stream);
+
 int atrex_agg_finalize(atrex_agg_t* h, const atrex_hw_peaks_t* peaks, atrex_entry_t* d_out, uint64_t out_cap,
                        uint64_t* n_out, void* stream) {
+    return finalize_impl(h, peaks, nullptr, nullptr, d_out, out_cap, n_out, stream);
+}
+
+int atrex_agg_finalize_with_totals(atrex_agg_t* h, const atrex_hw_peaks_t* peaks, const uint64_t* total_lo,
+                                   const uint64_t* total_hi, atrex_entry_t* d_out, uint64_t out_cap,
+                                   uint64_t* n_out, void* stream) {
+    if (!total_lo || !total_hi) return ATREX_ERR_INVALID;
+    return finalize_impl(h, peaks, total_lo, total_hi, d_out, out_cap, n_out, stream);
+}
+
+static int finalize_impl(atrex_agg_t* h, const atrex_hw_peaks_t* peaks, const uint64_t* total_lo,
+                         const uint64_t* total_hi, atrex_entry_t* d_out, uint64_t out_cap, uint64_t* n_out,
+                         void* stream) {
     if (!h || !peaks || !n_out) return ATREX_ERR_INVALID;
     if (d_out && ((uintptr_t)d_out & 15u) != 0) return ATREX_ERR_INVALID;
     if (!d_out) out_cap = 0;
@@ -498,6 +515,11 @@ int atrex_agg_finalize(atrex_agg_t* h, const atrex_hw_peaks_t* peaks, atrex_entr
     if (rc != ATREX_OK) return rc;
     rc = run_totals(h, s);
     if (rc != ATREX_OK) return rc;
+    if (total_lo) {
+        // normalise by the totals over all shards instead of this handle's own
+        CU(h, cudaMemcpyAsync(h->ctl->total_lo, total_lo, sizeof(ull) * ATREX_MAX_PHASES, cudaMemcpyHostToDevice, s));
+        CU(h, cudaMemcpyAsync(h->ctl->total_hi, total_hi, sizeof(ull) * ATREX_MAX_PHASES, cudaMemcpyHostToDevice, s));
+    }
     CU(h, cudaMemsetAsync(&h->ctl->n_out, 0, sizeof(ull), s));
     CU(h, launch_emit(finalize_params(h, d_out, out_cap), h->scan_grid(h->L.n_slots, 256 * 4), s));
     h->launches++;

@@ -114,3 +114,54 @@ def merge_ranked(candidates: list[np.ndarray], k: int) -> np.ndarray:
     wt = allc["wt_hi"].astype(object) * (1 << 64) + allc["wt_lo"].astype(object)
     order = sorted(range(len(allc)), key=lambda i: (-wt[i], int(allc["key"][i])))
     return allc[order[:k]]
+
+
+def owner_of_keys_torch(keys):
+    """``owner_of_keys`` on a CUDA int64 tensor of packed keys; ``world`` is applied by the caller."""
+    import torch
+    h = keys * torch.tensor(-7046029254386353131, dtype=torch.int64, device=keys.device)  # 0x9E3779B97F4A7C15
+    return (h >> 33) & 0x7FFFFFFF  # logical shift of the product's top 31 bits
+
+
+def bucket_entries_by_owner_torch(entries, n: int, world: int):
+    """Split a CUDA uint8 tensor of ``n`` 48-byte entries into per-destination tensors (on the device)."""
+    import torch
+    e = entries[: n * ENTRY_BYTES].view(torch.int64).view(n, ENTRY_BYTES // 8)
+    owner = owner_of_keys_torch(e[:, 0]) % world
+    order = torch.argsort(owner, stable=True)
+    counts = torch.bincount(owner, minlength=world).tolist()
+    sorted_e = e[order].contiguous().view(torch.uint8).view(-1)
+    out, off = [], 0
+    for c in counts:
+        out.append(sorted_e[off * ENTRY_BYTES:(off + c) * ENTRY_BYTES])
+        off += c
+    return out
+
+
+def merge_and_finalize_owned(owner_agg, parts, peak_bw, peak_flops, global_totals):
+    """Owner side of the exchange: fold the entry tensors received from every rank into
+    ``owner_agg`` (``atrex_agg_merge``) and finalize against the totals over all shards."""
+    for part in parts:
+        if part.numel():
+            owner_agg.merge(part, part.numel() // ENTRY_BYTES)
+    return owner_agg.finalize(peak_bw, peak_flops, global_totals=global_totals)
+
+
+def aggregate_sharded(local_agg, owner_agg, peak_bw, peak_flops, group=None):
+    """Full multi-GPU flow for one rank, after ``local_agg`` has ingested this rank's slice:
+    finalize locally, send every entry to its key's owner (NCCL all-to-all), fold what arrives into
+    ``owner_agg``, combine the per-phase totals exactly, and finalize the owned keys against them.
+    Returns (entries, n) of the keys this rank owns."""
+    import torch
+    import torch.distributed as dist
+    world = dist.get_world_size(group)
+    local, n = local_agg.finalize(peak_bw, peak_flops)
+    buckets = bucket_entries_by_owner_torch(local, n, world)
+    send_counts = torch.tensor([b.numel() for b in buckets], dtype=torch.int64, device=local.device)
+    recv_counts = torch.empty_like(send_counts)
+    dist.all_to_all_single(recv_counts, send_counts, group=group)
+    recv = torch.empty(int(recv_counts.sum()), dtype=torch.uint8, device=local.device)
+    dist.all_to_all_single(recv, torch.cat(buckets) if buckets else local[:0], recv_counts.tolist(),
+                           send_counts.tolist(), group=group)
+    totals = combine_phase_totals(local_agg.stats()["totals"], group=group)
+    return merge_and_finalize_owned(owner_agg, [recv], peak_bw, peak_flops, totals)
