@@ -49,6 +49,9 @@ def lib():
         L.oracle_stats.argtypes = [C.c_void_p, C.c_void_p]
         L.oracle_finalize.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
         L.oracle_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p]
+        L.oracle_score_candidate.restype = C.c_double
+        L.oracle_score_candidate.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_uint32, C.c_void_p, C.c_void_p]
         L.oracle_u128_to_f64.restype = C.c_double
         L.oracle_u128_to_f64.argtypes = [C.c_uint64, C.c_uint64]
         _lib = L
@@ -131,3 +134,23 @@ class Oracle:
 
 def u128_to_f64(x: int) -> float:
     return lib().oracle_u128_to_f64((x >> 64) & 0xFFFFFFFFFFFFFFFF, x & 0xFFFFFFFFFFFFFFFF)
+
+
+def score_candidates(roofline_s, unit_op, t_cand, correct, w):
+    """Eq. 4-6 for a batch: t_cand, correct are [B, n_units]. Returns (S_agg[B], S_op[B, n_ops], errors[B])."""
+    roofline_s = np.ascontiguousarray(roofline_s, dtype=np.float64)
+    unit_op = np.ascontiguousarray(unit_op, dtype=np.uint32)
+    t_cand = np.ascontiguousarray(t_cand, dtype=np.float64)
+    correct = np.ascontiguousarray(correct, dtype=np.uint8)
+    w = np.ascontiguousarray(w, dtype=np.float64)
+    b, n = t_cand.shape
+    agg = np.zeros(b, dtype=np.float64)
+    s_op = np.zeros((b, w.shape[0]), dtype=np.float64)
+    err = np.zeros(b, dtype=np.uint64)
+    for c in range(b):
+        e = C.c_uint64(0)
+        agg[c] = lib().oracle_score_candidate(roofline_s.ctypes.data, unit_op.ctypes.data, n, t_cand[c].ctypes.data,
+                                              correct[c].ctypes.data, w.ctypes.data, w.shape[0], s_op[c].ctypes.data,
+                                              C.byref(e))
+        err[c] = e.value
+    return agg, s_op, err

@@ -20,6 +20,8 @@
 //   roofline_s[k]   = max(F/P_dtype, M/beta)                  (Eq. 1)
 //   topk(phi, k)    = first k keys of phase phi by (wt descending, key ascending)
 //                                                             (Table 2's ranking)
+// and, downstream of the weights, the roofline score aggregation of Eq. 4-6
+// (oracle_score_candidate below).
 //
 // Readings where the paper is silent: invalid records (application or phase out of
 // range) are skipped and counted; the `pad` byte is ignored; a phase whose total is zero
@@ -312,6 +314,48 @@ int oracle_topk(void* h, const void* peaks, uint32_t phase, uint32_t k, void* ou
     for (uint32_t i = 0; i < m; ++i) e[i] = make_entry(*o, pk, totals, v[i].first, v[i].second);
     *n_out = m;
     return 0;
+}
+
+// Score aggregation (Eq. 4-6), one candidate at a time.
+//   Eq. 4  S_j = T_roofline,j / T_cand,j for every unit j = (operator, shape) that passed the
+//          correctness gate; a value above 1 is an evaluation error: it is counted, not clipped.
+//   Eq. 5  S_i = median of the S_j of operator i's correct shapes, 0 if it has none
+//          (even count: mean of the two middle values).
+//   Eq. 6  S_agg = sum_i w_i * S_i, accumulated in operator order.
+// Readings where the paper is silent: a correct unit whose candidate time is not a finite
+// positive number is an evaluation error too and is left out of the median; units are
+// identified by position, `unit_op[j]` names unit j's operator (any order).
+// out_s_op (n_ops doubles, may be null) receives S_i; returns S_agg; *n_errors counts the errors.
+double oracle_score_candidate(const double* roofline_s, const uint32_t* unit_op, uint64_t n_units,
+                              const double* t_cand, const uint8_t* correct, const double* w, uint32_t n_ops,
+                              double* out_s_op, uint64_t* n_errors) {
+    std::vector<std::vector<double>> per_op(n_ops);
+    uint64_t errors = 0;
+    for (uint64_t j = 0; j < n_units; ++j) {
+        if (!correct[j] || unit_op[j] >= n_ops) continue;
+        double t = t_cand[j];
+        if (!(t > 0.0) || std::isinf(t)) {
+            ++errors;
+            continue;
+        }
+        double s = roofline_s[j] / t;                 // Eq. 4
+        if (s > 1.0) ++errors;
+        per_op[unit_op[j]].push_back(s);
+    }
+    double agg = 0.0;
+    for (uint32_t i = 0; i < n_ops; ++i) {
+        std::vector<double>& v = per_op[i];
+        double s_i = 0.0;                             // Eq. 5: no correct shape -> 0
+        if (!v.empty()) {
+            std::sort(v.begin(), v.end());
+            size_t m = v.size();
+            s_i = (m & 1) ? v[m / 2] : (v[m / 2 - 1] + v[m / 2]) / 2.0;
+        }
+        if (out_s_op) out_s_op[i] = s_i;
+        agg = agg + w[i] * s_i;                       // Eq. 6, operator order
+    }
+    if (n_errors) *n_errors = errors;
+    return agg;
 }
 
 // The integer -> binary64 conversion used above, exposed so tests can pin its rounding.

@@ -304,3 +304,53 @@ def test_filtered_and_direct_totals_agree_with_the_full_group_by():
         f.direct_totals(c, acc, valid)
     assert [int(acc[2 * p]) | (int(acc[2 * p + 1]) << 64) for p in range(8)] == totals
     assert int(valid[0]) == len(recs) - 3 and int(valid[1]) == 3 == rejected
+
+
+# ---------------------------------------------------------------- score aggregation (Eq. 4-6)
+
+def test_score_worked_example(golden_dir):
+    g = load_golden(golden_dir, "score_example.json")
+    u = g["units"]
+    agg, s_op, err = oracle.score_candidates([x["roofline_s"] for x in u], [x["op"] for x in u],
+                                             [[x["t_cand"] for x in u]], [[x["correct"] for x in u]], g["w"])
+    assert list(s_op[0]) == g["S_op"] and float(agg[0]) == g["S_agg"] and int(err[0]) == g["errors"]
+    for x in u:  # the fixture's own per-unit column
+        if x["S_j"] is not None:
+            assert x["roofline_s"] / x["t_cand"] == x["S_j"]
+
+
+def test_score_against_python_statistics():
+    import statistics
+    rng = np.random.default_rng(5)
+    n_ops, n_units, batch = 30, 440, 6              # the paper's release: 30 operators, 440 shapes
+    unit_op = np.sort(rng.integers(0, n_ops, n_units)).astype(np.uint32)
+    roof = np.exp(rng.uniform(np.log(1e-6), np.log(1e-1), n_units))
+    w = rng.dirichlet(np.ones(n_ops) * 0.3)
+    t = roof[None, :] / rng.uniform(0.01, 1.1, (batch, n_units))     # a few land above the roof
+    ok = rng.random((batch, n_units)) < 0.6
+    ok[0, unit_op == 3] = False                                        # an operator with no correct shape
+    t[1, 5] = float("inf")
+    t[1, 6] = -1.0
+    t[1, 7] = float("nan")
+    ok[1, 5:8] = True
+    agg, s_op, err = oracle.score_candidates(roof, unit_op, t, ok, w)
+    for b in range(batch):
+        exp_err, total = 0, 0.0
+        for i in range(n_ops):
+            vals = []
+            for j in np.nonzero((unit_op == i) & ok[b])[0]:
+                if not (t[b, j] > 0.0) or math.isinf(t[b, j]):
+                    exp_err += 1
+                    continue
+                s = float(roof[j]) / float(t[b, j])
+                exp_err += s > 1.0
+                vals.append(s)
+            s_i = statistics.median(vals) if vals else 0.0
+            assert float(s_op[b, i]) == s_i, (b, i)
+            total = total + float(w[i]) * s_i
+        assert float(agg[b]) == total and int(err[b]) == exp_err
+    assert float(s_op[0, 3]) == 0.0
+    # all weights on one operator whose shapes all sit exactly on the roof: S_agg = 1
+    one = np.zeros(n_ops); one[0] = 1.0
+    a, _, e = oracle.score_candidates(roof, unit_op, roof[None, :].copy(), np.ones((1, n_units), bool), one)
+    assert float(a[0]) == 1.0 and int(e[0]) == 0
