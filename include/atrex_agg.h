@@ -208,6 +208,30 @@ int atrex_agg_last_cuda_error(const atrex_agg_t*);
 /* Number of kernels this handle has launched so far (for launch accounting in benchmarks). */
 uint64_t atrex_agg_launch_count(const atrex_agg_t*);
 
+/* Roofline score aggregation (Sec. 3.6, Eq. 4-6), batched over candidates.  No handle.
+ *   Eq. 4  S_j = roofline_s[j] / t_cand[c][j] for every unit j = (operator, shape) of candidate c with
+ *          correct[c][j] != 0.  A value above 1 is an evaluation error: it is counted and NOT clipped.
+ *          A correct unit whose time is not a finite positive number is counted as an error too and
+ *          left out.
+ *   Eq. 5  S_i = median of operator i's S_j (even count: mean of the two middle values), 0 if operator
+ *          i has no usable correct shape.
+ *   Eq. 6  S_agg = sum_i w[i] * S_i, accumulated in operator order.
+ * All pointers are DEVICE memory:
+ *   d_roofline_s [n_units] doubles (e.g. the roofline_s of finalize's entries), d_unit_op [n_units]
+ *   operator index of each unit (any order; units with an index >= n_ops are ignored),
+ *   d_t_cand [n_candidates][n_units] doubles, d_correct [n_candidates][n_units] bytes, d_w [n_ops];
+ *   outputs d_s_agg [n_candidates], d_s_op [n_candidates][n_ops] (may be NULL), d_errors
+ *   [n_candidates] u64 (may be NULL).
+ * n_units <= ATREX_SCORE_MAX_UNITS, n_ops <= ATREX_SCORE_MAX_OPS (else ATREX_ERR_TOO_LARGE).
+ * Asynchronous on `stream`.  Results are bit-reproducible: one round-to-nearest division per unit, an
+ * exact median, and products and sums rounded one by one in operator order. */
+#define ATREX_SCORE_MAX_UNITS 16384u
+#define ATREX_SCORE_MAX_OPS 4096u
+int atrex_score_aggregate(const double* d_roofline_s, const uint32_t* d_unit_op, uint64_t n_units,
+                          const double* d_t_cand, const uint8_t* d_correct, uint64_t n_candidates,
+                          const double* d_w, uint32_t n_ops, double* d_s_agg, double* d_s_op,
+                          uint64_t* d_errors, void* stream);
+
 /* Ranked top-k over an array of entries, for callers that cannot allocate device memory.
  *
  * (The paper has no counterpart to this call; it exists for deployment reasons only.)

@@ -41,7 +41,7 @@ EXPORTED_SYMBOLS = [
     "atrex_agg_ingest_host", "atrex_agg_merge", "atrex_agg_finalize", "atrex_agg_topk", "atrex_agg_stats",
     "atrex_agg_reset", "atrex_agg_destroy", "atrex_strerror", "atrex_agg_last_cuda_error",
     "atrex_agg_launch_count", "atrex_topk_entries_static", "atrex_agg_hot_directory",
-    "atrex_agg_finalize_with_totals",
+    "atrex_agg_finalize_with_totals", "atrex_score_aggregate",
 ]
 
 
@@ -90,6 +90,7 @@ def _load():
     L.atrex_agg_last_cuda_error.argtypes = [vp]
     L.atrex_agg_launch_count.restype = u64
     L.atrex_agg_launch_count.argtypes = [vp]
+    L.atrex_score_aggregate.argtypes = [vp, vp, u64, vp, vp, u64, vp, u32, vp, vp, vp, vp]
     L.atrex_topk_entries_static.argtypes = [vp, u64, u32, u32, vp, C.POINTER(u32), vp]
     return L
 
@@ -114,6 +115,7 @@ atrex_strerror = lib.atrex_strerror
 atrex_agg_last_cuda_error = lib.atrex_agg_last_cuda_error
 atrex_agg_launch_count = lib.atrex_agg_launch_count
 atrex_topk_entries_static = lib.atrex_topk_entries_static
+atrex_score_aggregate = lib.atrex_score_aggregate
 
 
 class AtrexError(RuntimeError):
@@ -132,6 +134,24 @@ def make_peaks(peak_bw: float, peak_flops) -> atrex_hw_peaks_t:
     for i in range(ATREX_MAX_DTYPES):
         pk.peak_flops[i] = float(pf[i])
     return pk
+
+
+def score_aggregate(roofline_s, unit_op, t_cand, correct, w, stream=None):
+    """Eq. 4-6 on the GPU.  CUDA tensors: roofline_s f64[n], unit_op int32[n], t_cand f64[B, n],
+    correct uint8[B, n], w f64[n_ops].  Returns (S_agg f64[B], S_op f64[B, n_ops], errors int64[B])."""
+    import torch
+    b, n = t_cand.shape
+    n_ops = w.numel()
+    dev = t_cand.device
+    s_agg = torch.empty(b, dtype=torch.float64, device=dev)
+    s_op = torch.empty(b, n_ops, dtype=torch.float64, device=dev)
+    err = torch.empty(b, dtype=torch.int64, device=dev)
+    s = torch.cuda.current_stream(dev).cuda_stream if stream is None else stream.cuda_stream
+    rc = atrex_score_aggregate(roofline_s.data_ptr(), unit_op.data_ptr(), n, t_cand.data_ptr(), correct.data_ptr(), b,
+                               w.data_ptr(), n_ops, s_agg.data_ptr(), s_op.data_ptr(), err.data_ptr(), s)
+    if rc != ATREX_OK:
+        raise AtrexError(rc, "atrex_score_aggregate")
+    return s_agg, s_op, err
 
 
 def topk_entries_static(entries, n: int, phase: int, k: int, out, stream=None) -> int:
