@@ -52,6 +52,9 @@ def lib():
         L.oracle_score_candidate.restype = C.c_double
         L.oracle_score_candidate.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_uint32, C.c_void_p, C.c_void_p]
+        L.oracle_eq3_weights.restype = C.c_uint64
+        L.oracle_eq3_weights.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p,
+                                         C.c_void_p, C.c_void_p]
         L.oracle_u128_to_f64.restype = C.c_double
         L.oracle_u128_to_f64.argtypes = [C.c_uint64, C.c_uint64]
         _lib = L
@@ -154,3 +157,15 @@ def score_candidates(roofline_s, unit_op, t_cand, correct, w):
                                               C.byref(e))
         err[c] = e.value
     return agg, s_op, err
+
+
+def eq3_weights(records, app_weights, n_ops: int, n_phases: int, retained=None):
+    """Literal Eq. 2-3 operator weights. Returns (w[n_ops], wtilde[n_ops], n_rejected)."""
+    r = np.ascontiguousarray(records)
+    aw = np.ascontiguousarray(app_weights, dtype=np.uint32)
+    w = np.zeros(n_ops, dtype=np.float64)
+    wt = np.zeros(n_ops, dtype=np.float64)
+    ret = None if retained is None else np.ascontiguousarray(retained, dtype=np.uint8)
+    rej = lib().oracle_eq3_weights(r.ctypes.data, r.shape[0], aw.ctypes.data, aw.shape[0], n_ops, n_phases,
+                                   None if ret is None else ret.ctypes.data, w.ctypes.data, wt.ctypes.data)
+    return w, wt, int(rej)

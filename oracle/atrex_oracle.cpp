@@ -358,6 +358,69 @@ double oracle_score_candidate(const double* roofline_s, const uint32_t* unit_op,
     return agg;
 }
 
+// Operator importance weights exactly as Eq. 2-3 state them (per-application denominators).
+//   Eq. 2  D[i][a][phi] = sum of the durations of operator i's invocations in application a during
+//          phase phi;  D_a[phi] = sum over ALL operators j of D[j][a][phi].
+//   Eq. 3  wtilde_i = sum_a p_a * (1/|Phi_i|) * sum_{phi in Phi_i} D[i][a][phi] / D_a[phi],
+//          w_i = wtilde_i / sum_{j retained} wtilde_j.
+//   p_a = c_a / sum_a c_a (card-hour fractions); Phi_i = the phases in which operator i has any
+//   observed time.  A record is valid iff app < n_apps, op < n_ops and phase < n_phases.
+// Readings where the paper is silent: a phase in which application a has no time at all
+// contributes nothing for that application (0/0 := skipped); an operator with no observed time,
+// or not retained, gets weight 0; sums run in ascending phase, application and operator order and
+// every operation is rounded once (this fixes the bit pattern).
+// retained: n_ops flags or null (= all).  Returns the number of rejected records.
+uint64_t oracle_eq3_weights(const void* records, uint64_t n, const uint32_t* app_weights, uint32_t n_apps,
+                            uint32_t n_ops, uint32_t n_phases, const uint8_t* retained, double* out_w,
+                            double* out_wtilde) {
+    const Rec* recs = (const Rec*)records;
+    std::vector<u128> D((size_t)n_phases * n_ops * n_apps, 0), Da((size_t)n_phases * n_apps, 0);
+    uint64_t rejected = 0;
+    for (uint64_t r = 0; r < n; ++r) {
+        const Rec& x = recs[r];
+        if (x.app_id >= n_apps || x.op_id >= n_ops || x.phase >= n_phases) {
+            ++rejected;
+            continue;
+        }
+        D[((size_t)x.phase * n_ops + x.op_id) * n_apps + x.app_id] += x.duration_ns;   // Eq. 2
+        Da[(size_t)x.phase * n_apps + x.app_id] += x.duration_ns;
+    }
+    u128 c_total = 0;
+    for (uint32_t a = 0; a < n_apps; ++a) c_total += app_weights[a];
+    std::vector<double> wt(n_ops, 0.0);
+    for (uint32_t i = 0; i < n_ops; ++i) {
+        std::vector<uint32_t> phi;                                   // Phi_i
+        for (uint32_t p = 0; p < n_phases; ++p) {
+            bool any = false;
+            for (uint32_t a = 0; a < n_apps && !any; ++a) any = D[((size_t)p * n_ops + i) * n_apps + a] != 0;
+            if (any) phi.push_back(p);
+        }
+        double acc = 0.0;
+        if (!phi.empty() && c_total != 0) {
+            for (uint32_t a = 0; a < n_apps; ++a) {
+                double inner = 0.0;
+                for (uint32_t p : phi) {
+                    u128 d_a = Da[(size_t)p * n_apps + a];
+                    if (d_a == 0) continue;
+                    inner = inner + (double)D[((size_t)p * n_ops + i) * n_apps + a] / (double)d_a;
+                }
+                double avg = inner / (double)phi.size();
+                double p_a = (double)app_weights[a] / (double)c_total;
+                acc = acc + p_a * avg;                              // Eq. 3, first part
+            }
+        }
+        wt[i] = acc;
+    }
+    double total = 0.0;
+    for (uint32_t i = 0; i < n_ops; ++i)
+        if (!retained || retained[i]) total = total + wt[i];
+    for (uint32_t i = 0; i < n_ops; ++i) {
+        if (out_wtilde) out_wtilde[i] = wt[i];
+        out_w[i] = ((!retained || retained[i]) && total > 0.0) ? wt[i] / total : 0.0;    // Eq. 3, normalisation
+    }
+    return rejected;
+}
+
 // The integer -> binary64 conversion used above, exposed so tests can pin its rounding.
 double oracle_u128_to_f64(uint64_t hi, uint64_t lo) { return (double)(((u128)hi << 64) | lo); }
 

@@ -354,3 +354,71 @@ def test_score_against_python_statistics():
     one = np.zeros(n_ops); one[0] = 1.0
     a, _, e = oracle.score_candidates(roof, unit_op, roof[None, :].copy(), np.ones((1, n_units), bool), one)
     assert float(a[0]) == 1.0 and int(e[0]) == 0
+
+
+# ---------------------------------------------------------------- literal Eq. 2-3 operator weights
+
+def test_eq3_worked_example(golden_dir):
+    g = load_golden(golden_dir, "eq3_example.json")
+    recs = records_from_dicts(g["records"])
+    w, wt, rej = oracle.eq3_weights(recs, g["app_weights"], g["n_ops"], g["n_phases"])
+    assert list(wt) == g["wtilde"] and rej == 0
+    assert list(w) == [x / 1.78125 for x in g["wtilde"]]
+    w, wt, _ = oracle.eq3_weights(recs, g["app_weights"], g["n_ops"], g["n_phases"], retained=[1, 1, 0])
+    assert list(w) == [0.21875 / g["retained_01_sum"], 0.75 / g["retained_01_sum"], 0.0]
+
+
+def test_eq3_special_cases_and_python_restatement():
+    spec = make_spec(1, small=True, n=30_000)
+    recs = tg.generate(spec)
+    recs["op_id"][:4] = 999                           # operators outside the table are rejected
+    n_ops = spec.n_ops
+    # one application, one phase: the weight is the plain share of observed time (a library group-sum)
+    one = recs.copy()
+    one["app_id"], one["phase"] = 0, 0
+    w, wt, rej = oracle.eq3_weights(one, [7], n_ops, 1)
+    valid = one[one["op_id"] < n_ops]
+    share = np.bincount(valid["op_id"], weights=None, minlength=n_ops) * 0
+    sums = np.zeros(n_ops, dtype=np.uint64)
+    np.add.at(sums, valid["op_id"], valid["duration_ns"].astype(np.uint64))
+    total = int(sums.sum())
+    assert rej == 4 and [float(x) for x in wt] == [float(int(s)) / float(total) * 1.0 for s in sums]
+    assert abs(float(w.sum()) - 1.0) < n_ops * 2.0**-52
+    # general case against a Python restatement with the same operation order
+    w, wt, rej = oracle.eq3_weights(recs, spec.app_weights, n_ops, spec.n_phases)
+    D, Da = {}, {}
+    for a, o, p, d in zip(recs["app_id"].tolist(), recs["op_id"].tolist(), recs["phase"].tolist(), recs["duration_ns"].tolist()):
+        if o >= n_ops:
+            continue
+        D[(o, a, p)] = D.get((o, a, p), 0) + d
+        Da[(a, p)] = Da.get((a, p), 0) + d
+    c_total = int(spec.app_weights.astype(np.uint64).sum())
+    exp = []
+    for i in range(n_ops):
+        phi = [p for p in range(spec.n_phases) if any(D.get((i, a, p), 0) for a in range(spec.n_apps))]
+        acc = 0.0
+        for a in range(spec.n_apps):
+            inner = 0.0
+            for p in phi:
+                if Da.get((a, p), 0):
+                    inner = inner + float(D.get((i, a, p), 0)) / float(Da[(a, p)])
+            acc = acc + (float(int(spec.app_weights[a])) / float(c_total)) * (inner / float(len(phi))) if phi else acc
+        exp.append(acc)
+    assert [float(x) for x in wt] == exp
+    tot = 0.0
+    for x in exp:
+        tot = tot + x
+    assert [float(x) for x in w] == [x / tot for x in exp]
+    assert abs(float(w.sum()) - 1.0) < n_ops * 2.0**-52               # Eq. 3: the weights sum to 1
+    # equal trace windows: if every application's phase total is the same, Eq. 3 reduces to the
+    # card-hour-weighted share that the main aggregation path computes (checked to rounding)
+    eq = recs[recs["op_id"] < n_ops].copy()
+    eq["phase"] = 0
+    eq["app_id"] = np.arange(len(eq)) % 2
+    eq["duration_ns"] = 1000
+    if (eq["app_id"] == 0).sum() != (eq["app_id"] == 1).sum():
+        eq = eq[:-1]
+    w2, _, _ = oracle.eq3_weights(eq, [1, 3], n_ops, 1)
+    num = np.zeros(n_ops)
+    np.add.at(num, eq["op_id"], np.where(eq["app_id"] == 0, 1.0, 3.0) * 1000.0)
+    assert np.allclose(w2, num / num.sum(), rtol=1e-12, atol=0)
