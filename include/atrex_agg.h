@@ -208,6 +208,36 @@ int atrex_agg_last_cuda_error(const atrex_agg_t*);
 /* Number of kernels this handle has launched so far (for launch accounting in benchmarks). */
 uint64_t atrex_agg_launch_count(const atrex_agg_t*);
 
+/* Operator importance weights exactly as Eq. 2-3 state them (per-application denominators).
+ *
+ * The main path above weights each record by its application's card-hour weight and normalises per
+ * phase.  Eq. 3 proper first turns every application's time into shares of that application's own
+ * phase total, averages an operator's shares over the phases it runs in, and only then weights by
+ * the card-hour fractions:
+ *   Eq. 2  D[i][a][phi] = summed duration_ns of operator i's records of application a in phase phi
+ *          D_a[phi]     = sum over all operators of D[.][a][phi]
+ *   Eq. 3  wtilde_i = sum_a p_a * (1/|Phi_i|) * sum_{phi in Phi_i} D[i][a][phi] / D_a[phi]
+ *          w_i      = wtilde_i / sum of wtilde_j over the retained operators j;  sum_i w_i = 1
+ *   with p_a = app_weights[a] / sum(app_weights) and Phi_i = the phases in which operator i has any time.
+ * A record is valid iff app_id < n_apps, op_id < n_ops and phase < n_phases (others are counted as
+ * rejected; shape_id is not used: the weights are per operator).  A phase in which an application has
+ * no time contributes nothing for that application; operators without time or not retained get 0.
+ * Sums run in ascending phase, application and operator order, each operation rounded once, so the
+ * results are bit-reproducible.  n_apps * n_ops * n_phases <= 2^28 (else ATREX_ERR_TOO_LARGE).
+ *
+ * create     app_weights: HOST, copied.  The library allocates its own device memory.
+ * ingest     d_records: DEVICE, 16-byte aligned; asynchronous; any number of calls; order-independent.
+ * finalize   h_retained: HOST n_ops flags (NULL = all retained); h_w, h_wtilde (may be NULL): HOST
+ *            n_ops doubles; h_rejected (may be NULL): HOST.  Synchronises `stream`; repeatable. */
+typedef struct atrex_eq3 atrex_eq3_t;
+int atrex_eq3_create(uint32_t n_apps, uint32_t n_ops, uint32_t n_phases, const uint32_t* app_weights, int32_t device,
+                     atrex_eq3_t** out);
+int atrex_eq3_ingest(atrex_eq3_t*, const atrex_record_t* d_records, uint64_t n, void* stream);
+int atrex_eq3_finalize(atrex_eq3_t*, const uint8_t* h_retained, double* h_w, double* h_wtilde, uint64_t* h_rejected,
+                       void* stream);
+int atrex_eq3_reset(atrex_eq3_t*, void* stream);
+void atrex_eq3_destroy(atrex_eq3_t*);
+
 /* Roofline score aggregation (Sec. 3.6, Eq. 4-6), batched over candidates.  No handle.
  *   Eq. 4  S_j = roofline_s[j] / t_cand[c][j] for every unit j = (operator, shape) of candidate c with
  *          correct[c][j] != 0.  A value above 1 is an evaluation error: it is counted and NOT clipped.

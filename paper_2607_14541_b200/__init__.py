@@ -3,5 +3,6 @@ and roofline ceilings (the paper's Sec. 3.3-3.4, Eq. 1-3), as hand-written CUDA 
 behind a C ABI (``include/atrex_agg.h``).  This package is the thin Python binding.
 """
 from .binding import *  # noqa: F401,F403
-from .binding import (Aggregator, AtrexError, make_peaks, topk_entries_static, score_aggregate, lib, LIB_PATH,  # noqa: F401
+from .binding import (Aggregator, AtrexError, make_peaks, topk_entries_static, score_aggregate, OperatorWeights,
+                      lib, LIB_PATH,  # noqa: F401
                       EXPORTED_SYMBOLS)

@@ -41,7 +41,8 @@ EXPORTED_SYMBOLS = [
     "atrex_agg_ingest_host", "atrex_agg_merge", "atrex_agg_finalize", "atrex_agg_topk", "atrex_agg_stats",
     "atrex_agg_reset", "atrex_agg_destroy", "atrex_strerror", "atrex_agg_last_cuda_error",
     "atrex_agg_launch_count", "atrex_topk_entries_static", "atrex_agg_hot_directory",
-    "atrex_agg_finalize_with_totals", "atrex_score_aggregate",
+    "atrex_agg_finalize_with_totals", "atrex_score_aggregate", "atrex_eq3_create", "atrex_eq3_ingest",
+    "atrex_eq3_finalize", "atrex_eq3_reset", "atrex_eq3_destroy",
 ]
 
 
@@ -90,6 +91,12 @@ def _load():
     L.atrex_agg_last_cuda_error.argtypes = [vp]
     L.atrex_agg_launch_count.restype = u64
     L.atrex_agg_launch_count.argtypes = [vp]
+    L.atrex_eq3_create.argtypes = [u32, u32, u32, vp, C.c_int32, C.POINTER(vp)]
+    L.atrex_eq3_ingest.argtypes = [vp, vp, u64, vp]
+    L.atrex_eq3_finalize.argtypes = [vp, vp, vp, vp, C.POINTER(u64), vp]
+    L.atrex_eq3_reset.argtypes = [vp, vp]
+    L.atrex_eq3_destroy.argtypes = [vp]
+    L.atrex_eq3_destroy.restype = None
     L.atrex_score_aggregate.argtypes = [vp, vp, u64, vp, vp, u64, vp, u32, vp, vp, vp, vp]
     L.atrex_topk_entries_static.argtypes = [vp, u64, u32, u32, vp, C.POINTER(u32), vp]
     return L
@@ -116,6 +123,11 @@ atrex_agg_last_cuda_error = lib.atrex_agg_last_cuda_error
 atrex_agg_launch_count = lib.atrex_agg_launch_count
 atrex_topk_entries_static = lib.atrex_topk_entries_static
 atrex_score_aggregate = lib.atrex_score_aggregate
+atrex_eq3_create = lib.atrex_eq3_create
+atrex_eq3_ingest = lib.atrex_eq3_ingest
+atrex_eq3_finalize = lib.atrex_eq3_finalize
+atrex_eq3_reset = lib.atrex_eq3_reset
+atrex_eq3_destroy = lib.atrex_eq3_destroy
 
 
 class AtrexError(RuntimeError):
@@ -134,6 +146,53 @@ def make_peaks(peak_bw: float, peak_flops) -> atrex_hw_peaks_t:
     for i in range(ATREX_MAX_DTYPES):
         pk.peak_flops[i] = float(pf[i])
     return pk
+
+
+class OperatorWeights:
+    """Operator importance weights per Eq. 2-3 as written (per-application denominators)."""
+
+    def __init__(self, app_weights, n_ops: int, n_phases: int, device: int = 0):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("the aggregation path is CUDA-only and no CUDA device is available")
+        self._torch, self.device, self.n_ops = torch, int(device), int(n_ops)
+        w = np.ascontiguousarray(app_weights, dtype=np.uint32)
+        h = C.c_void_p()
+        rc = atrex_eq3_create(int(w.shape[0]), int(n_ops), int(n_phases), w.ctypes.data, self.device, C.byref(h))
+        if rc != ATREX_OK:
+            raise AtrexError(rc, "atrex_eq3_create")
+        self._h = h
+
+    def _stream(self, stream=None):
+        return self._torch.cuda.current_stream(self.device).cuda_stream if stream is None else stream.cuda_stream
+
+    def ingest(self, records, n: int | None = None, stream=None):
+        if n is None:
+            n = records.numel() * records.element_size() // 16
+        rc = atrex_eq3_ingest(self._h, records.data_ptr(), int(n), self._stream(stream))
+        if rc != ATREX_OK:
+            raise AtrexError(rc, "atrex_eq3_ingest")
+
+    def finalize(self, retained=None, stream=None):
+        """Returns (w, wtilde, n_rejected)."""
+        w, wt = np.zeros(self.n_ops), np.zeros(self.n_ops)
+        rej = C.c_uint64(0)
+        ret = None if retained is None else np.ascontiguousarray(retained, dtype=np.uint8)
+        rc = atrex_eq3_finalize(self._h, None if ret is None else ret.ctypes.data, w.ctypes.data, wt.ctypes.data,
+                                C.byref(rej), self._stream(stream))
+        if rc != ATREX_OK:
+            raise AtrexError(rc, "atrex_eq3_finalize")
+        return w, wt, int(rej.value)
+
+    def reset(self, stream=None):
+        atrex_eq3_reset(self._h, self._stream(stream))
+
+    def close(self):
+        if getattr(self, "_h", None):
+            atrex_eq3_destroy(self._h)
+            self._h = None
+
+    __del__ = close
 
 
 def score_aggregate(roofline_s, unit_op, t_cand, correct, w, stream=None):
