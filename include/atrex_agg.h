@@ -34,7 +34,10 @@
  *                  (op_id, shape_id) has no work-table row gets the quiet NaN 0x7FF8000000000000
  *   A record is valid iff app_id < n_apps and phase < n_phases; invalid records are skipped
  *   and counted.  The `pad` byte is ignored.
- *   Limits: fewer than 2^40 records per handle between resets (so wt < 2^88).
+ *   Limits: fewer than 2^40 records per handle between resets, and wt < 2^88 per key (always true
+ *   when app_weight * duration_ns < 2^48, e.g. weights < 2^20 and durations < 2^28; larger
+ *   products are accepted and summed exactly, through a slower path, as long as the key's sum
+ *   stays below 2^88).
  */
 #ifndef ATREX_AGG_H
 #define ATREX_AGG_H

@@ -167,6 +167,13 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
         prod[r] = (ull)wgt * (ull)w[r][3];
         h[r] = hash32(khi[r] & 0xFFFFu, w[r][2]);
         todo[r] = ok;
+        // The limb arithmetic below and the 16-byte spill entries assume products below 2^48
+        // (e.g. weights < 2^20, durations < 2^28).  Anything larger is still exact: it goes
+        // straight to the table with full 64-bit adds.
+        if (ok && (prod[r] >> 48) != 0) {
+            table_accumulate(p.t, ((ull)khi[r] << 32) | w[r][2], h[r], prod[r], 0, 1);
+            todo[r] = false;
+        }
     }
     if (HOT) {
         uint32_t slot[R];

@@ -326,3 +326,36 @@ def test_gpu_sampler_matches_numpy_sampler():
         GpuSampler(spec).fill(out, start=1000, count=200_001)
         torch.cuda.synchronize()
         assert out.cpu().numpy().tobytes() == ref.tobytes(), index
+
+
+def test_full_u32_range_of_weights_and_durations(lib):
+    # products up to (2^32-1)^2 do not fit the 48-bit fast path; they must still be exact
+    rng = np.random.default_rng(11)
+    n = 300_000
+    recs = np.zeros(n, dtype=RECORD_DTYPE)
+    recs["app_id"] = rng.integers(0, 4, n)
+    recs["op_id"] = rng.integers(0, 3, n)
+    recs["shape_id"] = rng.integers(0, 50, n)
+    recs["phase"] = rng.integers(0, 2, n)
+    recs["duration_ns"] = rng.choice(np.array([0, 1, 70_000, 0x0FFFFFFF, 0x10000000, 0xFFFFFFFF], dtype=np.uint32), n)
+    weights = np.array([0xFFFFFFFF, 1, 0x00100000, 0x000FFFFF], dtype=np.uint32)
+    o = oracle_of(recs, weights, 2)
+    for flags in (0, lib.ATREX_FLAG_NO_HOT_DIRECTORY):
+        agg = gpu_aggregate(lib, recs, weights, 2, max_keys=1000, flags=flags, chunks=2)
+        got = assert_same_as_oracle(agg, o, 2)
+        assert int(got["wt_hi"].max()) > 0
+
+
+def test_many_apps_eight_phases_and_largest_geometry(lib):
+    # > 4096 applications (weights read from global memory), 8 phases, and the largest table
+    # geometry (4096 partitions)
+    spec = make_spec(1, small=True, n=400_003)
+    recs = tg.generate(spec)
+    rng = np.random.default_rng(3)
+    recs["app_id"] = rng.integers(0, 5000, len(recs))
+    recs["phase"] = rng.integers(0, 8, len(recs))
+    weights = rng.integers(1, 1 << 20, 5000).astype(np.uint32)
+    o = oracle_of(recs, weights, 8)
+    agg = gpu_aggregate(lib, recs, weights, 8, max_keys=1 << 25)
+    assert_same_as_oracle(agg, o, 8, ks=(3,))
+    assert agg.stats()["table_slots"] >= 4096 * 11000
