@@ -55,6 +55,9 @@ def lib():
         L.oracle_eq3_weights.restype = C.c_uint64
         L.oracle_eq3_weights.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.c_void_p,
                                          C.c_void_p, C.c_void_p]
+        L.oracle_sort_by_key.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+        L.oracle_rank_phase.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_void_p, C.c_void_p,
+                                        C.c_uint64, C.c_void_p]
         L.oracle_u128_to_f64.restype = C.c_double
         L.oracle_u128_to_f64.argtypes = [C.c_uint64, C.c_uint64]
         _lib = L
@@ -169,3 +172,27 @@ def eq3_weights(records, app_weights, n_ops: int, n_phases: int, retained=None):
     rej = lib().oracle_eq3_weights(r.ctypes.data, r.shape[0], aw.ctypes.data, aw.shape[0], n_ops, n_phases,
                                    None if ret is None else ret.ctypes.data, w.ctypes.data, wt.ctypes.data)
     return w, wt, int(rej)
+
+
+def sort_by_key(entries: np.ndarray) -> np.ndarray:
+    """Entries ordered by packed key ascending."""
+    e = np.ascontiguousarray(entries, dtype=ENTRY_DTYPE)
+    out = np.zeros(e.shape[0], dtype=ENTRY_DTYPE)
+    lib().oracle_sort_by_key(e.ctypes.data, e.shape[0], out.ctypes.data)
+    return out
+
+
+def rank_phase(entries: np.ndarray, phase: int, coverage_ppm: int, out_cap=None):
+    """Ranked units of one phase, running share, coverage cut (the construction behind Table 2).
+    Returns (ranked entries, cum share, dict(n_phase, n_keep, total, covered))."""
+    e = np.ascontiguousarray(entries, dtype=ENTRY_DTYPE)
+    cap = e.shape[0] if out_cap is None else int(out_cap)
+    out = np.zeros(max(cap, 1), dtype=ENTRY_DTYPE)
+    cum = np.zeros(max(cap, 1), dtype=np.float64)
+    res = np.zeros(6, dtype=np.uint64)
+    lib().oracle_rank_phase(e.ctypes.data, e.shape[0], phase, coverage_ppm, out.ctypes.data, cum.ctypes.data, cap,
+                            res.ctypes.data)
+    m = min(int(res[0]), cap)
+    return out[:m].copy(), cum[:m].copy(), {
+        "n_phase": int(res[0]), "n_keep": int(res[1]),
+        "total": int(res[2]) | (int(res[3]) << 64), "covered": int(res[4]) | (int(res[5]) << 64)}

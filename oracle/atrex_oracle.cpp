@@ -21,7 +21,9 @@
 //   topk(phi, k)    = first k keys of phase phi by (wt descending, key ascending)
 //                                                             (Table 2's ranking)
 // and, downstream of the weights, the roofline score aggregation of Eq. 4-6
-// (oracle_score_candidate below).
+// (oracle_score_candidate below), the literal Eq. 2-3 operator weights (oracle_eq3_weights)
+// and the ranked list with running share and coverage cut behind Table 2
+// (oracle_rank_phase, oracle_sort_by_key).
 //
 // Readings where the paper is silent: invalid records (application or phase out of
 // range) are skipped and counted; the `pad` byte is ignored; a phase whose total is zero
@@ -423,5 +425,70 @@ uint64_t oracle_eq3_weights(const void* records, uint64_t n, const uint32_t* app
 
 // The integer -> binary64 conversion used above, exposed so tests can pin its rounding.
 double oracle_u128_to_f64(uint64_t hi, uint64_t lo) { return (double)(((u128)hi << 64) | lo); }
+
+// Release artefacts made from a list of aggregated units (any order, one entry per key).
+//
+// oracle_sort_by_key: the same entries ordered by packed key ascending (entries with equal keys
+// keep their input order).
+void oracle_sort_by_key(const void* in, uint64_t n, void* out) {
+    const Entry* e = (const Entry*)in;
+    std::vector<Entry> v(e, e + n);
+    std::stable_sort(v.begin(), v.end(), [](const Entry& a, const Entry& b) { return a.key < b.key; });
+    if (n) std::memcpy(out, v.data(), n * sizeof(Entry));
+}
+
+// oracle_rank_phase: the construction behind Table 2 (operators ordered by weight with a
+// running "Cum." share), for the units of one phase:
+//   order   (wt descending, key ascending), wt the exact 128-bit integer;
+//   T       sum of wt over the phase's units;
+//   cum[i]  fl(fl(wt_0 + ... + wt_i) / fl(T)): the running sum is kept as an exact integer and
+//           rounded once, so the column does not drift with the length of the list; +0.0
+//           when T = 0;
+//   n_keep  the coverage cut: the smallest k whose first k units hold at least
+//           coverage_ppm / 10^6 of T, i.e. 10^6 * (wt_0 + ... + wt_{k-1}) >= coverage_ppm * T
+//           in integers (k = 0 when coverage_ppm = 0 or T = 0; units of weight zero are never
+//           needed, so k <= number of units with wt > 0).
+// The first min(n_phase, out_cap) ranked entries go to out_ranked and their cum to out_cum.
+// result = {n_phase, n_keep, T low, T high, covered low, covered high}, covered = the sum of the
+// first n_keep units.  Requires T * 10^6 < 2^128 (T < 2^108).
+void oracle_rank_phase(const void* in, uint64_t n, uint32_t phase, uint32_t coverage_ppm, void* out_ranked,
+                       double* out_cum, uint64_t out_cap, uint64_t result[6]) {
+    const Entry* e = (const Entry*)in;
+    std::vector<Entry> v;
+    u128 total = 0;
+    for (uint64_t i = 0; i < n; ++i)
+        if ((e[i].key >> 48) == phase) {
+            v.push_back(e[i]);
+            total += ((u128)e[i].wt_hi << 64) | e[i].wt_lo;
+        }
+    std::sort(v.begin(), v.end(), [](const Entry& a, const Entry& b) {
+        u128 wa = ((u128)a.wt_hi << 64) | a.wt_lo, wb = ((u128)b.wt_hi << 64) | b.wt_lo;
+        if (wa != wb) return wa > wb;
+        return a.key < b.key;
+    });
+    const u128 need = (u128)coverage_ppm * total;
+    u128 running = 0, covered = 0;
+    uint64_t n_keep = 0;
+    bool cut_found = (u128)1000000 * running >= need;  // k = 0 already covers a target of nothing
+    Entry* out = (Entry*)out_ranked;
+    for (uint64_t i = 0; i < v.size(); ++i) {
+        running += ((u128)v[i].wt_hi << 64) | v[i].wt_lo;
+        if (!cut_found && (u128)1000000 * running >= need) {
+            cut_found = true;
+            n_keep = i + 1;
+            covered = running;
+        }
+        if (i < out_cap) {
+            out[i] = v[i];
+            out_cum[i] = total == 0 ? 0.0 : (double)running / (double)total;
+        }
+    }
+    result[0] = v.size();
+    result[1] = n_keep;
+    result[2] = (uint64_t)total;
+    result[3] = (uint64_t)(total >> 64);
+    result[4] = (uint64_t)covered;
+    result[5] = (uint64_t)(covered >> 64);
+}
 
 }  // extern "C"

@@ -422,3 +422,105 @@ def test_eq3_special_cases_and_python_restatement():
     num = np.zeros(n_ops)
     np.add.at(num, eq["op_id"], np.where(eq["app_id"] == 0, 1.0, 3.0) * 1000.0)
     assert np.allclose(w2, num / num.sum(), rtol=1e-12, atol=0)
+
+
+# ---------------------------------------------------------------- ranked list, running share, coverage cut
+
+def _entries_from(keys, wts, counts=None):
+    e = np.zeros(len(keys), dtype=oracle.ENTRY_DTYPE)
+    e["key"] = np.asarray(keys, dtype=np.uint64)
+    e["wt_lo"] = np.asarray([w & (2**64 - 1) for w in wts], dtype=np.uint64)
+    e["wt_hi"] = np.asarray([w >> 64 for w in wts], dtype=np.uint64)
+    e["count"] = np.arange(1, len(keys) + 1, dtype=np.uint64) if counts is None else counts
+    return e
+
+
+def test_rank_worked_example(golden_dir):
+    g = load_golden(golden_dir, "rank_example.json")
+    keys = [(r["phase"] << 48) | (r["key_op"] << 32) | r["key_shape"] for r in g["entries"]]
+    e = _entries_from(keys, [int(r["wt"]) for r in g["entries"]])
+    ranked, cum, res = oracle.rank_phase(e, g["phase"], 0)
+    assert [[int(k >> 32) & 0xFFFF, int(k) & 0xFFFFFFFF] for k in ranked["key"]] == g["ranked_ops_shapes"]
+    assert list(cum) == g["cum"] and res["n_phase"] == 5 and res["total"] == int(g["total"])
+    assert [entry_wt(x) for x in ranked] == sorted([int(r["wt"]) for r in g["entries"] if r["phase"] == 1], reverse=True)
+    for c in g["cuts"]:
+        _, _, res = oracle.rank_phase(e, g["phase"], c["coverage_ppm"])
+        assert res["n_keep"] == c["n_keep"] and res["covered"] == int(c["covered"]), c
+    # a truncated output reports the same cut
+    ranked2, cum2, res = oracle.rank_phase(e, g["phase"], 875001, out_cap=2)
+    assert len(ranked2) == 2 and list(cum2) == g["cum"][:2] and res["n_keep"] == 4 and res["n_phase"] == 5
+    # a phase that has no units
+    ranked3, _, res = oracle.rank_phase(e, 5, 500000)
+    assert len(ranked3) == 0 and res == {"n_phase": 0, "n_keep": 0, "total": 0, "covered": 0}
+
+
+def test_rank_reproduces_the_printed_cumulative_column(golden_dir):
+    g = load_golden(golden_dir, "table2_cumulative.json")
+    wts = [10 * s for s in g["score_milli"]] + [10 * g["tail_score_milli"] // g["tail_operators"]] * g["tail_operators"]
+    assert sum(wts[10:]) == 10 * g["tail_score_milli"]
+    # keys in an order unrelated to the weights; the two pairs of equal printed scores get keys that
+    # make the expected order unambiguous
+    rng = random.Random(5)
+    order = list(range(len(wts)))
+    rng.shuffle(order)
+    keys = [0] * len(wts)
+    for rank, pos in enumerate(order):
+        keys[rank] = (rank % 7 << 32) | (1000 + pos)
+    shuffled = list(range(len(wts)))
+    rng.shuffle(shuffled)
+    e = _entries_from([keys[i] for i in shuffled], [wts[i] for i in shuffled])
+    ranked, cum, res = oracle.rank_phase(e, 0, 0)
+    assert [entry_wt(x) for x in ranked[:10]] == wts[:10]
+    for i, printed in enumerate(g["cum_printed"]):
+        assert abs(cum[i] - printed) <= (i + 1) * 0.0005 + 0.0005 + 0.001, (i, cum[i], printed)
+    assert cum[-1] == g["tail_cum_printed"] and res["n_phase"] == 30
+    for c in g["cuts"]:
+        assert oracle.rank_phase(e, 0, c["coverage_ppm"])[2]["n_keep"] == c["n_keep"], c
+
+
+def test_rank_against_python_integers_and_the_ranked_topk():
+    spec = make_spec(1, small=True, n=40_000)
+    recs = tg.generate(spec)
+    o, entries = run_oracle(recs, spec.app_weights, spec.n_phases)
+    rng = np.random.default_rng(3)
+    entries = entries[rng.permutation(entries.shape[0])]
+    for phase in range(spec.n_phases):
+        mine = [x for x in entries if int(x["key"]) >> 48 == phase]
+        py = sorted(mine, key=lambda x: (-entry_wt(x), int(x["key"])))
+        total = sum(entry_wt(x) for x in py)
+        for ppm in (0, 1, 333_333, 800_000, 999_999, 1_000_000):
+            ranked, cum, res = oracle.rank_phase(entries, phase, ppm)
+            assert [int(k) for k in ranked["key"]] == [int(x["key"]) for x in py]
+            assert res["total"] == total and res["n_phase"] == len(py)
+            prefix, acc = [], 0
+            for x in py:
+                acc += entry_wt(x)
+                prefix.append(acc)
+            assert [f64_bits(c) for c in cum] == [f64_bits(float(p) / float(total)) for p in prefix]
+            k = res["n_keep"]
+            before = prefix[k - 1] if k else 0
+            assert before * 1_000_000 >= ppm * total and res["covered"] == before
+            assert k == 0 or (prefix[k - 2] if k > 1 else 0) * 1_000_000 < ppm * total     # minimal
+            assert all(cum[i] <= cum[i + 1] for i in range(len(cum) - 1)) and cum[-1] == 1.0
+        # the head of the ranking is the ranked top-k (an independently pinned function)
+        top = o.topk(PEAK_BW, PEAK_FLOPS, phase, 25)
+        ranked, _, _ = oracle.rank_phase(entries, phase, 0, out_cap=25)
+        assert ranked.tobytes() == top.tobytes()
+    # all-zero weights: shares +0.0, nothing kept
+    z = entries.copy()
+    z["wt_lo"] = 0
+    z["wt_hi"] = 0
+    ranked, cum, res = oracle.rank_phase(z, 0, 900_000)
+    assert res["n_keep"] == 0 and res["total"] == 0 and not cum.any() and not np.signbit(cum).any()
+    assert [int(k) for k in ranked["key"]] == sorted(int(k) for k in z["key"] if int(k) >> 48 == 0)
+
+
+def test_sort_by_key_is_a_library_sort():
+    spec = make_spec(2, small=True, n=20_000)
+    _, entries = run_oracle(tg.generate(spec), spec.app_weights, spec.n_phases)
+    rng = np.random.default_rng(11)
+    shuffled = entries[rng.permutation(entries.shape[0])]
+    got = oracle.sort_by_key(shuffled)
+    assert got.tobytes() == shuffled[np.argsort(shuffled["key"], kind="stable")].tobytes()
+    assert got.tobytes() == entries.tobytes()          # finalize already walks the keys in order
+    assert oracle.sort_by_key(entries[:0]).shape[0] == 0
