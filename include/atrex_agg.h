@@ -265,6 +265,50 @@ int atrex_score_aggregate(const double* d_roofline_s, const uint32_t* d_unit_op,
                           const double* d_w, uint32_t n_ops, double* d_s_agg, double* d_s_op,
                           uint64_t* d_errors, void* stream);
 
+/* ---- Release artefacts: the entry list in key order, and the ranked list of one phase with its
+ * running share and coverage cut (Table 2: operators ordered by weight with a "Cum." column; Sec. 3.3:
+ * the weights are shipped as an artefact of their own and recomputed on refresh).
+ *
+ * Both calls work on an array of entries on the DEVICE (atrex_agg_finalize's output, or the
+ * concatenation of several shards' outputs), one entry per key, and on caller-provided DEVICE
+ * scratch of at least atrex_release_scratch_bytes(n) bytes, 256-byte aligned, whose contents are
+ * undefined afterwards.  n <= ATREX_RELEASE_MAX_ENTRIES (else ATREX_ERR_TOO_LARGE; the scratch
+ * size query then returns 0).  Too little scratch gives ATREX_ERR_NOMEM.  Input and output must
+ * not overlap.  Both synchronise `stream` and run on the device that holds d_entries. */
+#define ATREX_RELEASE_MAX_ENTRIES (1u << 28)
+uint64_t atrex_release_scratch_bytes(uint64_t n);
+
+/* d_out[0..n) = the entries ordered by packed key ascending (phase, then operator, then shape):
+ * a canonical order for a stored artefact, independent of table geometry and sharding.  Entries
+ * with equal keys (not produced by this library) keep their input order. */
+int atrex_entries_sort_by_key(const atrex_entry_t* d_entries, uint64_t n, atrex_entry_t* d_out,
+                              void* d_scratch, uint64_t scratch_bytes, void* stream);
+
+typedef struct {
+    uint64_t n_phase;                  /* entries of the phase                                   */
+    uint64_t n_keep;                   /* coverage cut: length of the shortest sufficient prefix */
+    uint64_t total_lo, total_hi;       /* T: sum of the phase's weighted times                   */
+    uint64_t covered_lo, covered_hi;   /* weighted time of the first n_keep ranked entries       */
+} atrex_rank_result_t;
+
+/* The entries of `phase` ranked by weighted time descending (exact 128-bit compare), equal times
+ * by key ascending -- the order of atrex_agg_topk, for the whole phase.
+ *   d_ranked, d_cum_share   DEVICE, capacity out_cap each (may be NULL with out_cap 0): the first
+ *                           min(n_phase, out_cap) ranked entries, and beside each its running
+ *                           share cum[i] = fl(fl(wt_0 + ... + wt_i) / fl(T)).  The running sum is an
+ *                           exact integer, rounded once per row, so the column is bit-reproducible and
+ *                           ends at exactly 1.0; T = 0 gives +0.0.
+ *   coverage_ppm            target share in millionths (<= 10^6).  n_keep is the smallest k with
+ *                           10^6 * (wt_0 + ... + wt_{k-1}) >= coverage_ppm * T in integers: the hot set
+ *                           that covers the target.  0 when coverage_ppm = 0 or T = 0; entries of
+ *                           weight zero are never needed.
+ *   h_result                HOST.
+ * T is computed from the entries passed in (it must be below 2^108, else ATREX_ERR_TOO_LARGE), so the
+ * list has to hold the whole phase for the shares to be Eq. 3's. */
+int atrex_entries_rank(const atrex_entry_t* d_entries, uint64_t n, uint32_t phase, uint32_t coverage_ppm,
+                       atrex_entry_t* d_ranked, double* d_cum_share, uint64_t out_cap,
+                       atrex_rank_result_t* h_result, void* d_scratch, uint64_t scratch_bytes, void* stream);
+
 /* Ranked top-k over an array of entries, for callers that cannot allocate device memory.
  *
  * (The paper has no counterpart to this call; it exists for deployment reasons only.)

@@ -4,5 +4,6 @@ behind a C ABI (``include/atrex_agg.h``).  This package is the thin Python bindi
 """
 from .binding import *  # noqa: F401,F403
 from .binding import (Aggregator, AtrexError, make_peaks, topk_entries_static, score_aggregate, OperatorWeights,
+                      sort_entries_by_key, rank_entries,
                       lib, LIB_PATH,  # noqa: F401
                       EXPORTED_SYMBOLS)

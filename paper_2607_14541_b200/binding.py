@@ -28,6 +28,7 @@ ATREX_ERR_TIMEOUT = -5
 ATREX_ERR_STATE = -6
 ATREX_ERR_NOMEM = -7
 ATREX_ERR_TOO_LARGE = -8
+ATREX_RELEASE_MAX_ENTRIES = 1 << 28
 ATREX_STATIC_TOPK_MAX_ENTRIES = 65536
 
 RECORD_DTYPE = np.dtype([("app_id", "<u4"), ("op_id", "<u2"), ("phase", "u1"), ("pad", "u1"),
@@ -42,7 +43,8 @@ EXPORTED_SYMBOLS = [
     "atrex_agg_reset", "atrex_agg_destroy", "atrex_strerror", "atrex_agg_last_cuda_error",
     "atrex_agg_launch_count", "atrex_topk_entries_static", "atrex_agg_hot_directory",
     "atrex_agg_finalize_with_totals", "atrex_score_aggregate", "atrex_eq3_create", "atrex_eq3_ingest",
-    "atrex_eq3_finalize", "atrex_eq3_reset", "atrex_eq3_destroy",
+    "atrex_eq3_finalize", "atrex_eq3_reset", "atrex_eq3_destroy", "atrex_release_scratch_bytes",
+    "atrex_entries_sort_by_key", "atrex_entries_rank",
 ]
 
 
@@ -54,6 +56,11 @@ class atrex_agg_config_t(C.Structure):
 
 class atrex_hw_peaks_t(C.Structure):
     _fields_ = [("peak_bw", C.c_double), ("peak_flops", C.c_double * ATREX_MAX_DTYPES)]
+
+
+class atrex_rank_result_t(C.Structure):
+    _fields_ = [("n_phase", C.c_uint64), ("n_keep", C.c_uint64), ("total_lo", C.c_uint64), ("total_hi", C.c_uint64),
+                ("covered_lo", C.c_uint64), ("covered_hi", C.c_uint64)]
 
 
 class atrex_stats_t(C.Structure):
@@ -99,6 +106,10 @@ def _load():
     L.atrex_eq3_destroy.restype = None
     L.atrex_score_aggregate.argtypes = [vp, vp, u64, vp, vp, u64, vp, u32, vp, vp, vp, vp]
     L.atrex_topk_entries_static.argtypes = [vp, u64, u32, u32, vp, C.POINTER(u32), vp]
+    L.atrex_release_scratch_bytes.restype = u64
+    L.atrex_release_scratch_bytes.argtypes = [u64]
+    L.atrex_entries_sort_by_key.argtypes = [vp, u64, vp, vp, u64, vp]
+    L.atrex_entries_rank.argtypes = [vp, u64, u32, u32, vp, vp, u64, C.POINTER(atrex_rank_result_t), vp, u64, vp]
     return L
 
 
@@ -128,6 +139,9 @@ atrex_eq3_ingest = lib.atrex_eq3_ingest
 atrex_eq3_finalize = lib.atrex_eq3_finalize
 atrex_eq3_reset = lib.atrex_eq3_reset
 atrex_eq3_destroy = lib.atrex_eq3_destroy
+atrex_release_scratch_bytes = lib.atrex_release_scratch_bytes
+atrex_entries_sort_by_key = lib.atrex_entries_sort_by_key
+atrex_entries_rank = lib.atrex_entries_rank
 
 
 class AtrexError(RuntimeError):
@@ -227,6 +241,55 @@ def topk_entries_static(entries, n: int, phase: int, k: int, out, stream=None) -
     if rc != ATREX_OK:
         raise AtrexError(rc, "atrex_topk_entries_static")
     return int(n_out.value)
+
+
+def _stream_ptr(stream):
+    return None if stream is None else (stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _release_scratch(entries, n: int):
+    import torch
+    nbytes = atrex_release_scratch_bytes(int(n))
+    if nbytes == 0:
+        raise AtrexError(ATREX_ERR_TOO_LARGE, "atrex_release_scratch_bytes")
+    buf = torch.empty(nbytes + 256, dtype=torch.uint8, device=entries.device)
+    return buf, (buf.data_ptr() + 255) // 256 * 256, nbytes
+
+
+def sort_entries_by_key(entries, n: int, stream=None):
+    """The ``n`` entries of the CUDA byte tensor ``entries`` in packed-key order (a new CUDA tensor)."""
+    import torch
+    out = torch.empty(max(int(n), 1) * 48, dtype=torch.uint8, device=entries.device)
+    if n:
+        buf, base, nbytes = _release_scratch(entries, n)
+        rc = atrex_entries_sort_by_key(entries.data_ptr(), int(n), out.data_ptr(), base, nbytes, _stream_ptr(stream))
+        if rc != ATREX_OK:
+            raise AtrexError(rc, "atrex_entries_sort_by_key")
+    return out[: int(n) * 48]
+
+
+def rank_entries(entries, n: int, phase: int, coverage_ppm: int = 0, out_cap=None, stream=None):
+    """Ranked entries of one phase with their running share and the coverage cut.
+
+    Returns (ranked CUDA byte tensor, cum-share CUDA float64 tensor, dict with n_phase, n_keep,
+    total, covered); the two tensors hold min(n_phase, out_cap) rows."""
+    import torch
+    cap = int(n) if out_cap is None else int(out_cap)
+    ranked = torch.empty(max(cap, 1) * 48, dtype=torch.uint8, device=entries.device)
+    cum = torch.empty(max(cap, 1), dtype=torch.float64, device=entries.device)
+    res = atrex_rank_result_t()
+    if n:
+        buf, base, nbytes = _release_scratch(entries, n)
+        rc = atrex_entries_rank(entries.data_ptr(), int(n), int(phase), int(coverage_ppm),
+                                ranked.data_ptr() if cap else None, cum.data_ptr() if cap else None, cap,
+                                C.byref(res), base, nbytes, _stream_ptr(stream))
+        if rc != ATREX_OK:
+            raise AtrexError(rc, "atrex_entries_rank")
+    m = min(int(res.n_phase), cap)
+    return ranked[: m * 48], cum[:m], {
+        "n_phase": int(res.n_phase), "n_keep": int(res.n_keep),
+        "total": int(res.total_lo) | (int(res.total_hi) << 64),
+        "covered": int(res.covered_lo) | (int(res.covered_hi) << 64)}
 
 
 class Aggregator:
