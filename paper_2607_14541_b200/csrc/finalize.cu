@@ -46,15 +46,26 @@ __global__ void __launch_bounds__(TOT_THREADS) totals_kernel(TableRef tab, ull n
     for (int p = 0; p < ATREX_MAX_PHASES; ++p) {
         s_lo[p][t] = 0; s_hi[p][t] = 0; s_cnt[p][t] = 0; s_nk[p][t] = 0;
     }
-    for (ull i = (ull)blockIdx.x * blockDim.x + t; i < n_slots; i += (ull)gridDim.x * blockDim.x) {
-        SlotView v = load_slot(tab, i);
-        if (!v.live) continue;
-        int p = (int)(v.key >> 48) & (ATREX_MAX_PHASES - 1);
-        ull o = s_lo[p][t], n = o + v.lo;
-        s_lo[p][t] = n;
-        s_hi[p][t] += v.hi + (n < o ? 1ull : 0ull);
-        s_cnt[p][t] += v.count;
-        s_nk[p][t] += 1;
+    // four slots per thread in flight: all key loads first, then the values of the live ones
+    constexpr int ILP = 4;
+    const ull stride = (ull)gridDim.x * blockDim.x;
+    for (ull i0 = (ull)blockIdx.x * blockDim.x + t; i0 < n_slots; i0 += stride * ILP) {
+        ull sk[ILP];
+        ulonglong2 x[ILP];
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) sk[u] = i0 + u * stride < n_slots ? tab.keys[i0 + u * stride] : 0ull;
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) x[u] = sk[u] != 0 ? tab.vals[i0 + u * stride] : make_ulonglong2(0, 0);
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) {
+            if (sk[u] == 0) continue;
+            const int p = (int)(~sk[u] >> 48) & (ATREX_MAX_PHASES - 1);
+            const ull o = s_lo[p][t], n = o + x[u].x;
+            s_lo[p][t] = n;
+            s_hi[p][t] += (x[u].y >> HI_SHIFT) + (n < o ? 1ull : 0ull);
+            s_cnt[p][t] += x[u].y & COUNT_MASK;
+            s_nk[p][t] += 1;
+        }
     }
     __syncthreads();
     if (t < ATREX_MAX_PHASES) {
@@ -127,45 +138,57 @@ __device__ __forceinline__ void load_phase_totals(const Control* ctl, double* dT
     __syncthreads();
 }
 
-// Four slots per thread per round: their table loads and work-table probes are independent, so
-// the dependent-load latency of the probes overlaps.
+// Each warp looks at 128 slots per round (four coalesced rows), queues the live ones in shared
+// memory and then works through the queue with all lanes busy: at a table load of a third, the
+// divisions and the work-table probe run on full warps instead of one lane in three.
 constexpr int EMIT_ILP = 4;
+constexpr int EMIT_WARPS = FIN_THREADS / 32;
 
 __global__ void __launch_bounds__(FIN_THREADS) emit_kernel(FinalizeParams p) {
     __shared__ double dT[ATREX_MAX_PHASES];
     __shared__ bool zeroT[ATREX_MAX_PHASES];
+    __shared__ ull q_key[EMIT_WARPS][32 * EMIT_ILP];
+    __shared__ ulonglong2 q_val[EMIT_WARPS][32 * EMIT_ILP];
     load_phase_totals(p.ctl, dT, zeroT);
-    const unsigned lane = threadIdx.x & 31u;
+    const unsigned lane = threadIdx.x & 31u, w = threadIdx.x >> 5;
     const ull stride = (ull)gridDim.x * blockDim.x;
     const ull rounds = (p.n_slots + stride * EMIT_ILP - 1) / (stride * EMIT_ILP);  // uniform: warps stay converged
     for (ull r = 0; r < rounds; ++r) {
-        SlotView v[EMIT_ILP];
-        unsigned live[EMIT_ILP];
-        int total = 0;
+        ull sk[EMIT_ILP];
 #pragma unroll
         for (int u = 0; u < EMIT_ILP; ++u) {
-            ull i = (r * EMIT_ILP + u) * stride + (ull)blockIdx.x * blockDim.x + threadIdx.x;
-            v[u].live = false;
-            if (i < p.n_slots) v[u] = load_slot(p.t, i);
-            live[u] = __ballot_sync(0xFFFFFFFFu, v[u].live);
-            total += __popc(live[u]);
+            const ull i = (r * EMIT_ILP + u) * stride + (ull)blockIdx.x * blockDim.x + threadIdx.x;
+            sk[u] = i < p.n_slots ? p.t.keys[i] : 0ull;
+        }
+        uint32_t total = 0;
+#pragma unroll
+        for (int u = 0; u < EMIT_ILP; ++u) {
+            const unsigned live = __ballot_sync(0xFFFFFFFFu, sk[u] != 0);
+            if (sk[u] != 0) {
+                const ull i = (r * EMIT_ILP + u) * stride + (ull)blockIdx.x * blockDim.x + threadIdx.x;
+                const uint32_t at = total + __popc(live & ((1u << lane) - 1u));
+                q_key[w][at] = ~sk[u];
+                q_val[w][at] = p.t.vals[i];
+            }
+            total += __popc(live);
         }
         if (total == 0) continue;
         ull base = 0;
         if (lane == 0) base = atomicAdd(&p.ctl->n_out, (ull)total);
         base = __shfl_sync(0xFFFFFFFFu, base, 0);
-        atrex_entry_t e[EMIT_ILP];
-#pragma unroll
-        for (int u = 0; u < EMIT_ILP; ++u)
-            if (v[u].live) e[u] = make_entry(v[u], dT, zeroT, p);
-#pragma unroll
-        for (int u = 0; u < EMIT_ILP; ++u) {
-            if (v[u].live) {
-                ull pos = base + __popc(live[u] & ((1u << lane) - 1u));
-                if (pos < p.out_cap) store_entry(p.out + pos, e[u]);
-            }
-            base += __popc(live[u]);
+        __syncwarp();
+        for (uint32_t j = lane; j < total; j += 32) {
+            SlotView v;
+            const ulonglong2 x = q_val[w][j];
+            v.key = q_key[w][j];
+            v.live = true;
+            v.lo = x.x;
+            v.count = x.y & COUNT_MASK;
+            v.hi = x.y >> HI_SHIFT;
+            const ull pos = base + j;
+            if (pos < p.out_cap) store_entry(p.out + pos, make_entry(v, dT, zeroT, p));
         }
+        __syncwarp();  // the queue is refilled in the next round
     }
 }
 
