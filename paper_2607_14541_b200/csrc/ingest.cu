@@ -412,6 +412,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     uint32_t* s_cnt = s_a1 + C;
     const uint32_t a_keys = smem_addr(s_keys), a_a0 = smem_addr(s_a0), a_a1 = smem_addr(s_a1), a_cnt = smem_addr(s_cnt);
     __shared__ uint32_t s_total;
+    __shared__ unsigned char s_owner[INGEST_THREADS / 32][32];  // per warp: who owns queue position t
     const uint32_t n_parts = 1u << q.t.lp;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
     // the spill buffers are drained lazily: unless forced, only when the scatter launch just
@@ -463,44 +464,85 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                     slot[u] = local_of(hash32(ent.x), (uint32_t)(ent.x >> 48), C) & ~1u;  // probe sequence starts at an even slot
                     searching[u] = ok[u];
                 }
-                // warp-convergent probe of all four entries, two slots per 16-byte load
-                uint32_t steps = 0;
-                while (__any_sync(0xFFFFFFFFu, searching[0] | searching[1] | searching[2] | searching[3])) {
+                // First look, straight-line for all four entries: most keys sit in the first pair
+                // of slots of their probe sequence.
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const ulonglong2 kk = lds_v2u64(a_keys + slot[u] * 8);
+                    const bool hit1 = kk.y == skey[u];
+                    if (hit1) slot[u] += 1;
+                    if (kk.x == skey[u] || hit1) searching[u] = false;
+                }
+                // The rest (new keys, collisions) is a minority scattered over the four rounds:
+                // hand the pending entries out one per lane, so that the general probe loop runs
+                // once per warp instead of once per round.  Each pending entry's owner publishes
+                // (round, lane) at the entry's queue position; lane t serves position t.
+                while (true) {
+                    uint32_t pend[4], before[4], total = 0;
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        if (!searching[u]) continue;
-                        const ulonglong2 kk = lds_v2u64(a_keys + slot[u] * 8);
-                        if (kk.x == skey[u]) {
-                            searching[u] = false;
-                        } else if (kk.x == 0) {
-                            ull old = atoms_cas64(a_keys + slot[u] * 8, 0ull, skey[u]);  // lost races re-read the pair
-                            if (old == 0) reds_or(a_cnt + slot[u] * 4, NEW_KEY_FLAG);
-                            if (old == 0 || old == skey[u]) searching[u] = false;
-                        } else if (kk.y == skey[u]) {
-                            slot[u] += 1;
-                            searching[u] = false;
-                        } else if (kk.y == 0) {
-                            ull old = atoms_cas64(a_keys + slot[u] * 8 + 8, 0ull, skey[u]);
-                            if (old == 0) reds_or(a_cnt + slot[u] * 4 + 4, NEW_KEY_FLAG);
-                            if (old == 0 || old == skey[u]) {
-                                slot[u] += 1;
-                                searching[u] = false;
-                            }
-                        } else {
-                            slot[u] = (slot[u] + 2 >= C) ? 0u : slot[u] + 2;
+                        pend[u] = __ballot_sync(0xFFFFFFFFu, searching[u]);
+                        before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
+                        total += __popc(pend[u]);
+                    }
+                    if (total == 0) break;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (searching[u] && before[u] < 32) s_owner[warp][before[u]] = (unsigned char)((u << 5) | lane);
+                    __syncwarp();
+                    const bool serving = lane < total;
+                    const uint32_t code = serving ? s_owner[warp][lane] : lane;
+                    const uint32_t src = code & 31u, su = code >> 5;
+                    ull key_s = 0;
+                    uint32_t slot_s = 0;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const ull k = __shfl_sync(0xFFFFFFFFu, skey[u], src);
+                        const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u], src);
+                        if (su == (uint32_t)u) {
+                            key_s = k;
+                            slot_s = sl;
                         }
                     }
-                    if (++steps > 2 * C) {  // partition full (bounded; counts lost races too)
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            if (searching[u]) {
-                                searching[u] = false;
-                                ok[u] = false;
+                    bool busy = serving;
+                    uint32_t steps = 0;
+                    while (__any_sync(0xFFFFFFFFu, busy)) {
+                        if (busy) {
+                            const ulonglong2 kk = lds_v2u64(a_keys + slot_s * 8);
+                            const bool hit1 = kk.y == key_s;
+                            if (kk.x == key_s || hit1) {
+                                slot_s += hit1 ? 1u : 0u;
+                                busy = false;
+                            } else if (kk.x == 0 || kk.y == 0) {
+                                // claim the first empty slot of the pair; a lost race re-reads the pair
+                                const uint32_t at = slot_s + (kk.x == 0 ? 0u : 1u);
+                                const ull old = atoms_cas64(a_keys + at * 8, 0ull, key_s);
+                                if (old == 0) reds_or(a_cnt + at * 4, NEW_KEY_FLAG);
+                                if (old == 0 || old == key_s) {
+                                    slot_s = at;
+                                    busy = false;
+                                }
+                            } else {
+                                slot_s = (slot_s + 2 >= C) ? 0u : slot_s + 2;
+                            }
+                            if (busy && ++steps > 2 * C) {  // partition full (bounded; counts lost races too)
+                                busy = false;
+                                slot_s = 0xFFFFFFFFu;
                                 atomicOr(&q.t.ctl->status, ST_TABLE_FULL);
                                 atomicAdd(&q.t.ctl->n_dropped, 1ull);
                             }
                         }
                     }
+                    // results go back to the owners
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const uint32_t found = __shfl_sync(0xFFFFFFFFu, slot_s, before[u] & 31u);
+                        if (searching[u] && before[u] < 32) {
+                            searching[u] = false;
+                            if (found == 0xFFFFFFFFu) ok[u] = false; else slot[u] = found;
+                        }
+                    }
+                    __syncwarp();  // the queue is rewritten in the next round
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -728,7 +770,7 @@ cudaError_t ingest_prepare() {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(scatter_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(partition_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
+    e = cudaFuncSetAttribute(partition_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 2048);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(hot_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM);
 }
