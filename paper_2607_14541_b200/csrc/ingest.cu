@@ -97,12 +97,17 @@ __device__ __forceinline__ ull atoms_cas64(uint32_t a, ull expected, ull desired
     return o;
 }
 
-// Shared-window byte addresses of the scatter pass's arrays.
+// Shared-window byte addresses of the scatter pass's arrays.  A directory slot is split over three
+// arrays: the key's low word (the shape) as a 32-bit tag, so that one 16-byte load compares a whole
+// 4-slot bucket (the shared-memory data pipe, not instruction issue, is what this kernel runs out of:
+// a bucket of full 8-byte keys costs twice the wavefronts); the key's high word (phase, operator), read
+// only to confirm a tag match; and the accumulators.
 struct SmemDir {
-    uint32_t keys;    // ull[slots], ~key, 0 = empty
     uint32_t a0;      // u32[slots] this launch's weighted time of the slot: bits 0..31 ...
     uint32_t a1;      // u32[slots] ... and bits 32.. (carries of a0 are added here by the adder)
     uint32_t cnt;     // u32[slots] this launch's record count of the slot
+    uint32_t tag;     // u32[slots] shape_id of the slot's key (any value in an empty slot)
+    uint32_t khi;     // u32[slots] phase << 16 | op_id of the slot's key, 0xFFFFFFFF = empty
     uint32_t cursor;  // u32[P] entries appended to this CTA's buffer of each partition
     uint32_t appw;    // u32[n_apps] card-hour weights, when they fit in shared memory ...
     const uint32_t* appw_g;  // ... else they are read from global memory
@@ -144,7 +149,8 @@ __device__ __forceinline__ void dir_add(const SmemDir& d, uint32_t slot, ull v, 
                                         uint32_t h) {
     if (limbs_add(d.a0 + slot * 4, d.a1 + slot * 4, d.cnt + slot * 4, v, count)) {
         ull hi, lo = limbs_drain(d.a0 + slot * 4, d.a1 + slot * 4, &hi);
-        table_accumulate(t, ~lds_u64(d.keys + slot * 8), h, lo, hi, 0);
+        const ull key = ((ull)lds_u32(d.khi + slot * 4) << 32) | lds_u32(d.tag + slot * 4);
+        table_accumulate(t, key, h, lo, hi, 0);
     }
 }
 
@@ -179,12 +185,17 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
         uint32_t slot[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            uint32_t b = dir_bucket(h[r], khi[r] >> 16, d.mult, p.hot_buckets) * DIR_WAYS;
-            const ulonglong2 k01 = lds_v2u64(d.keys + b * 8);
-            const ulonglong2 k23 = lds_v2u64(d.keys + b * 8 + 16);
-            const ull skey = ~(((ull)khi[r] << 32) | w[r][2]);
-            uint32_t way = k01.x == skey ? 0u : (k01.y == skey ? 1u : (k23.x == skey ? 2u : (k23.y == skey ? 3u : DIR_WAYS)));
-            slot[r] = (!todo[r] || way == DIR_WAYS) ? NO_SLOT : b + way;
+            const uint32_t b = dir_bucket(h[r], khi[r] >> 16, d.mult, p.hot_buckets) * DIR_WAYS;
+            uint4 t4;
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(t4.x), "=r"(t4.y), "=r"(t4.z), "=r"(t4.w)
+                         : "r"(d.tag + b * 4));
+            const uint32_t shape = w[r][2];
+            const uint32_t way = t4.x == shape ? 0u : (t4.y == shape ? 1u : (t4.z == shape ? 2u : (t4.w == shape ? 3u : DIR_WAYS)));
+            // a tag match is confirmed against the key's high word; a bucket that holds the same shape
+            // twice (under two operators) may send the second one to the spill path: slower, still exact
+            const bool hit = todo[r] && way != DIR_WAYS && lds_u32(d.khi + (b + (way & 3u)) * 4) == khi[r];
+            slot[r] = hit ? b + way : NO_SLOT;
         }
         if (DEDUPE) {
             // one key dominates the trace: combine the lanes that share the first hitting lane's slot
@@ -315,13 +326,15 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // carve shared memory: directory (keys, limbs, counts), spill cursors, card-hour weights
     unsigned char* sp = smem_raw;
-    ull* g_keys = reinterpret_cast<ull*>(sp);
-    sp += HOT ? (size_t)p.hot_slots * 8 : 0;
     uint32_t* g_a0 = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
     uint32_t* g_a1 = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
     uint32_t* g_cnt = reinterpret_cast<uint32_t*>(sp);
+    sp += HOT ? (size_t)p.hot_slots * 4 : 0;
+    uint32_t* g_tag = reinterpret_cast<uint32_t*>(sp);
+    sp += HOT ? (size_t)p.hot_slots * 4 : 0;
+    uint32_t* g_khi = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
     const uint32_t n_parts = 1u << p.t.lp;
     uint32_t* g_cursor = reinterpret_cast<uint32_t*>(sp);
@@ -329,10 +342,11 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     uint32_t* g_appw = reinterpret_cast<uint32_t*>(sp);
 
     SmemDir d;
-    d.keys = smem_addr(g_keys);
     d.a0 = smem_addr(g_a0);
     d.a1 = smem_addr(g_a1);
     d.cnt = smem_addr(g_cnt);
+    d.tag = smem_addr(g_tag);
+    d.khi = smem_addr(g_khi);
     d.cursor = smem_addr(g_cursor);
     d.appw = smem_addr(g_appw);
     d.appw_g = p.app_w;
@@ -345,7 +359,9 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
         for (uint32_t i = threadIdx.x; i < p.n_apps; i += blockDim.x) g_appw[i] = p.app_w[i];
     if (HOT) {
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
-            g_keys[i] = p.hot_keys[i];
+            const ull image = p.hot_keys[i];  // ~key, 0 = empty
+            g_tag[i] = (uint32_t)~image;
+            g_khi[i] = image ? (uint32_t)(~image >> 32) : 0xFFFFFFFFu;
             g_a0[i] = 0;
             g_a1[i] = 0;
             g_cnt[i] = 0;
@@ -388,9 +404,9 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     }
     if (HOT) {
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
-            uint32_t c = g_cnt[i], lo = g_a0[i], hi = g_a1[i];
+            const uint32_t c = g_cnt[i], lo = g_a0[i], hi = g_a1[i];
             if ((c | lo | hi) != 0) {
-                ull key = ~g_keys[i];
+                const ull key = ((ull)g_khi[i] << 32) | g_tag[i];
                 table_accumulate(p.t, key, hash32(key), (ull)lo | ((ull)hi << 32), 0, (ull)c);
             }
         }
