@@ -74,9 +74,10 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     L->n_slots = (ull)L->C << L->lp;
     L->n_groups = (uint32_t)n_sms;
     L->sub_launch = c->max_keys >= (1ull << 21) ? (1ull << 27) : (c->max_keys >= (1ull << 16) ? (1ull << 25) : (1ull << 24));
-    // room for 3.5 launches' worth of entries if every record spilled: three launches can then
-    // accumulate before a drain, with slack for uneven partitions
-    ull per_buf = (L->sub_launch * 7 / 2) / (((ull)n_sms) << L->lp);
+    // room for 4.5 launches' worth of entries if every record spilled; a drain is requested when a
+    // buffer passes 3/4 of that, which leaves more than one full launch of headroom.  At the bench
+    // workload (half of the records spill) four launches accumulate between drains.
+    ull per_buf = (L->sub_launch * 9 / 2) / (((ull)n_sms) << L->lp);
     if (per_buf < 64) per_buf = 64;
     L->cap = (uint32_t)((per_buf + 7) / 8 * 8);
     // work table: same partitions as the key table, 1.5 slots per row plus slack for uneven partitions
@@ -338,7 +339,7 @@ int atrex_agg_set_work_table(atrex_agg_t* h, const atrex_work_t* rows, uint64_t 
 }
 
 // Partition pass over the spill buffers.  Unforced, the kernel exits at once unless the scatter
-// launch just before it saw a buffer more than 5/8 full; forced (before results are read), it
+// launch just before it saw a buffer more than 3/4 full; forced (before results are read), it
 // drains whatever is there.
 static int drain_spill(atrex_agg* h, bool force, cudaStream_t s) {
     if (force && !h->spill_pending) return ATREX_OK;
@@ -403,7 +404,7 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
     const ull pairs_per_cta_iter = 2048;
     ull want = (p.n_pairs + pairs_per_cta_iter - 1) / pairs_per_cta_iter;
     int grid = (int)(want < 1 ? 1 : (want > (ull)h->n_sms ? (ull)h->n_sms : want));
-    p.drain_above = h->L.cap / 8 * 5;
+    p.drain_above = h->L.cap / 4 * 3;
     p.seq = ++h->scatter_seq;
     CU(h, launch_scatter(p, h->hot_ready, grid, s));
     h->spill_pending = true;
