@@ -454,6 +454,10 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
             s_a1[i] = 0;
             s_cnt[i] = 0;
         }
+        {   // the accumulators of this partition are read back at the end: start them towards L2 now
+            const unsigned char* vb = reinterpret_cast<const unsigned char*>(q.t.vals + base);
+            for (uint32_t off = threadIdx.x * 128u; off < C * 16u; off += blockDim.x * 128u) prefetch_l2(vb + off);
+        }
         __syncthreads();
 
         for (uint32_t g = warp; g < q.n_used; g += n_warps) {
@@ -589,15 +593,33 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 }
             }
         }
-        for (uint32_t i = threadIdx.x; i < C; i += blockDim.x) {
-            uint32_t c = s_cnt[i];
-            if (c == 0) continue;
-            ull* vp = reinterpret_cast<ull*>(q.t.vals + base + i);
-            ull lo = ld_relaxed(vp), cnthi = ld_relaxed(vp + 1);
-            ull nlo = lo + ((ull)s_a0[i] | ((ull)s_a1[i] << 32));
-            cnthi += (ull)(c & ~NEW_KEY_FLAG) + ((nlo < lo ? 1ull : 0ull) << HI_SHIFT);
-            *reinterpret_cast<ulonglong2*>(vp) = make_ulonglong2(nlo, cnthi);
-            if (c & NEW_KEY_FLAG) q.t.keys[base + i] = s_keys[i];
+        // read-modify-write of the touched slots, four per thread in flight (the loads miss L1 by
+        // design and mostly come from L2, where the prefetch at the start of the partition put them)
+        for (uint32_t i0 = threadIdx.x; i0 < C; i0 += 4 * blockDim.x) {
+            uint32_t c[4];
+            ulonglong2 old[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t i = i0 + u * blockDim.x;
+                c[u] = i < C ? s_cnt[i] : 0u;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                old[u] = make_ulonglong2(0, 0);
+                if (c[u]) {
+                    const ull* vp = reinterpret_cast<const ull*>(q.t.vals + base + i0 + u * blockDim.x);
+                    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(old[u].x), "=l"(old[u].y) : "l"(vp));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (c[u] == 0) continue;
+                const uint32_t i = i0 + u * blockDim.x;
+                const ull nlo = old[u].x + ((ull)s_a0[i] | ((ull)s_a1[i] << 32));
+                const ull cnthi = old[u].y + (ull)(c[u] & ~NEW_KEY_FLAG) + ((nlo < old[u].x ? 1ull : 0ull) << HI_SHIFT);
+                q.t.vals[base + i] = make_ulonglong2(nlo, cnthi);
+                if (c[u] & NEW_KEY_FLAG) q.t.keys[base + i] = s_keys[i];
+            }
         }
         // this partition's buffers are empty again
         for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) q.spill_cnt[((ull)g << q.t.lp) + part] = 0;
