@@ -709,10 +709,18 @@ __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
     for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) p.hot_keys[i] = 0;
     if (threadIdx.x == 0) s_inserted = s_max = s_n = 0;
     __syncthreads();
-    for (uint32_t i = threadIdx.x; i < n_cand; i += blockDim.x) {
-        uint32_t c = p.cand_cnt[i];
-        if (c != 0) atomicAdd(&hist[min(c, 1023u)], 1u);
-        if (c >= 1023u) atomicMax(&s_max, c);
+    // one CTA walks the candidate table: eight independent loads per thread at a time, or the scan
+    // is a chain of dependent memory round trips
+    constexpr int SCAN_ILP = 8;
+    for (uint32_t i0 = threadIdx.x; i0 < n_cand; i0 += SCAN_ILP * blockDim.x) {
+        uint32_t c[SCAN_ILP];
+#pragma unroll
+        for (int u = 0; u < SCAN_ILP; ++u) c[u] = i0 + u * blockDim.x < n_cand ? p.cand_cnt[i0 + u * blockDim.x] : 0u;
+#pragma unroll
+        for (int u = 0; u < SCAN_ILP; ++u) {
+            if (c[u] != 0) atomicAdd(&hist[min(c[u], 1023u)], 1u);
+            if (c[u] >= 1023u) atomicMax(&s_max, c[u]);
+        }
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -731,13 +739,21 @@ __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
     __syncthreads();
     const uint32_t thr = s_thr;
     // compact the selected candidates into shared memory, then install them class by class
-    for (uint32_t i = threadIdx.x; i < n_cand; i += blockDim.x) {
-        uint32_t c = p.cand_cnt[i];
-        if (c >= thr) {
-            uint32_t at = atomicAdd(&s_n, 1u);
-            if (at < SELECT_MAX) {
-                c_key[at] = p.cand_keys[i];
-                c_cnt[at] = c;
+    for (uint32_t i0 = threadIdx.x; i0 < n_cand; i0 += SCAN_ILP * blockDim.x) {
+        uint32_t c[SCAN_ILP];
+        ull k[SCAN_ILP];
+#pragma unroll
+        for (int u = 0; u < SCAN_ILP; ++u) c[u] = i0 + u * blockDim.x < n_cand ? p.cand_cnt[i0 + u * blockDim.x] : 0u;
+#pragma unroll
+        for (int u = 0; u < SCAN_ILP; ++u) k[u] = c[u] >= thr ? p.cand_keys[i0 + u * blockDim.x] : 0ull;
+#pragma unroll
+        for (int u = 0; u < SCAN_ILP; ++u) {
+            if (c[u] >= thr) {
+                uint32_t at = atomicAdd(&s_n, 1u);
+                if (at < SELECT_MAX) {
+                    c_key[at] = k[u];
+                    c_cnt[at] = c[u];
+                }
             }
         }
     }
