@@ -87,7 +87,7 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     size_t appw_smem = L->appw_in_smem ? (size_t)c->n_apps * 4 : 0;
     size_t fixed = appw_smem + 2048 + ((size_t)4 << L->lp);
     size_t budget = smem_optin > fixed ? smem_optin - fixed : 0;
-    L->hot_slots = (uint32_t)(budget / 20) & ~3u;   // whole 4-slot buckets
+    L->hot_slots = (uint32_t)(budget / 21) & ~15u;  // 21 B per slot in the scatter pass; whole buckets, aligned arrays
     if (c->flags & ATREX_FLAG_NO_HOT_DIRECTORY) L->hot_slots = 0;
     size_t o = 0;
     L->off_ctl = o;            o += round_up(sizeof(Control), ALIGN);

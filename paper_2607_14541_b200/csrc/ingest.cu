@@ -43,8 +43,13 @@ constexpr uint32_t NEW_KEY_FLAG = 0x80000000u;     // partition pass: slot claim
 // as little sampled weight as possible is lost to buckets that more than two hot keys map to.
 // The table hash `h` leaves the phase out, the directory must not: the phases of a hot
 // (operator, shape) are usually all hot and would otherwise fight over one bucket.
+// Directory placement of a key: the high bits of the mixed hash choose the bucket, its low byte is
+// the slot's tag.
+__device__ __forceinline__ uint32_t dir_mix(uint32_t h, uint32_t phase, uint32_t mult) {
+    return (h + phase * 0x9E3779B9u) * mult;
+}
 __device__ __forceinline__ uint32_t dir_bucket(uint32_t h, uint32_t phase, uint32_t mult, uint32_t n_buckets) {
-    return __umulhi((h + phase * 0x9E3779B9u) * mult, n_buckets);
+    return __umulhi(dir_mix(h, phase, mult), n_buckets);
 }
 __device__ __forceinline__ uint32_t dir_bucket_of_key(ull key, uint32_t mult, uint32_t n_buckets) {
     return dir_bucket(hash32(key), (uint32_t)(key >> 48), mult, n_buckets);
@@ -97,17 +102,17 @@ __device__ __forceinline__ ull atoms_cas64(uint32_t a, ull expected, ull desired
     return o;
 }
 
-// Shared-window byte addresses of the scatter pass's arrays.  A directory slot is split over three
-// arrays: the key's low word (the shape) as a 32-bit tag, so that one 16-byte load compares a whole
-// 4-slot bucket (the shared-memory data pipe, not instruction issue, is what this kernel runs out of:
-// a bucket of full 8-byte keys costs twice the wavefronts); the key's high word (phase, operator), read
-// only to confirm a tag match; and the accumulators.
+// Shared-window byte addresses of the scatter pass's arrays.  The shared-memory data pipe, not
+// instruction issue, is what this kernel runs out of, so a directory look-up first reads one 32-bit
+// word per 4-slot bucket -- an 8-bit tag per slot, taken from hash bits the bucket choice does not
+// use -- and only a lane whose tag matches reads the 8-byte key to confirm.  A wrong tag match
+// (1 in 64 look-ups) fails the confirmation and the record takes the spill path: slower, still exact.
 struct SmemDir {
+    uint32_t keys;    // ull[slots] ~key, 0 = empty
+    uint32_t tag;     // u32[buckets] four 8-bit tags
     uint32_t a0;      // u32[slots] this launch's weighted time of the slot: bits 0..31 ...
     uint32_t a1;      // u32[slots] ... and bits 32.. (carries of a0 are added here by the adder)
     uint32_t cnt;     // u32[slots] this launch's record count of the slot
-    uint32_t tag;     // u32[slots] shape_id of the slot's key (any value in an empty slot)
-    uint32_t khi;     // u32[slots] phase << 16 | op_id of the slot's key, 0xFFFFFFFF = empty
     uint32_t cursor;  // u32[P] entries appended to this CTA's buffer of each partition
     uint32_t appw;    // u32[n_apps] card-hour weights, when they fit in shared memory ...
     const uint32_t* appw_g;  // ... else they are read from global memory
@@ -149,8 +154,7 @@ __device__ __forceinline__ void dir_add(const SmemDir& d, uint32_t slot, ull v, 
                                         uint32_t h) {
     if (limbs_add(d.a0 + slot * 4, d.a1 + slot * 4, d.cnt + slot * 4, v, count)) {
         ull hi, lo = limbs_drain(d.a0 + slot * 4, d.a1 + slot * 4, &hi);
-        const ull key = ((ull)lds_u32(d.khi + slot * 4) << 32) | lds_u32(d.tag + slot * 4);
-        table_accumulate(t, key, h, lo, hi, 0);
+        table_accumulate(t, ~lds_u64(d.keys + slot * 8), h, lo, hi, 0);
     }
 }
 
@@ -185,17 +189,13 @@ __device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&
         uint32_t slot[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) {
-            const uint32_t b = dir_bucket(h[r], khi[r] >> 16, d.mult, p.hot_buckets) * DIR_WAYS;
-            uint4 t4;
-            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(t4.x), "=r"(t4.y), "=r"(t4.z), "=r"(t4.w)
-                         : "r"(d.tag + b * 4));
-            const uint32_t shape = w[r][2];
-            const uint32_t way = t4.x == shape ? 0u : (t4.y == shape ? 1u : (t4.z == shape ? 2u : (t4.w == shape ? 3u : DIR_WAYS)));
-            // a tag match is confirmed against the key's high word; a bucket that holds the same shape
-            // twice (under two operators) may send the second one to the spill path: slower, still exact
-            const bool hit = todo[r] && way != DIR_WAYS && lds_u32(d.khi + (b + (way & 3u)) * 4) == khi[r];
-            slot[r] = hit ? b + way : NO_SLOT;
+            const uint32_t x = dir_mix(h[r], khi[r] >> 16, d.mult);
+            const uint32_t b = __umulhi(x, p.hot_buckets);
+            const uint32_t eq = __vcmpeq4(lds_u32(d.tag + b * 4), (x & 0xFFu) * 0x01010101u);  // 0xFF per matching byte
+            const uint32_t at = b * DIR_WAYS + (((uint32_t)__ffs(eq) - 1u) >> 3);
+            const ull skey = ~(((ull)khi[r] << 32) | w[r][2]);
+            const bool hit = todo[r] && eq != 0 && lds_u64(d.keys + at * 8) == skey;
+            slot[r] = hit ? at : NO_SLOT;
         }
         if (DEDUPE) {
             // one key dominates the trace: combine the lanes that share the first hitting lane's slot
@@ -326,16 +326,16 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // carve shared memory: directory (keys, limbs, counts), spill cursors, card-hour weights
     unsigned char* sp = smem_raw;
+    ull* g_keys = reinterpret_cast<ull*>(sp);
+    sp += HOT ? (size_t)p.hot_slots * 8 : 0;
     uint32_t* g_a0 = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
     uint32_t* g_a1 = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
     uint32_t* g_cnt = reinterpret_cast<uint32_t*>(sp);
     sp += HOT ? (size_t)p.hot_slots * 4 : 0;
-    uint32_t* g_tag = reinterpret_cast<uint32_t*>(sp);
-    sp += HOT ? (size_t)p.hot_slots * 4 : 0;
-    uint32_t* g_khi = reinterpret_cast<uint32_t*>(sp);
-    sp += HOT ? (size_t)p.hot_slots * 4 : 0;
+    unsigned char* g_tag = sp;
+    sp += HOT ? (size_t)p.hot_slots : 0;
     const uint32_t n_parts = 1u << p.t.lp;
     uint32_t* g_cursor = reinterpret_cast<uint32_t*>(sp);
     sp += (size_t)n_parts * 4;
@@ -345,8 +345,8 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     d.a0 = smem_addr(g_a0);
     d.a1 = smem_addr(g_a1);
     d.cnt = smem_addr(g_cnt);
+    d.keys = smem_addr(g_keys);
     d.tag = smem_addr(g_tag);
-    d.khi = smem_addr(g_khi);
     d.cursor = smem_addr(g_cursor);
     d.appw = smem_addr(g_appw);
     d.appw_g = p.app_w;
@@ -360,8 +360,8 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
     if (HOT) {
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
             const ull image = p.hot_keys[i];  // ~key, 0 = empty
-            g_tag[i] = (uint32_t)~image;
-            g_khi[i] = image ? (uint32_t)(~image >> 32) : 0xFFFFFFFFu;
+            g_keys[i] = image;
+            g_tag[i] = (unsigned char)(dir_mix(hash32(~image), (uint32_t)(~image >> 48) & 0xFFu, d.mult) & 0xFFu);
             g_a0[i] = 0;
             g_a1[i] = 0;
             g_cnt[i] = 0;
@@ -406,7 +406,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
             const uint32_t c = g_cnt[i], lo = g_a0[i], hi = g_a1[i];
             if ((c | lo | hi) != 0) {
-                const ull key = ((ull)g_khi[i] << 32) | g_tag[i];
+                const ull key = ~g_keys[i];
                 table_accumulate(p.t, key, hash32(key), (ull)lo | ((ull)hi << 32), 0, (ull)c);
             }
         }
@@ -830,7 +830,7 @@ cudaError_t ingest_prepare() {
 }
 
 cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream) {
-    size_t smem = (hot ? (size_t)p.hot_slots * 20 : 0) + ((size_t)4 << p.t.lp) + (p.appw_in_smem ? (size_t)p.n_apps * 4 : 0);
+    size_t smem = (hot ? (size_t)p.hot_slots * 21 : 0) + ((size_t)4 << p.t.lp) + (p.appw_in_smem ? (size_t)p.n_apps * 4 : 0);
     if (hot)
         scatter_kernel<true><<<grid, INGEST_THREADS, smem, stream>>>(p);
     else
