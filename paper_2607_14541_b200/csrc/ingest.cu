@@ -464,13 +464,17 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
             const ull sb = ((ull)g << q.t.lp) + part;
             const uint32_t n_e = q.spill_cnt[sb];
             const ulonglong2* src = reinterpret_cast<const ulonglong2*>(q.spill) + sb * q.cap;
-            if (g + n_warps < q.n_used) {  // short-distance prefetch: this warp's next sub-buffer
+            // Short-distance L2 prefetch, a fixed 4 KB window per warp (a longer reach gets evicted
+            // before use: all warps of all CTAs together must stay well inside L2): the head of this
+            // warp's next sub-buffer now, and inside the loop the lines two batches ahead.
+            if (g + n_warps < q.n_used) {
                 const ull nb = ((ull)(g + n_warps) << q.t.lp) + part;
                 const uint32_t bytes = q.spill_cnt[nb] * 16u;
-                const unsigned char* nsrc = q.spill + nb * q.cap * 16ull;
-                for (uint32_t off = lane * 128u; off < bytes; off += 32u * 128u) prefetch_l2(nsrc + off);
+                if (lane * 128u < bytes) prefetch_l2(q.spill + nb * q.cap * 16ull + lane * 128u);
             }
             for (uint32_t e0 = 0; e0 < n_e; e0 += 128) {
+                if (lane < 16 && (e0 + 256u + lane * 8u) < n_e)
+                    prefetch_l2(reinterpret_cast<const unsigned char*>(src) + (e0 + 256u) * 16u + lane * 128u);
                 ull skey[4], v[4];
                 uint32_t slot[4];
                 bool searching[4], ok[4];
@@ -588,8 +592,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 if (warp < q.n_used) {
                     const ull nb = ((ull)warp << q.t.lp) + next;
                     const uint32_t bytes = q.spill_cnt[nb] * 16u;
-                    const unsigned char* nsrc = q.spill + nb * q.cap * 16ull;
-                    for (uint32_t off = lane * 128u; off < bytes; off += 32u * 128u) prefetch_l2(nsrc + off);
+                    if (lane * 128u < bytes) prefetch_l2(q.spill + nb * q.cap * 16ull + lane * 128u);
                 }
             }
         }
