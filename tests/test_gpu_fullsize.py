@@ -86,3 +86,48 @@ def test_full_size_trace_sampled_keys_and_invariants(index):
         wt_all = ent["wt_hi"].astype(object) * (1 << 64) + ent["wt_lo"].astype(object)
         assert (wt_all == ent["count"].astype(object) * P).all()
         assert int(ent["wt_hi"].max()) > 6000
+
+    # the release artefacts made from this entry list (config 2's three phases and config 3's
+    # 16 M entries exercise every word of the ranking order and several sort tiles per digit)
+    if index in (2, 3):
+        check_release_artefacts(p, agg, spec, ent, st)
+
+
+def _prefix_ints(wt_lo, wt_hi, positions):
+    """Exact inclusive prefix sums of 128-bit values at the given positions: numpy running sums of
+    32-bit pieces (no overflow below 2^32 rows), recombined as Python integers."""
+    mask = np.uint64(0xFFFFFFFF)
+    pieces = [wt_lo & mask, wt_lo >> np.uint64(32), wt_hi & mask, wt_hi >> np.uint64(32)]
+    sums = [np.cumsum(x, dtype=np.uint64) for x in pieces]
+    return [sum(int(s[i]) << (32 * j) for j, s in enumerate(sums)) for i in positions]
+
+
+def check_release_artefacts(p, agg, spec, ent, st):
+    dev_ent, n_ent = agg.finalize(spec.peak_bw, spec.peak_flops)
+    by_key = p.sort_entries_by_key(dev_ent, n_ent).cpu().numpy().view(p.ENTRY_DTYPE)
+    assert by_key.tobytes() == ent[np.argsort(ent["key"], kind="stable")].tobytes()    # keys are unique
+    for ph in range(spec.n_phases):
+        ppm = (900_000, 500_000, 999_999)[ph % 3]
+        ranked, cum, res = p.rank_entries(dev_ent, n_ent, ph, ppm)
+        ranked = ranked.cpu().numpy().view(p.ENTRY_DTYPE)
+        cum = cum.cpu().numpy()
+        sel = ent[(ent["key"] >> np.uint64(48)) == ph]
+        total = st["totals"][ph]
+        assert res["n_phase"] == len(sel) == len(ranked) and res["total"] == total
+        # same entries, in (weighted time descending, key ascending) order
+        assert np.array_equal(np.sort(ranked["key"]), np.sort(sel["key"]))
+        assert ranked[np.argsort(ranked["key"], kind="stable")].tobytes() == sel[np.argsort(sel["key"], kind="stable")].tobytes()
+        hi, lo, key = ranked["wt_hi"], ranked["wt_lo"], ranked["key"]
+        in_order = (hi[:-1] > hi[1:]) | ((hi[:-1] == hi[1:]) & ((lo[:-1] > lo[1:]) | ((lo[:-1] == lo[1:]) & (key[:-1] < key[1:]))))
+        assert in_order.all()
+        assert agg.topk(ph, spec.topk).tobytes() == ranked[: spec.topk].tobytes()
+        # running share at sampled rows, and the cut, against exact integer prefix sums
+        k = res["n_keep"]
+        rows = sorted(set([0, 1, len(ranked) // 3, len(ranked) - 1] + [max(k - 2, 0), max(k - 1, 0), min(k, len(ranked) - 1)]
+                          + list(range(0, len(ranked), max(1, len(ranked) // 200)))))
+        prefix = dict(zip(rows, _prefix_ints(lo, hi, rows)))
+        for r in rows:
+            assert f64_bits(float(cum[r])) == f64_bits(oracle.u128_to_f64(prefix[r]) / oracle.u128_to_f64(total)), (ph, r)
+        assert (np.diff(cum) >= 0).all() and cum[-1] == 1.0
+        assert k >= 1 and prefix[k - 1] * 1_000_000 >= ppm * total and res["covered"] == prefix[k - 1]
+        assert k == 1 or prefix[k - 2] * 1_000_000 < ppm * total
