@@ -156,6 +156,14 @@ struct atrex_agg {
         t.lp = L.lp;
         t.C = L.C;
         t.ctl = ctl;
+        // eight odd primes that do not divide the number of slot pairs
+        uint32_t n = 0;
+        t.strides = 0;
+        for (uint32_t c = 7; n < 8; c += 2) {
+            bool prime = true;
+            for (uint32_t d = 3; d * d <= c; d += 2) prime = prime && (c % d != 0);
+            if (prime && (L.C / 2) % c != 0) t.strides |= (ull)c << (8 * n++);
+        }
         return t;
     }
     WorkRef work_ref() const {

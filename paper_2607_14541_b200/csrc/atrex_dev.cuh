@@ -101,19 +101,30 @@ struct TableRef {
     ull* keys;            // [P * C]
     ulonglong2* vals;     // [P * C] {lo, cnthi}
     uint32_t lp;          // log2(P)
-    uint32_t C;           // slots per partition
+    uint32_t C;           // slots per partition (even)
     Control* ctl;
+    ull strides;          // eight probe strides in slot pairs, one byte each: odd primes that do not divide C / 2
 };
 
 constexpr ull NO_INDEX = ~0ull;
 
 __device__ __forceinline__ uint32_t part_of(uint32_t h, uint32_t lp) { return h >> (32 - lp); }  // lp >= 1
 
-// Start slot inside the partition.  The phase, which the partition choice ignores, is mixed in
-// here so that the phases of one (operator, shape) do not pile up on the same slot.
-// (Probe sequences start at the even slot at or below this one and then visit consecutive slots.)
+// Probe sequence of a key inside its partition (double hashing over slot pairs): it starts at the
+// pair holding local_of() and moves on by one of eight strides chosen by other hash bits; inside a
+// pair the even slot comes first.  The strides are coprime to the number of pairs, so the sequence
+// visits every pair once.  Every prober -- this file's global-memory path and the partition pass's
+// shared-memory path -- follows the same order, and a key sits at the first slot of its sequence
+// that was free when it arrived.  Clusters of linear probing, which at the load factors reached
+// here (up to 0.7) made the slowest of a warp's probes several times the average, do not form.
+// The phase, which the partition choice ignores, is mixed into the start so that the phases of one
+// (operator, shape) do not pile up on the same pair.
 __device__ __forceinline__ uint32_t local_of(uint32_t h, uint32_t phase, uint32_t C) {
     return __umulhi((h ^ (phase * 0x9E3779B9u)) * 0x85EBCA6Bu, C);
+}
+__device__ __forceinline__ uint32_t stride_index(uint32_t h) { return (h >> 3) & 7u; }
+__device__ __forceinline__ uint32_t stride_of(const TableRef& t, uint32_t index) {
+    return (uint32_t)(t.strides >> (8 * index)) & 0xFFu;
 }
 
 // Find (or claim) the slot of `key` directly in HBM.  Returns NO_INDEX when the key's
@@ -123,6 +134,7 @@ __device__ __forceinline__ ull find_or_claim(const TableRef& t, ull key, uint32_
     const ull skey = ~key;
     const ull base = (ull)part_of(h, t.lp) * t.C;
     uint32_t s = local_of(h, (uint32_t)(key >> 48), t.C) & ~1u;
+    const uint32_t advance = 2u * stride_of(t, stride_index(h));
     for (uint32_t probe = 0; probe < t.C; ++probe) {
         ull* kp = t.keys + base + s;
         ull k = ld_relaxed(kp);
@@ -131,7 +143,12 @@ __device__ __forceinline__ ull find_or_claim(const TableRef& t, ull key, uint32_
             ull old = atomicCAS(kp, 0ull, skey);
             if (old == 0 || old == skey) return base + s;
         }
-        s = (s + 1 == t.C) ? 0u : s + 1;
+        if (s & 1u) {  // second slot of the pair done: on to the next pair
+            s = (s & ~1u) + advance;
+            if (s >= t.C) s -= t.C;
+        } else {
+            s |= 1u;
+        }
     }
     return NO_INDEX;
 }

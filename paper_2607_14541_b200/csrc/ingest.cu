@@ -476,7 +476,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 if (lane < 16 && (e0 + 256u + lane * 8u) < n_e)
                     prefetch_l2(reinterpret_cast<const unsigned char*>(src) + (e0 + 256u) * 16u + lane * 128u);
                 ull skey[4], v[4];
-                uint32_t slot[4];
+                uint32_t slot[4], strides = 0;  // strides: each entry's stride index, one byte each
                 bool searching[4], ok[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -485,7 +485,9 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                     ulonglong2 ent = ok[u] ? __ldcs(src + e) : make_ulonglong2(0, 0);
                     skey[u] = ~ent.x;
                     v[u] = ent.y;
-                    slot[u] = local_of(hash32(ent.x), (uint32_t)(ent.x >> 48), C) & ~1u;  // probe sequence starts at an even slot
+                    const uint32_t hh = hash32(ent.x);
+                    slot[u] = local_of(hh, (uint32_t)(ent.x >> 48), C) & ~1u;  // first pair of the probe sequence
+                    strides |= stride_index(hh) << (8 * u);
                     searching[u] = ok[u];
                 }
                 // First look, straight-line for all four entries: most keys sit in the first pair
@@ -522,12 +524,14 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const ull k = __shfl_sync(0xFFFFFFFFu, skey[u], src);
-                        const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u], src);
+                        const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u] | (((strides >> (8 * u)) & 7u) << 16), src);
                         if (su == (uint32_t)u) {
                             key_s = k;
                             slot_s = sl;
                         }
                     }
+                    const uint32_t advance = 2u * stride_of(q.t, slot_s >> 16);
+                    slot_s &= 0xFFFFu;
                     bool busy = serving;
                     uint32_t steps = 0;
                     while (__any_sync(0xFFFFFFFFu, busy)) {
@@ -547,7 +551,8 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                                     busy = false;
                                 }
                             } else {
-                                slot_s = (slot_s + 2 >= C) ? 0u : slot_s + 2;
+                                slot_s += advance;
+                                if (slot_s >= C) slot_s -= C;
                             }
                             if (busy && ++steps > 2 * C) {  // partition full (bounded; counts lost races too)
                                 busy = false;
