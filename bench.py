@@ -31,9 +31,9 @@ if ROOT not in sys.path:
 
 METRIC = "trace records aggregated/sec"
 # DRAM bytes (read + written) per 2^27-record ingest call of this workload, from the ncu captures
-# summarised under profiles/: scatter_kernel 4.41 GB per launch plus
-# the three partition drains of a step (12.15 GB) spread over its eight calls.
-NCU_DRAM_BYTES_PER_INGEST_CALL = 5.93e9
+# summarised under profiles/: scatter_kernel 4.43 GB per launch plus
+# the two real partition drains of a step (11.79 GB) spread over its eight calls.
+NCU_DRAM_BYTES_PER_INGEST_CALL = 5.90e9
 UNIT = "records/s"
 WORKLOAD_INDEX = 3
 RECORD_BYTES = 16
@@ -266,7 +266,8 @@ def run_ours(args):
                     "launch_ms_best": min(ingest_ms), "peak_source": peak_src,
                     "frac_of_nominal_8TBs": achieved / 8000.0,
                     "note": "duration = CUDA events around each ingest call (scatter launch + partition launch, "
-                            "which drains the spill buffers every third call); call 0 of a step also holds the "
+                            "which drains the spill buffers when one passes 3/4 of its capacity: calls 4 and 8 "
+                            "here); call 0 of a step also holds the "
                             "hot-directory build; achieved = 16 B x records / duration"}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True,
