@@ -41,7 +41,7 @@ int log2_of(ull p) {
 }
 
 struct Layout {
-    size_t off_ctl, off_keys, off_vals, off_work, off_appw, off_hot, off_staging[2], off_sel, off_topk_out,
+    size_t off_ctl, off_keys, off_vals, off_work, off_appw, off_hot, off_staging[2], off_sel, off_topk_out, off_hist_all,
         off_spill_cnt, off_spill, off_hot_scratch, total;
     ull n_slots, work_slots;
     uint32_t lp, C;              // partitions = 1 << lp, slots per partition
@@ -98,7 +98,8 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     L->off_hot = o;            o += round_up((size_t)(L->hot_slots ? L->hot_slots : 2) * 8, ALIGN);
     L->off_staging[0] = o;     o += STAGING_BYTES;
     L->off_staging[1] = o;     o += STAGING_BYTES;
-    L->off_sel = o;            o += round_up((size_t)SEL_CAP * 32, ALIGN);
+    L->off_sel = o;            o += round_up((size_t)SEL_CAP * 32 * c->n_phases, ALIGN);   // one region per phase
+    L->off_hist_all = o;       o += round_up((size_t)ATREX_MAX_PHASES * TOPK_BINS * 4, ALIGN);
     L->off_topk_out = o;       o += round_up((size_t)ATREX_MAX_TOPK * sizeof(atrex_entry_t), ALIGN);
     L->off_hot_scratch = o;    o += round_up(HOT_SCRATCH_BYTES, ALIGN);
     L->off_spill_cnt = o;      o += round_up(((size_t)L->n_groups << L->lp) * 4, ALIGN);
@@ -119,6 +120,17 @@ struct DeviceGuard {
 
 }  // namespace
 
+// What one ranking request worked out for every phase, kept until the next finalize: the
+// first-digit histograms (one pass over the table for all phases) and, for the last k asked for,
+// each phase's selection (one more pass for all phases).  A second phase's top-k of the same k then
+// costs no pass over the table at all.
+struct TopkCache {
+    ull hist_gen = 0;                       // finalize generation the histograms belong to (0 = none)
+    ull sel_gen = 0;                        // ... and the selections
+    uint32_t k = 0;                         // k the selections were made for
+    ull total[ATREX_MAX_PHASES] = {};       // candidates collected per phase
+};
+
 struct atrex_agg {
     atrex_agg_config_t cfg;
     Layout L;
@@ -138,6 +150,10 @@ struct atrex_agg {
     ull* sel = nullptr;
     atrex_entry_t* topk_out = nullptr;
     Control* h_ctl = nullptr;  // pinned mirror
+    uint32_t* hist_all = nullptr;     // [ATREX_MAX_PHASES][TOPK_BINS] first-digit histograms of all phases
+    uint32_t* h_hist_all = nullptr;   // pinned mirror
+    TopkCache topk;
+    ull fin_gen = 0;                  // bumped by every successful finalize
     bool hot_ready = false;
     bool finalized = false;
     bool spill_pending = false;   // entries may sit in the spill buffers
@@ -268,12 +284,15 @@ int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out) {
         h->staging[1] = h->ws + L.off_staging[1];
         h->sel = (ull*)(h->ws + L.off_sel);
         h->topk_out = (atrex_entry_t*)(h->ws + L.off_topk_out);
+        h->hist_all = (uint32_t*)(h->ws + L.off_hist_all);
         cudaError_t e = cudaSuccess;
         if (e == cudaSuccess) e = cudaMemset(h->ws + L.off_ctl, 0, L.off_appw - L.off_ctl);  // control, table, work
         if (e == cudaSuccess) e = cudaMemcpy(h->d_appw, cfg->app_weights, (size_t)cfg->n_apps * 4, cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = cudaMemset(h->hot_keys, 0, (size_t)(L.hot_slots ? L.hot_slots : 2) * 8);
         if (e == cudaSuccess) e = cudaMemset(h->spill_cnt, 0, ((size_t)L.n_groups << L.lp) * 4);
         if (e == cudaSuccess) e = cudaHostAlloc((void**)&h->h_ctl, sizeof(Control), cudaHostAllocDefault);
+        if (e == cudaSuccess)
+            e = cudaHostAlloc((void**)&h->h_hist_all, (size_t)ATREX_MAX_PHASES * TOPK_BINS * 4, cudaHostAllocDefault);
         if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
         for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
             e = cudaEventCreateWithFlags(&h->ev_ready[i], cudaEventDisableTiming);
@@ -302,6 +321,7 @@ void atrex_agg_destroy(atrex_agg_t* h) {
     }
     if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
     if (h->h_ctl) cudaFreeHost(h->h_ctl);
+    if (h->h_hist_all) cudaFreeHost(h->h_hist_all);
     if (h->owns_workspace && h->ws) cudaFree(h->ws);
     delete h;
 }
@@ -538,7 +558,60 @@ static int finalize_impl(atrex_agg_t* h, const atrex_hw_peaks_t* peaks, const ui
     rc = device_status_to_error(h->h_ctl);
     if (rc != ATREX_OK) return rc;
     h->finalized = true;
+    h->fin_gen++;
     if (d_out && h->h_ctl->n_out > out_cap) return ATREX_ERR_OUT_TOO_SMALL;
+    return ATREX_OK;
+}
+
+// Radix-select plan of one phase for the best k: fixes leading digits of the ranking composite until
+// the class holding the k-th entry is small enough to sort.  The first digit comes from the cached
+// all-phase histograms; deeper digits (only when more than TOPK_CAND_CAP keys share the leading
+// digits) take one single-phase pass each.
+static int plan_phase(atrex_agg_t* h, uint32_t q, uint32_t k, TopkAllParams* all, ull* total, cudaStream_t s) {
+    const ull n_phase = h->h_ctl->keys_per_phase[q];
+    all->n_prefix_digits[q] = 0;
+    if (n_phase == 0) {
+        *total = 0;
+        return ATREX_OK;
+    }
+    all->active_mask |= 1u << q;
+    if (n_phase <= k) {
+        all->collect_all_mask |= 1u << q;
+        *total = n_phase;
+        return ATREX_OK;
+    }
+    const uint32_t n_digits = (144 - all->shift[q] + 11) / 12;
+    ull need = k, cand = 0;
+    const uint32_t* hist = h->h_hist_all + (size_t)q * TOPK_BINS;
+    while (true) {
+        ull above = 0;
+        int bin = TOPK_BINS - 1;
+        for (; bin > 0; --bin) {
+            if (above + hist[bin] >= need) break;
+            above += hist[bin];
+        }
+        need -= above;
+        cand = hist[bin];
+        all->prefix_digit[q][all->n_prefix_digits[q]++] = (uint16_t)bin;
+        if (cand <= TOPK_CAND_CAP || all->n_prefix_digits[q] == n_digits) break;
+        // next digit of this phase alone
+        TopkParams p;
+        memset(&p, 0, sizeof(p));
+        p.t = h->table_ref();
+        p.n_slots = h->L.n_slots;
+        p.ctl = h->ctl;
+        p.phase = q;
+        p.shift = all->shift[q];
+        p.n_prefix_digits = all->n_prefix_digits[q];
+        memcpy(p.prefix_digit, all->prefix_digit[q], sizeof(p.prefix_digit));
+        CU(h, cudaMemsetAsync(h->ctl->hist, 0, sizeof(h->ctl->hist), s));
+        CU(h, launch_topk_hist(p, h->scan_grid(h->L.n_slots, 256 * 4), s));
+        h->launches++;
+        CU(h, cudaMemcpyAsync(h->h_ctl->hist, h->ctl->hist, sizeof(h->ctl->hist), cudaMemcpyDeviceToHost, s));
+        CU(h, cudaStreamSynchronize(s));
+        hist = h->h_ctl->hist;
+    }
+    *total = (k - need) + cand;
     return ATREX_OK;
 }
 
@@ -549,61 +622,65 @@ int atrex_agg_topk(atrex_agg_t* h, uint32_t phase, uint32_t k, atrex_entry_t* h_
     if (k == 0) return ATREX_OK;
     DeviceGuard guard(h->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
-    const ull n_phase = h->h_ctl->keys_per_phase[phase];
-    if (n_phase == 0) return ATREX_OK;
+    if (h->h_ctl->keys_per_phase[phase] == 0) return ATREX_OK;
+    const uint32_t n_phases = h->cfg.n_phases;
+    TopkCache& cache = h->topk;
 
-    TopkParams p;
-    memset(&p, 0, sizeof(p));
-    p.t = h->table_ref();
-    p.n_slots = h->L.n_slots;
-    p.ctl = h->ctl;
-    p.phase = phase;
-    p.sel = h->sel;
-    p.sel_cap = SEL_CAP;
-    const int grid = h->scan_grid(h->L.n_slots, 256 * 4);
-    ull total;
-    if (n_phase <= k) {
-        p.collect_all = 1;
-        total = n_phase;
-    } else {
-        // most-significant-digit radix select on the ranking composite; digits start at the
-        // highest bit the phase total has (no key's weighted time exceeds it)
-        {
-            ull hi = h->h_ctl->total_hi[phase], lo = h->h_ctl->total_lo[phase];
+    if (cache.sel_gen != h->fin_gen || cache.k != k) {
+        TopkAllParams all;
+        memset(&all, 0, sizeof(all));
+        all.t = h->table_ref();
+        all.n_slots = h->L.n_slots;
+        all.hist = h->hist_all;
+        all.sel = h->sel;
+        all.sel_count = h->ctl->sel_count_all;
+        all.sel_cap = SEL_CAP;
+        // digits start at the highest bit a phase's total has (no key's weighted time exceeds it)
+        for (uint32_t q = 0; q < n_phases; ++q) {
+            ull hi = h->h_ctl->total_hi[q], lo = h->h_ctl->total_lo[q];
             int top_bit = hi ? 64 + (63 - __builtin_clzll(hi)) : (lo ? 63 - __builtin_clzll(lo) : 0);
-            p.shift = (uint32_t)(143 - (top_bit + 56));
+            all.shift[q] = (uint32_t)(143 - (top_bit + 56));
         }
-        const uint32_t n_digits = (144 - p.shift + 11) / 12;
-        ull need = k, cand = 0;
-        uint32_t* hist = h->h_ctl->hist;
-        while (true) {
-            CU(h, cudaMemsetAsync(h->ctl->hist, 0, sizeof(h->ctl->hist), s));
-            CU(h, launch_topk_hist(p, grid, s));
+        if (cache.hist_gen != h->fin_gen) {
+            // first digit of every non-empty phase: one pass over the table
+            for (uint32_t q = 0; q < n_phases; ++q)
+                if (h->h_ctl->keys_per_phase[q] != 0) all.active_mask |= 1u << q;
+            CU(h, cudaMemsetAsync(h->hist_all, 0, (size_t)ATREX_MAX_PHASES * TOPK_BINS * 4, s));
+            CU(h, launch_topk_hist_all(all, h->n_sms, s));
             h->launches++;
-            CU(h, cudaMemcpyAsync(hist, h->ctl->hist, sizeof(h->ctl->hist), cudaMemcpyDeviceToHost, s));
+            CU(h, cudaMemcpyAsync(h->h_hist_all, h->hist_all, (size_t)ATREX_MAX_PHASES * TOPK_BINS * 4,
+                                  cudaMemcpyDeviceToHost, s));
             CU(h, cudaStreamSynchronize(s));
-            ull above = 0;
-            int bin = TOPK_BINS - 1;
-            for (; bin > 0; --bin) {
-                if (above + hist[bin] >= need) break;
-                above += hist[bin];
-            }
-            need -= above;
-            cand = hist[bin];
-            p.prefix_digit[p.n_prefix_digits++] = (uint16_t)bin;
-            if (cand <= TOPK_CAND_CAP || p.n_prefix_digits == n_digits) break;
+            cache.hist_gen = h->fin_gen;
+            all.active_mask = 0;
         }
-        total = (k - need) + cand;
+        for (uint32_t q = 0; q < n_phases; ++q) {
+            int rc = plan_phase(h, q, k, &all, &cache.total[q], s);
+            if (rc != ATREX_OK) return rc;
+            if (cache.total[q] > SEL_CAP) return ATREX_ERR_STATE;  // cannot happen: composites are unique
+        }
+        // every phase's candidates in one pass, each into its own zero-padded region
+        CU(h, cudaMemsetAsync(h->ctl->sel_count_all, 0, sizeof(h->ctl->sel_count_all), s));
+        for (uint32_t q = 0; q < n_phases; ++q) {
+            if (cache.total[q] == 0) continue;
+            const size_t n_pow2 = pow2_at_least(cache.total[q] < 2 ? 2 : cache.total[q]);
+            CU(h, cudaMemsetAsync(h->sel + (size_t)q * SEL_CAP * 4, 0, n_pow2 * 32, s));
+        }
+        CU(h, launch_topk_collect_all(all, h->scan_grid(h->L.n_slots, 256 * 4), s));
+        h->launches++;
+        for (uint32_t q = 0; q < n_phases; ++q) {   // sorted once, read by this and later calls
+            if (cache.total[q] == 0) continue;
+            const uint32_t n_pow2 = (uint32_t)pow2_at_least(cache.total[q] < 2 ? 2 : cache.total[q]);
+            CU(h, launch_topk_sort(h->sel + (size_t)q * SEL_CAP * 4, n_pow2, s));
+            h->launches++;
+        }
+        cache.sel_gen = h->fin_gen;
+        cache.k = k;
     }
-    if (total > SEL_CAP) return ATREX_ERR_STATE;  // cannot happen: composites are unique
-    uint32_t n_pow2 = (uint32_t)pow2_at_least(total < 2 ? 2 : total);
-    CU(h, cudaMemsetAsync(&h->ctl->sel_count, 0, sizeof(ull), s));
-    CU(h, cudaMemsetAsync(h->sel, 0, (size_t)n_pow2 * 32, s));
-    CU(h, launch_topk_collect(p, grid, s));
-    CU(h, launch_topk_sort(h->sel, n_pow2, s));
-    uint32_t m = (uint32_t)(total < k ? total : k);
-    CU(h, launch_topk_emit(finalize_params(h, h->topk_out, m), h->sel, m, s));
-    h->launches += 3;
+    const ull total = cache.total[phase];
+    const uint32_t m = (uint32_t)(total < k ? total : k);
+    CU(h, launch_topk_emit(finalize_params(h, h->topk_out, m), h->sel + (size_t)phase * SEL_CAP * 4, m, s));
+    h->launches++;
     CU(h, cudaMemcpyAsync(h_out, h->topk_out, (size_t)m * sizeof(atrex_entry_t), cudaMemcpyDeviceToHost, s));
     CU(h, cudaStreamSynchronize(s));
     *n_out = m;

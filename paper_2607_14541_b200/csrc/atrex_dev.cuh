@@ -70,6 +70,7 @@ struct Control {
     ull total_hi[ATREX_MAX_PHASES];
     ull keys_per_phase[ATREX_MAX_PHASES];
     ull count_per_phase[ATREX_MAX_PHASES];
+    ull sel_count_all[ATREX_MAX_PHASES];  // top-k: candidates collected per phase
     uint32_t hist[TOPK_BINS];
 };
 

@@ -279,16 +279,84 @@ __global__ void __launch_bounds__(FIN_THREADS) topk_hist_kernel(TopkParams p) {
         if (h[i] != 0) atomicAdd(&p.ctl->hist[i], h[i]);
 }
 
-__global__ void __launch_bounds__(FIN_THREADS) topk_collect_kernel(TopkParams p) {
-    for (ull i = (ull)blockIdx.x * blockDim.x + threadIdx.x; i < p.n_slots; i += (ull)gridDim.x * blockDim.x) {
-        SlotView v = load_slot(p.t, i);
-        if (!v.live || (uint32_t)(v.key >> 48) != p.phase) continue;
-        Composite x = composite_of(v);
-        if (!p.collect_all && compare_prefix(x, p) < 0) continue;
-        ull pos = atomicAdd(&p.ctl->sel_count, 1ull);
-        if (pos < p.sel_cap) {
-            ull* dst = p.sel + pos * 4;
-            dst[0] = x.c[2]; dst[1] = x.c[1]; dst[2] = x.c[0]; dst[3] = i;
+// -1: below the prefix, 0: equal on all fixed digits, +1: above (one phase of a multi-phase pass)
+__device__ __forceinline__ int compare_prefix_of(const Composite& x, const TopkAllParams& p, uint32_t q) {
+    for (uint32_t d = 0; d < p.n_prefix_digits[q]; ++d) {
+        uint32_t a = digit_of(x, (int)d, (int)p.shift[q]), b = p.prefix_digit[q][d];
+        if (a != b) return a > b ? 1 : -1;
+    }
+    return 0;
+}
+
+// Next-digit histograms of all active phases in one pass (shared memory: one row per phase).
+__global__ void __launch_bounds__(1024) topk_hist_all_kernel(const __grid_constant__ TopkAllParams p) {
+    extern __shared__ uint32_t h_all[];  // [ATREX_MAX_PHASES][TOPK_BINS], rows of inactive phases unused
+    for (uint32_t i = threadIdx.x; i < ATREX_MAX_PHASES * TOPK_BINS; i += blockDim.x)
+        if ((p.active_mask >> (i / TOPK_BINS)) & 1u) h_all[i] = 0;
+    __syncthreads();
+    constexpr int ILP = 4;
+    const ull stride = (ull)gridDim.x * blockDim.x;
+    for (ull i0 = (ull)blockIdx.x * blockDim.x + threadIdx.x; i0 < p.n_slots; i0 += stride * ILP) {
+        ull sk[ILP];
+        ulonglong2 x[ILP];
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) sk[u] = i0 + u * stride < p.n_slots ? p.t.keys[i0 + u * stride] : 0ull;
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) {
+            const uint32_t q = (uint32_t)(~sk[u] >> 48) & (ATREX_MAX_PHASES - 1);
+            const bool mine = sk[u] != 0 && ((p.active_mask >> q) & 1u);
+            x[u] = mine ? p.t.vals[i0 + u * stride] : make_ulonglong2(0, 0);
+            if (!mine) sk[u] = 0;
+        }
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) {
+            if (sk[u] == 0) continue;
+            SlotView v;
+            v.key = ~sk[u];
+            v.lo = x[u].x;
+            v.hi = x[u].y >> HI_SHIFT;
+            const uint32_t q = (uint32_t)(v.key >> 48) & (ATREX_MAX_PHASES - 1);
+            const Composite c = composite_of(v);
+            if (compare_prefix_of(c, p, q) != 0) continue;
+            atomicAdd(&h_all[q * TOPK_BINS + digit_of(c, (int)p.n_prefix_digits[q], (int)p.shift[q])], 1u);
+        }
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < ATREX_MAX_PHASES * TOPK_BINS; i += blockDim.x)
+        if (((p.active_mask >> (i / TOPK_BINS)) & 1u) && h_all[i] != 0) atomicAdd(&p.hist[i], h_all[i]);
+}
+
+// Candidates of all active phases in one pass, each phase into its own selection region.
+__global__ void __launch_bounds__(FIN_THREADS) topk_collect_all_kernel(const __grid_constant__ TopkAllParams p) {
+    constexpr int ILP = 4;
+    const ull stride = (ull)gridDim.x * blockDim.x;
+    for (ull i0 = (ull)blockIdx.x * blockDim.x + threadIdx.x; i0 < p.n_slots; i0 += stride * ILP) {
+        ull sk[ILP];
+        ulonglong2 x[ILP];
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) sk[u] = i0 + u * stride < p.n_slots ? p.t.keys[i0 + u * stride] : 0ull;
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) {
+            const uint32_t q = (uint32_t)(~sk[u] >> 48) & (ATREX_MAX_PHASES - 1);
+            const bool mine = sk[u] != 0 && ((p.active_mask >> q) & 1u);
+            x[u] = mine ? p.t.vals[i0 + u * stride] : make_ulonglong2(0, 0);
+            if (!mine) sk[u] = 0;
+        }
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) {
+            if (sk[u] == 0) continue;
+            SlotView v;
+            v.key = ~sk[u];
+            v.lo = x[u].x;
+            v.hi = x[u].y >> HI_SHIFT;
+            const uint32_t q = (uint32_t)(v.key >> 48) & (ATREX_MAX_PHASES - 1);
+            const Composite c = composite_of(v);
+            if (!((p.collect_all_mask >> q) & 1u) && compare_prefix_of(c, p, q) < 0) continue;
+            const ull pos = atomicAdd(&p.sel_count[q], 1ull);
+            if (pos < p.sel_cap) {
+                ull* dst = p.sel + ((ull)q * p.sel_cap + pos) * 4;
+                dst[0] = c.c[2]; dst[1] = c.c[1]; dst[2] = c.c[0]; dst[3] = i0 + u * stride;
+            }
         }
     }
 }
@@ -335,7 +403,10 @@ __global__ void __launch_bounds__(FIN_THREADS) topk_emit_kernel(FinalizeParams p
 }
 
 // ---- launchers ----------------------------------------------------------------------------
-cudaError_t finalize_prepare() { return cudaSuccess; }
+cudaError_t finalize_prepare() {
+    return cudaFuncSetAttribute(topk_hist_all_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)(ATREX_MAX_PHASES * TOPK_BINS * sizeof(uint32_t)));
+}
 
 cudaError_t launch_totals(const TableRef& t, ull n_slots, int grid, cudaStream_t stream) {
     totals_kernel<<<grid, TOT_THREADS, 0, stream>>>(t, n_slots);
@@ -353,13 +424,19 @@ cudaError_t launch_work_insert(const atrex_work_t* rows, ull n, const WorkRef& w
     return cudaGetLastError();
 }
 
-cudaError_t launch_topk_hist(const TopkParams& p, int grid, cudaStream_t stream) {
-    topk_hist_kernel<<<grid, FIN_THREADS, 0, stream>>>(p);
+cudaError_t launch_topk_hist_all(const TopkAllParams& p, int n_sms, cudaStream_t stream) {
+    const size_t smem = (size_t)ATREX_MAX_PHASES * TOPK_BINS * sizeof(uint32_t);
+    topk_hist_all_kernel<<<n_sms, 1024, smem, stream>>>(p);
     return cudaGetLastError();
 }
 
-cudaError_t launch_topk_collect(const TopkParams& p, int grid, cudaStream_t stream) {
-    topk_collect_kernel<<<grid, FIN_THREADS, 0, stream>>>(p);
+cudaError_t launch_topk_collect_all(const TopkAllParams& p, int grid, cudaStream_t stream) {
+    topk_collect_all_kernel<<<grid, FIN_THREADS, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_topk_hist(const TopkParams& p, int grid, cudaStream_t stream) {
+    topk_hist_kernel<<<grid, FIN_THREADS, 0, stream>>>(p);
     return cudaGetLastError();
 }
 

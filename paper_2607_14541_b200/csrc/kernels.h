@@ -79,6 +79,22 @@ struct TopkParams {
     uint32_t sel_cap;
 };
 
+// Top-k over several phases in one pass over the table: phase q of `active_mask` has its own digit
+// alignment, fixed prefix, histogram row and selection region.
+struct TopkAllParams {
+    TableRef t;
+    ull n_slots;
+    uint32_t active_mask;                              // phases taking part in this pass
+    uint32_t collect_all_mask;                         // phases whose every entry is collected
+    uint32_t shift[ATREX_MAX_PHASES];
+    uint32_t n_prefix_digits[ATREX_MAX_PHASES];
+    uint16_t prefix_digit[ATREX_MAX_PHASES][12];
+    uint32_t* hist;                                    // [ATREX_MAX_PHASES][TOPK_BINS] next-digit counts
+    ull* sel;                                          // [ATREX_MAX_PHASES][sel_cap][4]
+    ull* sel_count;                                    // [ATREX_MAX_PHASES]
+    uint32_t sel_cap;
+};
+
 cudaError_t ingest_prepare();
 cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream);
 cudaError_t launch_partition(const PartitionParams& p, int n_sms, cudaStream_t stream);
@@ -90,8 +106,9 @@ cudaError_t launch_totals(const TableRef& t, ull n_slots, int grid, cudaStream_t
 cudaError_t launch_emit(const FinalizeParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_work_insert(const atrex_work_t* rows, ull n, const WorkRef& w, Control* ctl, int grid,
                                cudaStream_t stream);
+cudaError_t launch_topk_hist_all(const TopkAllParams& p, int n_sms, cudaStream_t stream);
+cudaError_t launch_topk_collect_all(const TopkAllParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_topk_hist(const TopkParams& p, int grid, cudaStream_t stream);
-cudaError_t launch_topk_collect(const TopkParams& p, int grid, cudaStream_t stream);
 cudaError_t launch_topk_sort(ull* sel, uint32_t n_pow2, cudaStream_t stream);
 cudaError_t launch_topk_emit(const FinalizeParams& p, const ull* sel, uint32_t n, cudaStream_t stream);
 
