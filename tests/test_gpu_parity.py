@@ -359,3 +359,25 @@ def test_many_apps_eight_phases_and_largest_geometry(lib):
     agg = gpu_aggregate(lib, recs, weights, 8, max_keys=1 << 25)
     assert_same_as_oracle(agg, o, 8, ks=(3,))
     assert agg.stats()["table_slots"] >= 4096 * 11000
+
+
+def test_topk_requests_in_any_order_and_after_more_records(lib):
+    """The ranking keeps what it worked out for all phases until the next finalize: answers must not
+    depend on the order of (phase, k) requests, and must follow the table after more records arrive."""
+    spec = make_spec(2, small=True, n=600_000)                  # three phases
+    recs = tg.generate(spec)
+    first, second = recs[:350_000], recs[350_000:]
+    agg = gpu_aggregate(lib, first, spec.app_weights, spec.n_phases, max_keys=spec.max_keys)
+    o = oracle_of(first, spec.app_weights, spec.n_phases)
+    agg.finalize(PEAK_BW, PEAK_FLOPS)
+    for phase, k in ((2, 10), (0, 10), (1, 10), (1, 3), (0, 500), (2, 500), (1, 1), (0, 10), (2, 4096)):
+        assert agg.topk(phase, k).tobytes() == o.topk(PEAK_BW, PEAK_FLOPS, phase, k).tobytes(), (phase, k)
+    agg.ingest(to_dev(second), n=len(second))
+    with pytest.raises(lib.AtrexError):
+        agg.topk(0, 10)                                          # stale until the next finalize
+    o.ingest(second, threads=4)
+    agg.finalize(PEAK_BW, PEAK_FLOPS)
+    for phase, k in ((1, 10), (0, 10), (2, 10), (0, 7)):
+        assert agg.topk(phase, k).tobytes() == o.topk(PEAK_BW, PEAK_FLOPS, phase, k).tobytes(), (phase, k)
+    agg.finalize(PEAK_BW, [2 * x for x in PEAK_FLOPS])          # other peaks: same ranking, other roofline times
+    assert agg.topk(1, 10).tobytes() == o.topk(PEAK_BW, [2 * x for x in PEAK_FLOPS], 1, 10).tobytes()
