@@ -186,7 +186,10 @@ int atrex_agg_finalize_with_totals(atrex_agg_t*, const atrex_hw_peaks_t* peaks, 
 /* Table 2: the min(k, keys of `phase`) entries with the largest weighted time, compared as
  * exact 128-bit integers, ties broken by ascending key; written in that order to `h_out`
  * (HOST, capacity k).  k <= ATREX_MAX_TOPK.  Uses the totals and peaks of the last finalize
- * (ATREX_ERR_STATE if there was none since the last ingest).  Synchronises `stream`. */
+ * (ATREX_ERR_STATE if there was none since the last ingest).  Synchronises `stream`.
+ * Cost: the first call after a finalize selects the best k of EVERY phase in two passes over the
+ * table and keeps the selections; further calls with the same k (any phase) only copy their
+ * answer out, a call with another k repeats the second pass. */
 int atrex_agg_topk(atrex_agg_t*, uint32_t phase, uint32_t k, atrex_entry_t* h_out, uint32_t* n_out,
                    void* stream);
 
