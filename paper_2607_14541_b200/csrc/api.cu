@@ -23,7 +23,6 @@ constexpr uint32_t CAND_BITS = 17;                     // candidate table of the
 constexpr size_t SKETCH_BYTES = (size_t)4 << 20;        // 2^20 counters (ingest.cu SKETCH_BITS)
 constexpr size_t HOT_SCRATCH_BYTES = SKETCH_BYTES + ((size_t)12 << CAND_BITS);
 constexpr uint32_t APPW_SMEM_MAX = 4096;
-constexpr uint32_t MAX_PROBE = 4096;                   // work-table probe bound
 constexpr uint32_t SEL_CAP = ATREX_MAX_TOPK + TOPK_CAND_CAP;
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -32,12 +31,6 @@ ull pow2_at_least(ull x) {
     ull p = 1;
     while (p < x) p <<= 1;
     return p;
-}
-
-int log2_of(ull p) {
-    int l = 0;
-    while ((1ull << l) < p) ++l;
-    return l;
 }
 
 struct Layout {
