@@ -35,13 +35,14 @@ ull pow2_at_least(ull x) {
 
 struct Layout {
     size_t off_ctl, off_keys, off_vals, off_work, off_appw, off_hot, off_staging[2], off_sel, off_topk_out, off_hist_all,
-        off_spill_cnt, off_spill, off_hot_scratch, total;
+        off_spill_cnt, off_spill, off_hot_scratch, off_queue, total;
     ull n_slots, work_slots;
     uint32_t lp, C;              // partitions = 1 << lp, slots per partition
     uint32_t Cw;                 // work-table slots per partition
     uint32_t n_groups, cap;      // spill buffers: [P][n_groups][cap] entries
     ull sub_launch;              // records per scatter + partition launch pair
     uint32_t hot_slots;
+    uint32_t queue_cap;        // deferred entries per CTA in the partition pass
     bool appw_in_smem;
 };
 
@@ -73,6 +74,12 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     ull per_buf = (L->sub_launch * 9 / 2) / (((ull)n_sms) << L->lp);
     if (per_buf < 64) per_buf = 64;
     L->cap = (uint32_t)((per_buf + 7) / 8 * 8);
+    // entries of one partition whose first look fails wait in a per-CTA queue: room for a quarter of
+    // the partition's worst-case stream, at most 32 K entries (the rest is settled in line)
+    {
+        ull q = (ull)L->cap * n_sms / 4;
+        L->queue_cap = (uint32_t)(q < 1024 ? 1024 : (q > 32768 ? 32768 : q));
+    }
     // work table: same partitions as the key table, 1.5 slots per row plus slack for uneven partitions
     L->Cw = c->max_work_rows ? (uint32_t)((((c->max_work_rows * 3 / 2) >> L->lp) + 64 + 31) / 32 * 32) : 0;
     L->work_slots = (ull)L->Cw << L->lp;
@@ -95,6 +102,7 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     L->off_hist_all = o;       o += round_up((size_t)ATREX_MAX_PHASES * TOPK_BINS * 4, ALIGN);
     L->off_topk_out = o;       o += round_up((size_t)ATREX_MAX_TOPK * sizeof(atrex_entry_t), ALIGN);
     L->off_hot_scratch = o;    o += round_up(HOT_SCRATCH_BYTES, ALIGN);
+    L->off_queue = o;          o += round_up((size_t)L->n_groups * L->queue_cap * 16, ALIGN);
     L->off_spill_cnt = o;      o += round_up(((size_t)L->n_groups << L->lp) * 4, ALIGN);
     L->off_spill = o;          o += round_up(((size_t)L->n_groups << L->lp) * L->cap * 16, ALIGN) + ALIGN;  // + prefetch overrun
     L->total = o;
@@ -135,6 +143,7 @@ struct atrex_agg {
     ulonglong2* vals = nullptr;
     uint32_t* spill_cnt = nullptr;
     unsigned char* spill = nullptr;
+    ulonglong2* queue = nullptr;
     unsigned char* hot_scratch = nullptr;
     WorkSlot* work = nullptr;
     uint32_t* d_appw = nullptr;
@@ -269,6 +278,7 @@ int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out) {
         h->vals = (ulonglong2*)(h->ws + L.off_vals);
         h->spill_cnt = (uint32_t*)(h->ws + L.off_spill_cnt);
         h->spill = h->ws + L.off_spill;
+        h->queue = (ulonglong2*)(h->ws + L.off_queue);
         h->hot_scratch = h->ws + L.off_hot_scratch;
         h->work = (WorkSlot*)(h->ws + L.off_work);
         h->d_appw = (uint32_t*)(h->ws + L.off_appw);
@@ -371,6 +381,8 @@ static int drain_spill(atrex_agg* h, bool force, cudaStream_t s) {
     q.n_groups = h->L.n_groups;
     q.n_used = h->L.n_groups;
     q.cap = h->L.cap;
+    q.queue = h->queue;
+    q.queue_cap = h->L.queue_cap;
     q.force = force ? 1u : 0u;
     q.seq = h->scatter_seq;
     CU(h, launch_partition(q, h->n_sms, s));

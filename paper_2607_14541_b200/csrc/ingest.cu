@@ -419,6 +419,62 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
 // is processed, the next one's keys and spill entries are pulled into L2.
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
+// Shared-window addresses of the partition pass's arrays.
+struct PartSmem {
+    uint32_t keys, a0, a1, cnt;
+};
+
+// General probe, one entry per lane (busy = this lane has one): walks the key's probe sequence from
+// the pair at `slot`, claims the first free slot if the key is not there.  Warp-convergent.  Returns
+// the key's slot, or PROBE_FAILED when the partition has no room.
+constexpr uint32_t PROBE_FAILED = 0xFFFFFFFFu;
+
+__device__ __forceinline__ uint32_t probe_general(const PartSmem& m, ull skey, uint32_t slot, uint32_t advance, bool busy,
+                                                  uint32_t C, Control* ctl) {
+    uint32_t steps = 0;
+    while (__any_sync(0xFFFFFFFFu, busy)) {
+        if (busy) {
+            const ulonglong2 kk = lds_v2u64(m.keys + slot * 8);
+            const bool hit1 = kk.y == skey;
+            if (kk.x == skey || hit1) {
+                slot += hit1 ? 1u : 0u;
+                busy = false;
+            } else if (kk.x == 0 || kk.y == 0) {
+                // claim the first empty slot of the pair; a lost race re-reads the pair
+                const uint32_t at = slot + (kk.x == 0 ? 0u : 1u);
+                const ull old = atoms_cas64(m.keys + at * 8, 0ull, skey);
+                if (old == 0) reds_or(m.cnt + at * 4, NEW_KEY_FLAG);
+                if (old == 0 || old == skey) {
+                    slot = at;
+                    busy = false;
+                }
+            } else {
+                slot += advance;
+                if (slot >= C) slot -= C;
+            }
+            if (busy && ++steps > 2 * C) {  // partition full (bounded; counts lost races too)
+                busy = false;
+                slot = PROBE_FAILED;
+                atomicOr(&ctl->status, ST_TABLE_FULL);
+                atomicAdd(&ctl->n_dropped, 1ull);
+            }
+        }
+    }
+    return slot;
+}
+
+// One entry's product and count into its slot's limbs; the adder that fills the high limb moves the
+// slot's sums to HBM (this CTA owns the slot, so those adds are exact; the write-back adds on top).
+__device__ __forceinline__ void part_accumulate(const PartSmem& m, uint32_t slot, ull v, ulonglong2* vals_of_partition) {
+    if (limbs_add(m.a0 + slot * 4, m.a1 + slot * 4, m.cnt + slot * 4, v, 1u)) {
+        ull hi, lo = limbs_drain(m.a0 + slot * 4, m.a1 + slot * 4, &hi);
+        ull* vp = reinterpret_cast<ull*>(vals_of_partition + slot);
+        ull old = atomicAdd(vp, lo);
+        hi += (old + lo < old) ? 1ull : 0ull;
+        if (hi) atomicAdd(vp + 1, hi << HI_SHIFT);
+    }
+}
+
 __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionParams q) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t C = q.t.C;
@@ -426,8 +482,13 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     uint32_t* s_a0 = reinterpret_cast<uint32_t*>(s_keys + C);
     uint32_t* s_a1 = s_a0 + C;
     uint32_t* s_cnt = s_a1 + C;
-    const uint32_t a_keys = smem_addr(s_keys), a_a0 = smem_addr(s_a0), a_a1 = smem_addr(s_a1), a_cnt = smem_addr(s_cnt);
-    __shared__ uint32_t s_total;
+    PartSmem m;
+    m.keys = smem_addr(s_keys);
+    m.a0 = smem_addr(s_a0);
+    m.a1 = smem_addr(s_a1);
+    m.cnt = smem_addr(s_cnt);
+    __shared__ uint32_t s_total, s_qn;
+    ulonglong2* const my_queue = q.queue + (size_t)blockIdx.x * q.queue_cap;
     __shared__ unsigned char s_owner[INGEST_THREADS / 32][32];  // per warp: who owns queue position t
     const uint32_t n_parts = 1u << q.t.lp;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
@@ -437,7 +498,10 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(&q.t.ctl->n_drains, 1ull);
 
     for (uint32_t part = blockIdx.x; part < n_parts; part += gridDim.x) {
-        if (threadIdx.x == 0) s_total = 0;
+        if (threadIdx.x == 0) {
+            s_total = 0;
+            s_qn = 0;
+        }
         __syncthreads();  // also: the previous partition's write-back has finished reading shared memory
         uint32_t local_total = 0;
         for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) local_total += q.spill_cnt[((ull)g << q.t.lp) + part];
@@ -491,100 +555,107 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                     searching[u] = ok[u];
                 }
                 // First look, straight-line for all four entries: most keys sit in the first pair
-                // of slots of their probe sequence.
+                // of slots of their probe sequence, and most new keys find room there.
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const ulonglong2 kk = lds_v2u64(a_keys + slot[u] * 8);
+                    const ulonglong2 kk = lds_v2u64(m.keys + slot[u] * 8);
                     const bool hit1 = kk.y == skey[u];
                     if (hit1) slot[u] += 1;
-                    if (kk.x == skey[u] || hit1) searching[u] = false;
-                }
-                // The rest (new keys, collisions) is a minority scattered over the four rounds:
-                // hand the pending entries out one per lane, so that the general probe loop runs
-                // once per warp instead of once per round.  Each pending entry's owner publishes
-                // (round, lane) at the entry's queue position; lane t serves position t.
-                while (true) {
-                    uint32_t pend[4], before[4], total = 0;
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        pend[u] = __ballot_sync(0xFFFFFFFFu, searching[u]);
-                        before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
-                        total += __popc(pend[u]);
-                    }
-                    if (total == 0) break;
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (searching[u] && before[u] < 32) s_owner[warp][before[u]] = (unsigned char)((u << 5) | lane);
-                    __syncwarp();
-                    const bool serving = lane < total;
-                    const uint32_t code = serving ? s_owner[warp][lane] : lane;
-                    const uint32_t src = code & 31u, su = code >> 5;
-                    ull key_s = 0;
-                    uint32_t slot_s = 0;
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const ull k = __shfl_sync(0xFFFFFFFFu, skey[u], src);
-                        const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u] | (((strides >> (8 * u)) & 7u) << 16), src);
-                        if (su == (uint32_t)u) {
-                            key_s = k;
-                            slot_s = sl;
-                        }
-                    }
-                    const uint32_t advance = 2u * stride_of(q.t, slot_s >> 16);
-                    slot_s &= 0xFFFFu;
-                    bool busy = serving;
-                    uint32_t steps = 0;
-                    while (__any_sync(0xFFFFFFFFu, busy)) {
-                        if (busy) {
-                            const ulonglong2 kk = lds_v2u64(a_keys + slot_s * 8);
-                            const bool hit1 = kk.y == key_s;
-                            if (kk.x == key_s || hit1) {
-                                slot_s += hit1 ? 1u : 0u;
-                                busy = false;
-                            } else if (kk.x == 0 || kk.y == 0) {
-                                // claim the first empty slot of the pair; a lost race re-reads the pair
-                                const uint32_t at = slot_s + (kk.x == 0 ? 0u : 1u);
-                                const ull old = atoms_cas64(a_keys + at * 8, 0ull, key_s);
-                                if (old == 0) reds_or(a_cnt + at * 4, NEW_KEY_FLAG);
-                                if (old == 0 || old == key_s) {
-                                    slot_s = at;
-                                    busy = false;
-                                }
-                            } else {
-                                slot_s += advance;
-                                if (slot_s >= C) slot_s -= C;
-                            }
-                            if (busy && ++steps > 2 * C) {  // partition full (bounded; counts lost races too)
-                                busy = false;
-                                slot_s = 0xFFFFFFFFu;
-                                atomicOr(&q.t.ctl->status, ST_TABLE_FULL);
-                                atomicAdd(&q.t.ctl->n_dropped, 1ull);
-                            }
-                        }
-                    }
-                    // results go back to the owners
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const uint32_t found = __shfl_sync(0xFFFFFFFFu, slot_s, before[u] & 31u);
-                        if (searching[u] && before[u] < 32) {
+                    if (kk.x == skey[u] || hit1) {
+                        searching[u] = false;
+                    } else if (searching[u] && (kk.x == 0 || kk.y == 0)) {
+                        // a new key whose first pair has room is inserted at once, so that its later
+                        // occurrences find it here; losing the slot to another key defers the entry
+                        const uint32_t at = slot[u] + (kk.x == 0 ? 0u : 1u);
+                        const ull old = atoms_cas64(m.keys + at * 8, 0ull, skey[u]);
+                        if (old == 0) reds_or(m.cnt + at * 4, NEW_KEY_FLAG);
+                        if (old == 0 || old == skey[u]) {
+                            slot[u] = at;
                             searching[u] = false;
-                            if (found == 0xFFFFFFFFu) ok[u] = false; else slot[u] = found;
                         }
                     }
-                    __syncwarp();  // the queue is rewritten in the next round
                 }
+                // The rest (new keys, collisions: a few per batch) is not settled here, where the fixed
+                // cost of a general probe round would be paid for a handful of entries: it goes to this
+                // CTA's queue and is settled after the partition's stream, 32 entries per warp round.
+                uint32_t pend[4], before[4], total = 0;
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    if (ok[u] && limbs_add(a_a0 + slot[u] * 4, a_a1 + slot[u] * 4, a_cnt + slot[u] * 4, v[u], 1u)) {
-                        // drain: this CTA owns the slot, so adds into HBM are exact; the write-back
-                        // below adds on top of them
-                        ull hi, lo = limbs_drain(a_a0 + slot[u] * 4, a_a1 + slot[u] * 4, &hi);
-                        ull* vp = reinterpret_cast<ull*>(q.t.vals + base + slot[u]);
-                        ull old = atomicAdd(vp, lo);
-                        hi += (old + lo < old) ? 1ull : 0ull;
-                        if (hi) atomicAdd(vp + 1, hi << HI_SHIFT);
+                    pend[u] = __ballot_sync(0xFFFFFFFFu, searching[u]);
+                    before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
+                    total += __popc(pend[u]);
+                }
+                if (total != 0) {
+                    uint32_t qbase = 0;
+                    if (lane == 0) qbase = atomicAdd(&s_qn, total);
+                    qbase = __shfl_sync(0xFFFFFFFFu, qbase, 0);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (searching[u] && qbase + before[u] < q.queue_cap) {
+                            my_queue[qbase + before[u]] = make_ulonglong2(~skey[u], v[u]);
+                            searching[u] = false;
+                            ok[u] = false;
+                        }
+                    }
+                    // Queue full (a partition made of new keys only): settle the remainder in line.
+                    // The pending entries are handed out one per lane: each one's owner publishes
+                    // (round, lane) at the entry's position; lane t serves position t.
+                    while (qbase + total > q.queue_cap) {
+                        total = 0;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            pend[u] = __ballot_sync(0xFFFFFFFFu, searching[u]);
+                            before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
+                            total += __popc(pend[u]);
+                        }
+                        if (total == 0) break;
+                        qbase = q.queue_cap;  // stay in this loop until nothing is pending
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (searching[u] && before[u] < 32) s_owner[warp][before[u]] = (unsigned char)((u << 5) | lane);
+                        __syncwarp();
+                        const bool serving = lane < total;
+                        const uint32_t code = serving ? s_owner[warp][lane] : lane;
+                        const uint32_t from = code & 31u, su = code >> 5;
+                        ull key_s = 0;
+                        uint32_t slot_s = 0;
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const ull k = __shfl_sync(0xFFFFFFFFu, skey[u], from);
+                            const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u] | (((strides >> (8 * u)) & 7u) << 16), from);
+                            if (su == (uint32_t)u) {
+                                key_s = k;
+                                slot_s = sl;
+                            }
+                        }
+                        const uint32_t found_s = probe_general(m, key_s, slot_s & 0xFFFFu, 2u * stride_of(q.t, slot_s >> 16),
+                                                               serving, C, q.t.ctl);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const uint32_t found = __shfl_sync(0xFFFFFFFFu, found_s, before[u] & 31u);
+                            if (searching[u] && before[u] < 32) {
+                                searching[u] = false;
+                                if (found == PROBE_FAILED) ok[u] = false; else slot[u] = found;
+                            }
+                        }
+                        __syncwarp();  // the owner table is rewritten in the next round
                     }
                 }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (ok[u]) part_accumulate(m, slot[u], v[u], q.t.vals + base);
+            }
+        }
+        __syncthreads();
+        {   // the queued entries, one per lane
+            const uint32_t qn = min(s_qn, q.queue_cap);
+            for (uint32_t i0 = warp * 32u; i0 < qn; i0 += n_warps * 32u) {
+                const bool serving = i0 + lane < qn;
+                const ulonglong2 ent = serving ? __ldcg(my_queue + i0 + lane) : make_ulonglong2(0, 0);
+                const uint32_t hh = hash32(ent.x);
+                const uint32_t start = local_of(hh, (uint32_t)(ent.x >> 48), C) & ~1u;
+                const uint32_t found = probe_general(m, ~ent.x, start, 2u * stride_of(q.t, stride_index(hh)), serving, C, q.t.ctl);
+                if (serving && found != PROBE_FAILED) part_accumulate(m, found, ent.y, q.t.vals + base);
             }
         }
         __syncthreads();

@@ -34,6 +34,8 @@ struct PartitionParams {
     uint32_t cap;
     uint32_t force;            // 1: drain unconditionally; 0: only if the scatter launch `seq` asked for it
     ull seq;
+    ulonglong2* queue;         // [gridDim][queue_cap] entries whose first look failed, settled after the partition's stream
+    uint32_t queue_cap;
 };
 
 struct HotBuildParams {
