@@ -384,9 +384,9 @@ def test_topk_requests_in_any_order_and_after_more_records(lib):
 
 
 def test_crowded_small_partitions_overflow_the_deferred_queue(lib):
-    """Tiny partitions (128 slots) at a load factor of 0.76, no hot directory, 260 K entries per partition
-    in one drain: more entries fail the first look (about 50 K per partition) than the partition pass's
-    per-CTA queue holds (32 K), so the in-line fallback runs as well.  Still exact."""
+    """Tiny partitions (128 slots) at a load factor of 0.76, no hot directory, about 200 K entries per
+    partition in the first drain: more entries fail the first look (45-50 K per partition) than the
+    partition pass's per-CTA queue holds (32 K), so the in-line fallback runs as well.  Still exact."""
     rng = np.random.default_rng(77)
     n, n_keys = 1 << 26, 25_000
     k = rng.integers(0, n_keys, n, dtype=np.uint32)
