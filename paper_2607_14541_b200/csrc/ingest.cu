@@ -865,8 +865,11 @@ __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
     }
     __syncthreads();
     const uint32_t mult = s_thr;
+    for (uint32_t i = threadIdx.x; i < n_buckets; i += blockDim.x) occupancy[i] = 0;
+    __syncthreads();
     // install from the most to the least frequent class (counts within a class differ < 2x), so
-    // that a key can only lose its bucket to keys about as frequent as itself
+    // that a key can only lose its bucket to keys about as frequent as itself; a bucket's ways are
+    // handed out by its shared-memory counter
     for (int round = 0; round < 11; ++round) {
         uint32_t hi = round == 0 ? 0xFFFFFFFFu : (2048u >> round), lo = max(1024u >> round, thr);
         if (lo < hi) {
@@ -874,10 +877,12 @@ __global__ void __launch_bounds__(1024, 1) hot_select_kernel(HotBuildParams p) {
                 uint32_t c = c_cnt[i];
                 if (c >= lo && c < hi) {
                     ull skey = c_key[i];
-                    uint32_t b = dir_bucket_of_key(~skey, mult, n_buckets) * DIR_WAYS;
-                    bool placed = false;
-                    for (uint32_t way = 0; way < DIR_WAYS && !placed; ++way) placed = atomicCAS(&p.hot_keys[b + way], 0ull, skey) == 0;
-                    if (placed) atomicAdd(&s_inserted, 1u);
+                    const uint32_t b = dir_bucket_of_key(~skey, mult, n_buckets);
+                    const uint32_t way = atomicAdd(&occupancy[b], 1u);
+                    if (way < DIR_WAYS) {
+                        p.hot_keys[b * DIR_WAYS + way] = skey;
+                        atomicAdd(&s_inserted, 1u);
+                    }
                 }
             }
         }
