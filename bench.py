@@ -339,8 +339,12 @@ def cpu_baseline(args, spec, records, torch):
     recs = records[: count * RECORD_BYTES].cpu().numpy().view(tg.RECORD_DTYPE)
     threads = host_threads()
     dt, used = time_oracle(spec, recs, threads)
+    single = min(count, 1 << 22)                       # the same oracle on one thread, a shorter prefix
+    dt1, _ = time_oracle(spec, recs[:single], 1)
     return {"value": count / dt, "unit": UNIT, "cores": used, "kind": "oracle", "seconds": dt,
-            "sample": f"first {count} records of the workload, std::map group-by on {used} threads + finalize + topk"}
+            "sample": f"first {count} records of the workload, std::map group-by on {used} threads + finalize + topk",
+            "single_thread": {"value": single / dt1, "unit": UNIT, "seconds": dt1,
+                              "sample": f"first {single} records, one thread"}}
 
 
 def main():
