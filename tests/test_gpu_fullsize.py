@@ -87,6 +87,16 @@ def test_full_size_trace_sampled_keys_and_invariants(index):
         assert (wt_all == ent["count"].astype(object) * P).all()
         assert int(ent["wt_hi"].max()) > 6000
 
+    # chunking must not matter: the same 2^30 records in ONE call give the same entries
+    if index == 3:
+        agg1 = p.Aggregator(spec.app_weights, spec.n_phases, spec.max_keys, max_work_rows=len(work))
+        agg1.set_work_table(work)
+        agg1.ingest(records, n=n)
+        a, na = agg1.finalize(spec.peak_bw, spec.peak_flops)
+        b, nb = agg.finalize(spec.peak_bw, spec.peak_flops)
+        assert na == nb and torch.equal(p.sort_entries_by_key(a, na), p.sort_entries_by_key(b, nb))
+        del agg1, a, b
+
     # the release artefacts made from this entry list (config 2's three phases and config 3's
     # 16 M entries exercise every word of the ranking order and several sort tiles per digit)
     if index in (2, 3):
