@@ -416,7 +416,11 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
 // --------------------------------------------------------------------------------------
 // Pass 2: a CTA aggregates one partition at a time entirely in shared memory.  CTAs are
 // persistent and take partitions blockIdx.x, blockIdx.x + gridDim.x, ...; while one partition
-// is processed, the next one's keys and spill entries are pulled into L2.
+// is processed, the next one's keys and spill entries are pulled into L2.  Per partition: copy the
+// keys in; stream the entries of all scatter CTAs, four per lane, and settle each with one look at
+// the first pair of its probe sequence (hit, or a new key with room there); entries that need more
+// than that wait in a per-CTA queue in global memory and are settled, 32 per warp round, once the
+// stream is through; then write the deltas back.
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 // Shared-window addresses of the partition pass's arrays.
@@ -489,7 +493,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     m.cnt = smem_addr(s_cnt);
     __shared__ uint32_t s_total, s_qn;
     ulonglong2* const my_queue = q.queue + (size_t)blockIdx.x * q.queue_cap;
-    __shared__ unsigned char s_owner[INGEST_THREADS / 32][32];  // per warp: who owns queue position t
+    __shared__ unsigned char s_owner[INGEST_THREADS / 32][32];  // in-line fallback, per warp: (round, lane) owning hand-out position t
     const uint32_t n_parts = 1u << q.t.lp;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
     // the spill buffers are drained lazily: unless forced, only when the scatter launch just
