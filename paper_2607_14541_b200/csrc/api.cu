@@ -35,7 +35,7 @@ ull pow2_at_least(ull x) {
 
 struct Layout {
     size_t off_ctl, off_keys, off_vals, off_work, off_appw, off_hot, off_staging[2], off_sel, off_topk_out, off_hist_all,
-        off_spill_cnt, off_spill, off_hot_scratch, off_queue, total;
+        off_spill_cnt, off_spill, off_hot_scratch, off_queue, off_hot_img, total;
     ull n_slots, work_slots;
     uint32_t lp, C;              // partitions = 1 << lp, slots per partition
     uint32_t Cw;                 // work-table slots per partition
@@ -96,6 +96,7 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     L->off_work = o;           o += round_up(L->work_slots * sizeof(WorkSlot), ALIGN);
     L->off_appw = o;           o += round_up((size_t)c->n_apps * 4, ALIGN);
     L->off_hot = o;            o += round_up((size_t)(L->hot_slots ? L->hot_slots : 2) * 8, ALIGN);
+    L->off_hot_img = o;        o += round_up((size_t)L->n_groups * (L->hot_slots ? L->hot_slots : 2) * 16, ALIGN);
     L->off_staging[0] = o;     o += STAGING_BYTES;
     L->off_staging[1] = o;     o += STAGING_BYTES;
     L->off_sel = o;            o += round_up((size_t)SEL_CAP * 32 * c->n_phases, ALIGN);   // one region per phase
@@ -148,6 +149,8 @@ struct atrex_agg {
     WorkSlot* work = nullptr;
     uint32_t* d_appw = nullptr;
     ull* hot_keys = nullptr;
+    ulonglong2* hot_img = nullptr;   // [n_groups][hot_slots] per-CTA directory sums not yet in the table
+    bool hot_dirty = false;          // the image rows may hold sums
     unsigned char* staging[2] = {nullptr, nullptr};
     ull* sel = nullptr;
     atrex_entry_t* topk_out = nullptr;
@@ -283,6 +286,7 @@ int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out) {
         h->work = (WorkSlot*)(h->ws + L.off_work);
         h->d_appw = (uint32_t*)(h->ws + L.off_appw);
         h->hot_keys = (ull*)(h->ws + L.off_hot);
+        h->hot_img = (ulonglong2*)(h->ws + L.off_hot_img);
         h->staging[0] = h->ws + L.off_staging[0];
         h->staging[1] = h->ws + L.off_staging[1];
         h->sel = (ull*)(h->ws + L.off_sel);
@@ -292,6 +296,7 @@ int atrex_agg_create(const atrex_agg_config_t* cfg, atrex_agg_t** out) {
         if (e == cudaSuccess) e = cudaMemset(h->ws + L.off_ctl, 0, L.off_appw - L.off_ctl);  // control, table, work
         if (e == cudaSuccess) e = cudaMemcpy(h->d_appw, cfg->app_weights, (size_t)cfg->n_apps * 4, cudaMemcpyHostToDevice);
         if (e == cudaSuccess) e = cudaMemset(h->hot_keys, 0, (size_t)(L.hot_slots ? L.hot_slots : 2) * 8);
+        if (e == cudaSuccess) e = cudaMemset(h->hot_img, 0, (size_t)L.n_groups * (L.hot_slots ? L.hot_slots : 2) * 16);
         if (e == cudaSuccess) e = cudaMemset(h->spill_cnt, 0, ((size_t)L.n_groups << L.lp) * 4);
         if (e == cudaSuccess) e = cudaHostAlloc((void**)&h->h_ctl, sizeof(Control), cudaHostAllocDefault);
         if (e == cudaSuccess)
@@ -336,6 +341,8 @@ int atrex_agg_reset(atrex_agg_t* h, void* stream) {
     CU(h, cudaMemsetAsync(h->ctl, 0, sizeof(Control), s));
     CU(h, cudaMemsetAsync(h->keys, 0, h->L.off_work - h->L.off_keys, s));  // keys and vals
     CU(h, cudaMemsetAsync(h->spill_cnt, 0, ((size_t)h->L.n_groups << h->L.lp) * 4, s));  // discard undrained entries
+    if (h->hot_dirty) CU(h, cudaMemsetAsync(h->hot_img, 0, (size_t)h->L.n_groups * (h->L.hot_slots ? h->L.hot_slots : 2) * 16, s));
+    h->hot_dirty = false;
     h->spill_pending = false;
     h->hot_ready = false;
     h->finalized = false;
@@ -387,6 +394,12 @@ static int drain_spill(atrex_agg* h, bool force, cudaStream_t s) {
     q.seq = h->scatter_seq;
     CU(h, launch_partition(q, h->n_sms, s));
     h->launches++;
+    if (force && h->hot_dirty) {
+        // results are about to be read: the directory sums kept per scatter CTA join the table
+        CU(h, launch_hot_fold(h->hot_keys, h->hot_img, h->L.n_groups, h->L.hot_slots, h->table_ref(), s));
+        h->launches++;
+        h->hot_dirty = false;
+    }
     if (force) h->spill_pending = false;
     return ATREX_OK;
 }
@@ -429,6 +442,7 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
     p.hot_keys = h->hot_keys;
     p.hot_slots = h->L.hot_slots;
     p.hot_buckets = h->L.hot_slots / 4;
+    p.hot_img = h->hot_img;
     p.t = h->table_ref();
     p.spill = h->spill;
     p.spill_cnt = h->spill_cnt;
@@ -440,6 +454,7 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
     p.drain_above = h->L.cap / 4 * 3;
     p.seq = ++h->scatter_seq;
     CU(h, launch_scatter(p, h->hot_ready, grid, s));
+    if (h->hot_ready) h->hot_dirty = true;
     h->spill_pending = true;
     h->launches++;
     return drain_spill(h, /*force=*/false, s);

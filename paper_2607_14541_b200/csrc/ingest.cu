@@ -403,12 +403,60 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams
         atomicMax(&p.t.ctl->max_fill, (ull)fullest);
     }
     if (HOT) {
+        // This launch's directory sums go to the CTA's own row of the directory image: plain coalesced
+        // read-modify-writes, no atomics (148 CTAs adding the same ~9 K keys into the table at the end
+        // of every launch cost 59 us per launch).  hot_fold_kernel adds the rows into the table before
+        // results are read.
+        ulonglong2* img = p.hot_img + (size_t)blockIdx.x * p.hot_slots;
         for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
             const uint32_t c = g_cnt[i], lo = g_a0[i], hi = g_a1[i];
             if ((c | lo | hi) != 0) {
-                const ull key = ~g_keys[i];
-                table_accumulate(p.t, key, hash32(key), (ull)lo | ((ull)hi << 32), 0, (ull)c);
+                const ulonglong2 o = img[i];
+                const ull nlo = o.x + ((ull)lo | ((ull)hi << 32));
+                img[i] = make_ulonglong2(nlo, o.y + (ull)c + ((nlo < o.x ? 1ull : 0ull) << HI_SHIFT));
             }
+        }
+    }
+}
+
+// Adds every CTA's directory image row into the table and clears the rows.  A CTA handles 32
+// directory slots: warp w sums rows w, w + 8, ... of those slots (exact: 128-bit sum, count), the
+// eight partial sums meet in shared memory and warp 0 does one table update per slot.
+constexpr int FOLD_WARPS = 8;
+
+__global__ void __launch_bounds__(FOLD_WARPS * 32) hot_fold_kernel(const ull* hot_keys, ulonglong2* hot_img,
+                                                                   uint32_t n_groups, uint32_t hot_slots, TableRef t) {
+    __shared__ ull s_lo[FOLD_WARPS][32], s_hi[FOLD_WARPS][32], s_cnt[FOLD_WARPS][32];
+    const uint32_t lane = threadIdx.x & 31u, w = threadIdx.x >> 5;
+    const uint32_t i = blockIdx.x * 32u + lane;
+    ull lo = 0, hi = 0, count = 0;
+    if (i < hot_slots) {
+        for (uint32_t g = w; g < n_groups; g += FOLD_WARPS) {
+            ulonglong2* at = hot_img + (size_t)g * hot_slots + i;
+            const ulonglong2 v = *at;
+            if ((v.x | v.y) == 0) continue;
+            const ull s = lo + v.x;
+            hi += (v.y >> HI_SHIFT) + (s < lo ? 1ull : 0ull);
+            lo = s;
+            count += v.y & COUNT_MASK;
+            *at = make_ulonglong2(0, 0);
+        }
+    }
+    s_lo[w][lane] = lo;
+    s_hi[w][lane] = hi;
+    s_cnt[w][lane] = count;
+    __syncthreads();
+    if (w == 0 && i < hot_slots) {
+#pragma unroll
+        for (int k = 1; k < FOLD_WARPS; ++k) {
+            const ull s = lo + s_lo[k][lane];
+            hi += s_hi[k][lane] + (s < lo ? 1ull : 0ull);
+            lo = s;
+            count += s_cnt[k][lane];
+        }
+        if ((lo | hi | count) != 0) {
+            const ull key = ~hot_keys[i];
+            table_accumulate(t, key, hash32(key), lo, hi, count);
         }
     }
 }
@@ -939,6 +987,13 @@ cudaError_t launch_hot_build(const HotBuildParams& p, int n_sms, cudaStream_t st
     hot_count_kernel<<<grid, 256, 0, stream>>>(p);
     hot_admit_kernel<<<grid, 256, 0, stream>>>(p);
     hot_select_kernel<<<1, 1024, SELECT_SMEM, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_hot_fold(const ull* hot_keys, ulonglong2* hot_img, uint32_t n_groups, uint32_t hot_slots,
+                            const TableRef& t, cudaStream_t stream) {
+    if (hot_slots == 0) return cudaSuccess;
+    hot_fold_kernel<<<(hot_slots + 31) / 32, FOLD_WARPS * 32, 0, stream>>>(hot_keys, hot_img, n_groups, hot_slots, t);
     return cudaGetLastError();
 }
 

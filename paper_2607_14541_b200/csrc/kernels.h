@@ -15,6 +15,7 @@ struct IngestParams {
     const ull* hot_keys;       // directory image, hot_slots entries of ~key (0 = empty)
     uint32_t hot_slots;        // multiple of 4
     uint32_t hot_buckets;      // hot_slots / 4
+    ulonglong2* hot_img;       // [n_groups][hot_slots] each CTA's directory sums since the last fold, {lo, count | hi << 40}
     TableRef t;
     // spill buffers: entry i of scatter CTA g for partition p at spill + ((g * P + p) * cap + i) * 16 bytes
     unsigned char* spill;
@@ -101,6 +102,8 @@ cudaError_t ingest_prepare();
 cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream);
 cudaError_t launch_partition(const PartitionParams& p, int n_sms, cudaStream_t stream);
 cudaError_t launch_hot_build(const HotBuildParams& p, int n_sms, cudaStream_t stream);
+cudaError_t launch_hot_fold(const ull* hot_keys, ulonglong2* hot_img, uint32_t n_groups, uint32_t hot_slots,
+                            const TableRef& t, cudaStream_t stream);
 cudaError_t launch_merge(const atrex_entry_t* in, ull n, const TableRef& t, int grid, cudaStream_t stream);
 
 cudaError_t finalize_prepare();
