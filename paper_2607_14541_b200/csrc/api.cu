@@ -392,6 +392,7 @@ static int drain_spill(atrex_agg* h, bool force, cudaStream_t s) {
     q.queue_cap = h->L.queue_cap;
     q.force = force ? 1u : 0u;
     q.seq = h->scatter_seq;
+    CU(h, cudaMemsetAsync(&h->ctl->part_cursor, 0, sizeof(ull), s));
     CU(h, launch_partition(q, h->n_sms, s));
     h->launches++;
     if (force && h->hot_dirty) {

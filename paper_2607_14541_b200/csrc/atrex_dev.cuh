@@ -65,7 +65,8 @@ struct Control {
     ull max_fill;              // fullest spill buffer seen since reset (entries)
     ull n_drains;              // partition passes that actually ran
     ull dir_mult;              // multiplier of the hot directory's bucket hash chosen at build time
-    ull pad1[2];
+    ull part_cursor;           // partition pass: next partition to hand out (zeroed before each launch)
+    ull pad1[1];
     ull total_lo[ATREX_MAX_PHASES];
     ull total_hi[ATREX_MAX_PHASES];
     ull keys_per_phase[ATREX_MAX_PHASES];

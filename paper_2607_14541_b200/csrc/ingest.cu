@@ -549,19 +549,33 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     if (!q.force && ld_relaxed(&q.t.ctl->drain_seq) != q.seq) return;
     if (blockIdx.x == 0 && threadIdx.x == 0) atomicAdd(&q.t.ctl->n_drains, 1ull);
 
-    for (uint32_t part = blockIdx.x; part < n_parts; part += gridDim.x) {
+    // Partitions are handed out by a counter (their entry counts differ by a few per cent, and a static
+    // split leaves the kernel waiting for its slowest CTA); a CTA always holds its next partition as
+    // well, so that it can pull that one's keys and entries towards L2 early.
+    __shared__ uint32_t s_next;
+    if (blockIdx.x >= n_parts) return;                             // (never: at least 256 partitions)
+    if (threadIdx.x == 0) s_next = (uint32_t)atomicAdd(&q.t.ctl->part_cursor, 1ull);
+    uint32_t part = blockIdx.x;                                     // the first round is the static one
+    while (part < n_parts) {
+        __syncthreads();  // s_next is set; the previous partition's write-back has finished reading shared memory
+        const uint32_t next = gridDim.x + s_next;                   // the counter starts at 0: partitions >= gridDim
+        __syncthreads();
         if (threadIdx.x == 0) {
             s_total = 0;
             s_qn = 0;
+            s_next = (uint32_t)atomicAdd(&q.t.ctl->part_cursor, 1ull);
         }
-        __syncthreads();  // also: the previous partition's write-back has finished reading shared memory
+        __syncthreads();
         uint32_t local_total = 0;
         for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) local_total += q.spill_cnt[((ull)g << q.t.lp) + part];
         local_total = __reduce_add_sync(0xFFFFFFFFu, local_total);
         if (lane == 0 && local_total) atomicAdd(&s_total, local_total);
 
         __syncthreads();
-        if (s_total == 0) continue;  // nothing was spilled to this partition (uniform)
+        if (s_total == 0) {  // nothing was spilled to this partition (uniform)
+            part = next;
+            continue;
+        }
 
         const ull base = (ull)part * C;
         for (uint32_t i = threadIdx.x; i < C; i += blockDim.x) {
@@ -713,7 +727,6 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
         __syncthreads();
         {   // while the deltas are written back, pull the next partition's keys and each warp's
             // first sub-buffer towards L2 (used within microseconds, so they are still there)
-            const uint32_t next = part + gridDim.x;
             if (next < n_parts) {
                 const unsigned char* nk = reinterpret_cast<const unsigned char*>(q.t.keys + (ull)next * C);
                 for (uint32_t off = threadIdx.x * 128u; off < C * 8u; off += blockDim.x * 128u) prefetch_l2(nk + off);
@@ -754,6 +767,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
         }
         // this partition's buffers are empty again
         for (uint32_t g = threadIdx.x; g < q.n_used; g += blockDim.x) q.spill_cnt[((ull)g << q.t.lp) + part] = 0;
+        part = next;
     }
 }
 
