@@ -590,11 +590,20 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
         }
 
         const ull base = (ull)part * C;
-        for (uint32_t i = threadIdx.x; i < C; i += blockDim.x) {
-            s_keys[i] = q.t.keys[base + i];
-            s_a0[i] = 0;
-            s_a1[i] = 0;
-            s_cnt[i] = 0;
+        for (uint32_t i0 = threadIdx.x; i0 < C; i0 += 4 * blockDim.x) {  // four key loads per thread in flight
+            ull k[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) k[u] = i0 + u * blockDim.x < C ? q.t.keys[base + i0 + u * blockDim.x] : 0ull;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t i = i0 + u * blockDim.x;
+                if (i < C) {
+                    s_keys[i] = k[u];
+                    s_a0[i] = 0;
+                    s_a1[i] = 0;
+                    s_cnt[i] = 0;
+                }
+            }
         }
         {   // the accumulators of this partition are read back at the end: start them towards L2 now
             const unsigned char* vb = reinterpret_cast<const unsigned char*>(q.t.vals + base);
