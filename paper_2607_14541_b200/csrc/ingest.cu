@@ -551,8 +551,11 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     m.a0 = smem_addr(s_a0);
     m.a1 = smem_addr(s_a1);
     m.cnt = smem_addr(s_cnt);
-    __shared__ uint32_t s_total, s_qn;
-    ulonglong2* const my_queue = q.queue + (size_t)blockIdx.x * q.queue_cap;
+    __shared__ uint32_t s_total;
+    // each warp owns a segment of the CTA's queue: no shared counter, and a warp can settle its own
+    // leftovers as soon as its share of the stream is through
+    const uint32_t queue_cap_w = q.queue_cap / (INGEST_THREADS / 32);
+    ulonglong2* const my_queue = q.queue + (size_t)blockIdx.x * q.queue_cap + (size_t)(threadIdx.x >> 5) * queue_cap_w;
     __shared__ unsigned char s_owner[INGEST_THREADS / 32][32];  // in-line fallback, per warp: (round, lane) owning hand-out position t
     const uint32_t n_parts = 1u << q.t.lp;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
@@ -574,7 +577,6 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
         __syncthreads();
         if (threadIdx.x == 0) {
             s_total = 0;
-            s_qn = 0;
             s_next = (uint32_t)atomicAdd(&q.t.ctl->part_cursor, 1ull);
         }
         __syncthreads();
@@ -611,6 +613,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
         }
         __syncthreads();
 
+        uint32_t qn_w = 0;  // entries in this warp's queue segment (warp-uniform)
         for (uint32_t g = warp; g < q.n_used; g += n_warps) {
             const ull sb = ((ull)g << q.t.lp) + part;
             const uint32_t n_e = q.spill_cnt[sb];
@@ -673,12 +676,11 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                     total += __popc(pend[u]);
                 }
                 if (total != 0) {
-                    uint32_t qbase = 0;
-                    if (lane == 0) qbase = atomicAdd(&s_qn, total);
-                    qbase = __shfl_sync(0xFFFFFFFFu, qbase, 0);
+                    uint32_t qbase = qn_w;
+                    qn_w = min(qn_w + total, queue_cap_w);
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        if (searching[u] && qbase + before[u] < q.queue_cap) {
+                        if (searching[u] && qbase + before[u] < queue_cap_w) {
                             my_queue[qbase + before[u]] = make_ulonglong2(~skey[u], v[u]);
                             searching[u] = false;
                             ok[u] = false;
@@ -687,7 +689,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                     // Queue full (a partition made of new keys only): settle the remainder in line.
                     // The pending entries are handed out one per lane: each one's owner publishes
                     // (round, lane) at the entry's position; lane t serves position t.
-                    while (qbase + total > q.queue_cap) {
+                    while (qbase + total > queue_cap_w) {
                         total = 0;
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
@@ -696,7 +698,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                             total += __popc(pend[u]);
                         }
                         if (total == 0) break;
-                        qbase = q.queue_cap;  // stay in this loop until nothing is pending
+                        qbase = queue_cap_w;  // stay in this loop until nothing is pending
 #pragma unroll
                         for (int u = 0; u < 4; ++u)
                             if (searching[u] && before[u] < 32) s_owner[warp][before[u]] = (unsigned char)((u << 5) | lane);
@@ -733,11 +735,11 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                     if (ok[u]) part_accumulate(m, slot[u], v[u], q.t.vals + base);
             }
         }
-        __syncthreads();
-        {   // the queued entries, one per lane
-            const uint32_t qn = min(s_qn, q.queue_cap);
-            for (uint32_t i0 = warp * 32u; i0 < qn; i0 += n_warps * 32u) {
-                const bool serving = i0 + lane < qn;
+        {   // this warp's queued entries, one per lane (other warps may still be streaming: the general
+            // probe copes with keys appearing meanwhile)
+            __syncwarp();
+            for (uint32_t i0 = 0; i0 < qn_w; i0 += 32u) {
+                const bool serving = i0 + lane < qn_w;
                 const ulonglong2 ent = serving ? __ldcg(my_queue + i0 + lane) : make_ulonglong2(0, 0);
                 const uint32_t hh = hash32(ent.x);
                 const uint32_t start = local_of(hh, (uint32_t)(ent.x >> 48), C) & ~1u;
