@@ -479,8 +479,8 @@ __global__ void __launch_bounds__(FOLD_WARPS * 32) hot_fold_kernel(const ull* ho
 // is processed, the next one's keys and spill entries are pulled into L2.  Per partition: copy the
 // keys in; stream the entries of all scatter CTAs, four per lane, and settle each with one look at
 // the first pair of its probe sequence (hit, or a new key with room there); entries that need more
-// than that wait in a per-CTA queue in global memory and are settled, 32 per warp round, once the
-// stream is through; then write the deltas back.
+// than that wait in the warp's segment of a per-CTA queue in global memory and are settled, 32 per
+// round, once the warp's share of the stream is through; then write the deltas back.
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 // Shared-window addresses of the partition pass's arrays.
