@@ -31,9 +31,9 @@ if ROOT not in sys.path:
 
 METRIC = "trace records aggregated/sec"
 # DRAM bytes (read + written) per 2^27-record ingest call of this workload, from the ncu captures
-# summarised under profiles/: scatter_kernel 4.43 GB per launch plus
-# the two real partition drains of a step (12.16 GB) spread over its eight calls.
-NCU_DRAM_BYTES_PER_INGEST_CALL = 5.95e9
+# summarised under profiles/: scatter_kernel 4.47 GB per launch plus
+# the two real partition drains of a step (12.20 GB) spread over its eight calls.
+NCU_DRAM_BYTES_PER_INGEST_CALL = 5.99e9
 UNIT = "records/s"
 WORKLOAD_INDEX = 3
 RECORD_BYTES = 16
