@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(TOT_THREADS) totals_kernel(TableRef tab, ull n
 #pragma unroll
         for (int u = 0; u < ILP; ++u) sk[u] = i0 + u * stride < n_slots ? tab.keys[i0 + u * stride] : 0ull;
 #pragma unroll
-        for (int u = 0; u < ILP; ++u) x[u] = sk[u] != 0 ? tab.vals[i0 + u * stride] : make_ulonglong2(0, 0);
+        for (int u = 0; u < ILP; ++u) x[u] = i0 + u * stride < n_slots ? tab.vals[i0 + u * stride] : make_ulonglong2(0, 0);  // unconditional: no wait for the keys
 #pragma unroll
         for (int u = 0; u < ILP; ++u) {
             if (sk[u] == 0) continue;
@@ -155,20 +155,21 @@ __global__ void __launch_bounds__(FIN_THREADS) emit_kernel(FinalizeParams p) {
     const ull rounds = (p.n_slots + stride * EMIT_ILP - 1) / (stride * EMIT_ILP);  // uniform: warps stay converged
     for (ull r = 0; r < rounds; ++r) {
         ull sk[EMIT_ILP];
+        ulonglong2 xv[EMIT_ILP];
 #pragma unroll
         for (int u = 0; u < EMIT_ILP; ++u) {
             const ull i = (r * EMIT_ILP + u) * stride + (ull)blockIdx.x * blockDim.x + threadIdx.x;
             sk[u] = i < p.n_slots ? p.t.keys[i] : 0ull;
+            xv[u] = i < p.n_slots ? p.t.vals[i] : make_ulonglong2(0, 0);  // with the key, not after it
         }
         uint32_t total = 0;
 #pragma unroll
         for (int u = 0; u < EMIT_ILP; ++u) {
             const unsigned live = __ballot_sync(0xFFFFFFFFu, sk[u] != 0);
             if (sk[u] != 0) {
-                const ull i = (r * EMIT_ILP + u) * stride + (ull)blockIdx.x * blockDim.x + threadIdx.x;
                 const uint32_t at = total + __popc(live & ((1u << lane) - 1u));
                 q_key[w][at] = ~sk[u];
-                q_val[w][at] = p.t.vals[i];
+                q_val[w][at] = xv[u];
             }
             total += __popc(live);
         }
@@ -303,10 +304,12 @@ __global__ void __launch_bounds__(1024) topk_hist_all_kernel(const __grid_consta
         for (int u = 0; u < ILP; ++u) sk[u] = i0 + u * stride < p.n_slots ? p.t.keys[i0 + u * stride] : 0ull;
 #pragma unroll
         for (int u = 0; u < ILP; ++u) {
+            x[u] = i0 + u * stride < p.n_slots ? p.t.vals[i0 + u * stride] : make_ulonglong2(0, 0);  // no wait for the keys
+        }
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) {
             const uint32_t q = (uint32_t)(~sk[u] >> 48) & (ATREX_MAX_PHASES - 1);
-            const bool mine = sk[u] != 0 && ((p.active_mask >> q) & 1u);
-            x[u] = mine ? p.t.vals[i0 + u * stride] : make_ulonglong2(0, 0);
-            if (!mine) sk[u] = 0;
+            if (!(sk[u] != 0 && ((p.active_mask >> q) & 1u))) sk[u] = 0;
         }
 #pragma unroll
         for (int u = 0; u < ILP; ++u) {
@@ -337,10 +340,12 @@ __global__ void __launch_bounds__(FIN_THREADS) topk_collect_all_kernel(const __g
         for (int u = 0; u < ILP; ++u) sk[u] = i0 + u * stride < p.n_slots ? p.t.keys[i0 + u * stride] : 0ull;
 #pragma unroll
         for (int u = 0; u < ILP; ++u) {
+            x[u] = i0 + u * stride < p.n_slots ? p.t.vals[i0 + u * stride] : make_ulonglong2(0, 0);  // no wait for the keys
+        }
+#pragma unroll
+        for (int u = 0; u < ILP; ++u) {
             const uint32_t q = (uint32_t)(~sk[u] >> 48) & (ATREX_MAX_PHASES - 1);
-            const bool mine = sk[u] != 0 && ((p.active_mask >> q) & 1u);
-            x[u] = mine ? p.t.vals[i0 + u * stride] : make_ulonglong2(0, 0);
-            if (!mine) sk[u] = 0;
+            if (!(sk[u] != 0 && ((p.active_mask >> q) & 1u))) sk[u] = 0;
         }
 #pragma unroll
         for (int u = 0; u < ILP; ++u) {
