@@ -42,6 +42,10 @@ def lib():
         L.oracle_ingest_threads.restype = C.c_uint32
         L.oracle_ingest_threads.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint32]
         L.oracle_ingest_filtered.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint64]
+        L.oracle_ingest_slice.restype = C.c_uint32
+        L.oracle_ingest_slice.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint32]
+        L.oracle_slice_classes.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p]
+        L.oracle_finalize_given_totals.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p]
         L.oracle_direct_totals.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p]
         L.oracle_set_work.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
         L.oracle_n_keys.restype = C.c_uint64
@@ -101,6 +105,26 @@ class Oracle:
         k = np.ascontiguousarray(keys, dtype=np.uint64)
         lib().oracle_ingest_filtered(self._h, r.ctypes.data, r.shape[0], k.ctypes.data, k.shape[0])
 
+    def ingest_slice(self, records: np.ndarray, modulus: int, residue: int, threads: int = 0) -> int:
+        """Aggregate only the valid records whose key's slice class (a fixed scramble of the key,
+        modulo ``modulus``) equals ``residue``; returns the threads used."""
+        r = np.ascontiguousarray(records)
+        assert r.dtype.itemsize == 16
+        return lib().oracle_ingest_slice(self._h, r.ctypes.data, r.shape[0], modulus, residue, threads)
+
+    def finalize_given_totals(self, peak_bw: float, peak_flops, totals) -> np.ndarray:
+        """Entries of this handle's keys with Eq. 3's denominators taken from ``totals`` (ints, one per phase)."""
+        n = self.n_keys()
+        out = np.zeros(n, dtype=ENTRY_DTYPE)
+        n_out = C.c_uint64(0)
+        pk = _peaks_buf(peak_bw, peak_flops)
+        t = np.zeros(16, dtype=np.uint64)
+        for q, v in enumerate(list(totals)[:8]):
+            t[2 * q], t[2 * q + 1] = v & 0xFFFFFFFFFFFFFFFF, v >> 64
+        rc = lib().oracle_finalize_given_totals(self._h, pk.ctypes.data, t.ctypes.data, out.ctypes.data, n, C.byref(n_out))
+        assert rc == 0 and n_out.value == n
+        return out
+
     def direct_totals(self, records: np.ndarray, acc: np.ndarray, valid: np.ndarray) -> None:
         """acc: uint64[16] (lo, hi per phase), valid: uint64[2]; both updated in place."""
         r = np.ascontiguousarray(records)
@@ -136,6 +160,14 @@ class Oracle:
         pk = _peaks_buf(peak_bw, peak_flops)
         lib().oracle_topk(self._h, pk.ctypes.data, phase, k, out.ctypes.data, C.byref(n_out))
         return out[:n_out.value].copy()
+
+
+def slice_class(keys, modulus: int) -> np.ndarray:
+    """Slice class of each key, as ``Oracle.ingest_slice`` assigns it."""
+    k = np.ascontiguousarray(keys, dtype=np.uint64)
+    out = np.zeros(k.shape[0], dtype=np.uint64)
+    lib().oracle_slice_classes(k.ctypes.data, k.shape[0], modulus, out.ctypes.data)
+    return out
 
 
 def u128_to_f64(x: int) -> float:

@@ -228,6 +228,63 @@ void oracle_ingest_filtered(void* h, const void* records, uint64_t n, const uint
     }
 }
 
+// Full-size slice checks.  The key space is cut into `modulus` classes by a fixed scramble of the
+// packed key (a function of the key alone -- nothing here looks at anybody's output), and only the
+// valid records whose key falls into class `residue` are aggregated: the same definition as
+// oracle_ingest restricted to a slice of the key space, so that a trace too large for the full map
+// can still be compared entry by entry on that slice, lost and invented keys included.
+// Threads aggregate contiguous runs of the records into their own maps, merged by key with integer
+// adds as in oracle_ingest_threads.  Returns the number of threads used.
+inline uint64_t slice_class(uint64_t key, uint64_t modulus) {
+    uint64_t z = key + 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    return z % modulus;
+}
+
+uint32_t oracle_ingest_slice(void* h, const void* records, uint64_t n, uint64_t modulus, uint64_t residue,
+                             uint32_t threads) {
+    Oracle* o = (Oracle*)h;
+    if (modulus == 0) return 0;
+    if (threads == 0) threads = std::thread::hardware_concurrency();
+    if (threads == 0) threads = 1;
+    if (n < threads) threads = 1;
+    std::vector<Groups> parts(threads);
+    std::vector<std::thread> pool;
+    const Rec* recs = (const Rec*)records;
+    for (uint32_t t = 0; t < threads; ++t) {
+        uint64_t lo = n * t / threads, hi = n * (t + 1) / threads;
+        pool.emplace_back([&, t, lo, hi] {
+            Groups& g = parts[t];
+            for (uint64_t i = lo; i < hi; ++i) {
+                const Rec& r = recs[i];
+                if (r.app_id >= o->n_apps || r.phase >= o->n_phases) continue;
+                uint64_t k = pack_key(r);
+                if (slice_class(k, modulus) != residue) continue;
+                Acc& a = g[k];
+                a.count += 1;
+                a.wt += (u128)o->app_weight[r.app_id] * (u128)r.duration_ns;
+            }
+        });
+    }
+    for (auto& th : pool) th.join();
+    for (uint32_t t = 0; t < threads; ++t) {
+        for (const auto& kv : parts[t]) {
+            Acc& a = o->groups[kv.first];
+            a.count += kv.second.count;
+            a.wt += kv.second.wt;
+        }
+    }
+    return threads;
+}
+
+// The class oracle_ingest_slice puts a key in (exported so that a test can cut another
+// implementation's output along the same lines).
+void oracle_slice_classes(const uint64_t* keys, uint64_t n, uint64_t modulus, uint64_t* out) {
+    for (uint64_t i = 0; i < n; ++i) out[i] = modulus ? slice_class(keys[i], modulus) : 0;
+}
+
 // Per-phase totals straight from the records, without any grouping: Eq. 2's D^phi as a plain
 // sum.  acc[2p], acc[2p+1] (low, high) are updated in place so the call can be repeated per
 // chunk; valid[0] / valid[1] accumulate the valid and rejected record counts.
@@ -292,6 +349,23 @@ int oracle_finalize(void* h, const void* peaks, void* out, uint64_t cap, uint64_
     if (cap < o->groups.size()) return -1;
     u128 totals[8];
     phase_totals(*o, totals);
+    Entry* e = (Entry*)out;
+    uint64_t i = 0;
+    for (const auto& kv : o->groups) e[i++] = make_entry(*o, pk, totals, kv.first, kv.second);
+    return 0;
+}
+
+// As oracle_finalize, but Eq. 3's per-phase denominators are given (totals[2p], totals[2p+1] = low
+// and high 64 bits of T[p]) instead of summed over this handle's own keys: used when the handle
+// holds only a slice of the key space and the totals come from oracle_direct_totals.
+int oracle_finalize_given_totals(void* h, const void* peaks, const uint64_t totals_in[16], void* out, uint64_t cap,
+                                 uint64_t* n_out) {
+    Oracle* o = (Oracle*)h;
+    const Peaks& pk = *(const Peaks*)peaks;
+    *n_out = o->groups.size();
+    if (cap < o->groups.size()) return -1;
+    u128 totals[8];
+    for (int p = 0; p < 8; ++p) totals[p] = ((u128)totals_in[2 * p + 1] << 64) | totals_in[2 * p];
     Entry* e = (Entry*)out;
     uint64_t i = 0;
     for (const auto& kv : o->groups) e[i++] = make_entry(*o, pk, totals, kv.first, kv.second);

@@ -55,13 +55,21 @@ bool config_ok(const atrex_agg_config_t* c) {
 }
 
 void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, Layout* L) {
-    // partition geometry: one partition's keys + per-launch accumulators (20 B per slot) must
-    // fit one SM's shared memory; provision 1.3 slots per key
+    // Partition geometry: one partition's keys + per-launch accumulators (20 B per slot) must fit one
+    // SM's shared memory.  A key can only live in its hash partition, so a partition is sized for the
+    // tail of its load, not for the mean: with m = max_keys / P keys expected, the keys of one
+    // (operator, shape) -- up to n_phases of them -- always fall together, which bounds the standard
+    // deviation by sqrt(n_phases * m); six of those plus a constant, and never less than 1.3 m.
     const uint32_t c_max = (uint32_t)((smem_optin - 2048) / 20) & ~127u;
-    const ull need = c->max_keys + c->max_keys * 3 / 10 + 1;
+    auto slots_for = [&](uint32_t lp) -> ull {
+        const ull m = (c->max_keys + (1ull << lp) - 1) >> lp;
+        const ull flat = m + m * 3 / 10 + 1;
+        const ull tail = m + (ull)std::ceil(6.0 * std::sqrt((double)c->n_phases * (double)m)) + 32;
+        return flat > tail ? flat : tail;
+    };
     L->lp = LP_MIN;
-    while (L->lp < LP_MAX && (need + (1ull << L->lp) - 1) / (1ull << L->lp) > c_max) ++L->lp;
-    ull per = (need + (1ull << L->lp) - 1) >> L->lp;
+    while (L->lp < LP_MAX && slots_for(L->lp) > c_max) ++L->lp;
+    ull per = slots_for(L->lp);
     if (per > c_max || L->lp > LP_MIN) per = c_max;  // big tables: use all of shared memory, lower load factor
     if (per < 128) per = 128;
     L->C = (uint32_t)((per + 31) / 32 * 32);

@@ -7,8 +7,9 @@
 //                              are counted), cnthi = count in bits 0..39, number of wraps of
 //                              `lo` plus merged high words in bits 40..63
 //                              (count < 2^40, weighted time < 2^88)
-//                 A key lives in partition hash >> (64 - log2 P), at a slot found by linear
-//                 probing inside that partition only.  C is chosen so that one partition's
+//                 A key lives in the partition given by the top log2 P bits of its 32-bit hash, at
+//                 a slot found by double hashing over slot pairs inside that partition only (see
+//                 find_or_claim below).  C is chosen so that one partition's
 //                 keys and per-launch accumulators fit in one SM's shared memory: the
 //                 aggregation pass owns a partition per CTA and needs no global atomics.
 //   spill bufs  : [G][P][cap] 16-byte {key, weighted duration} entries and [G][P] counts,

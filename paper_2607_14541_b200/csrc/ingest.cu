@@ -14,8 +14,10 @@
 //     buffer for the key's partition.  Appends of one (CTA, partition) pair are sequential in
 //     memory; the next 128-byte line of a buffer is prefetched into L2 shortly before the
 //     appends reach it, because a partial store into a line that is not cached stalls on a fill.
-//   At the end the CTA adds its directory accumulators to the table (these few thousand slots
-//   stay L2-resident) and stores its per-partition cursors: the buffers persist across launches.
+//   At the end the CTA adds its directory accumulators to its own row of a directory image
+//   ([CTA][slot], plain coalesced read-modify-writes; hot_fold_kernel adds the rows into the table
+//   before results are read) and stores its per-partition cursors: the buffers persist across
+//   launches.
 //
 // Pass 2  PARTITION  (persistent CTAs, one partition at a time each).  Runs lazily: only when a
 //   buffer is filling up, or when results are about to be read.  The CTA copies its

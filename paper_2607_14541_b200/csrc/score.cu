@@ -11,6 +11,8 @@
 // the result has one bit pattern.  The median is found by ranking (each value's rank is the
 // number of values that sort before it, ties broken by position), which needs no sorting
 // network and no scratch memory beyond the CTA's shared memory.
+#include <mutex>
+
 #include "kernels.h"
 
 using namespace atrex;
@@ -109,6 +111,25 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_kernel(const double* __re
     }
 }
 
+constexpr int SCORE_MAX_DEVICES = 64;
+std::mutex g_score_lock;
+bool g_score_prepared[SCORE_MAX_DEVICES];   // per device: the kernel's shared-memory limit has been raised
+
+struct ScoreDeviceGuard {
+    int prev = -1;
+    bool switched = false, ok = true;
+    explicit ScoreDeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != dev) {
+            switched = cudaSetDevice(dev) == cudaSuccess;
+            ok = switched;
+        }
+    }
+    ~ScoreDeviceGuard() {
+        if (switched && prev >= 0) cudaSetDevice(prev);
+    }
+};
+
 }  // namespace
 
 extern "C" int atrex_score_aggregate(const double* d_roofline_s, const uint32_t* d_unit_op, uint64_t n_units,
@@ -121,13 +142,27 @@ extern "C" int atrex_score_aggregate(const double* d_roofline_s, const uint32_t*
     if (n_units > ATREX_SCORE_MAX_UNITS || n_ops > ATREX_SCORE_MAX_OPS || n_candidates > 0x7FFFFFFFull)
         return ATREX_ERR_TOO_LARGE;
     const size_t smem = (size_t)n_units * 8 + (size_t)n_ops * 8 + ((size_t)2 * n_ops + 1) * 4;
-    static bool prepared = false;
-    if (!prepared) {
-        if (cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
-            cudaGetLastError();
-            return ATREX_ERR_CUDA;
+    // the inputs live on some device: run there, and raise that device's shared-memory limit once
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, d_t_cand) != cudaSuccess || attr.type != cudaMemoryTypeDevice || attr.device < 0 ||
+        attr.device >= SCORE_MAX_DEVICES) {
+        cudaGetLastError();
+        return ATREX_ERR_INVALID;
+    }
+    ScoreDeviceGuard guard(attr.device);
+    if (!guard.ok) {
+        cudaGetLastError();
+        return ATREX_ERR_CUDA;
+    }
+    {
+        std::lock_guard<std::mutex> hold(g_score_lock);
+        if (!g_score_prepared[attr.device]) {
+            if (cudaFuncSetAttribute(score_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) {
+                cudaGetLastError();
+                return ATREX_ERR_CUDA;
+            }
+            g_score_prepared[attr.device] = true;
         }
-        prepared = true;
     }
     score_kernel<<<(unsigned)n_candidates, SCORE_THREADS, smem, (cudaStream_t)stream>>>(
         d_roofline_s, d_unit_op, (uint32_t)n_units, d_t_cand, d_correct, d_w, n_ops, d_s_agg, d_s_op,

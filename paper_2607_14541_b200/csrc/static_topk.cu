@@ -32,9 +32,13 @@ unsigned char* g_scratch_addr[MAX_DEVICES];  // per device, filled on that devic
 struct DeviceGuard {
     int prev = -1;
     bool switched = false;
+    bool ok = true;   // false: `dev` could not be made current, nothing may run
     explicit DeviceGuard(int dev) {
         if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
-        if (prev != dev) switched = cudaSetDevice(dev) == cudaSuccess;
+        if (prev != dev) {
+            switched = cudaSetDevice(dev) == cudaSuccess;
+            ok = switched;
+        }
     }
     ~DeviceGuard() {
         if (switched && prev >= 0) cudaSetDevice(prev);
@@ -84,6 +88,10 @@ extern "C" int atrex_topk_entries_static(const atrex_entry_t* d_entries, uint64_
     const int dev = attr.device;
     if (dev < 0 || dev >= MAX_DEVICES) return ATREX_ERR_INVALID;
     DeviceGuard guard(dev);
+    if (!guard.ok) {   // resolving the array's address with another device current would cache a wrong address
+        cudaGetLastError();
+        return ATREX_ERR_CUDA;
+    }
     cudaStream_t s = (cudaStream_t)stream;
 
     unsigned char* scratch;

@@ -402,3 +402,26 @@ def test_crowded_small_partitions_overflow_the_deferred_queue(lib):
     assert st["table_slots"] == 256 * 128 and st["n_spilled"] == n and st["n_overflow"] == 0
     o = oracle_of(recs, weights, 2, threads=16)
     assert_same_as_oracle(agg, o, 2)
+
+
+@pytest.mark.parametrize("max_keys", [23_000, 25_000, 31_500, 50_000])
+def test_table_filled_exactly_to_max_keys(lib, max_keys):
+    """A caller who stays within max_keys must never see ATREX_ERR_CAPACITY: a key can only live in
+    its hash partition, so partitions are sized for the tail of their load.  These sizes sit where a
+    flat 1.3 slots per key left the fullest partition of a random key set short in a third of the
+    cases; both phases of every (operator, shape) are present, which widens the spread further."""
+    rng = np.random.default_rng(max_keys)
+    pairs = np.unique(rng.integers(0, 1 << 40, size=max_keys, dtype=np.uint64))[: max_keys // 2]
+    recs = np.zeros(2 * len(pairs) * 2, dtype=RECORD_DTYPE)          # every key twice
+    recs["op_id"] = np.tile((pairs >> np.uint64(24)).astype(np.uint16), 4)
+    recs["shape_id"] = np.tile((pairs & np.uint64(0xFFFFFF)).astype(np.uint32) * np.uint32(2654435761), 4)
+    recs["phase"] = np.repeat(np.array([0, 1, 0, 1], dtype=np.uint8), len(pairs))
+    recs["app_id"] = rng.integers(0, 4, size=len(recs))
+    recs["duration_ns"] = rng.integers(1, 1 << 28, size=len(recs))
+    rng.shuffle(recs)
+    weights = np.array([1, 7, 1000, (1 << 20) - 1], dtype=np.uint32)
+    o = oracle_of(recs, weights, 2)
+    n_keys = o.stats()["n_keys"]
+    assert n_keys == 2 * len(pairs) and max_keys - 1 <= n_keys <= max_keys
+    agg = gpu_aggregate(lib, recs, weights, 2, max_keys=n_keys)
+    assert_same_as_oracle(agg, o, 2)

@@ -306,6 +306,46 @@ def test_filtered_and_direct_totals_agree_with_the_full_group_by():
     assert int(valid[0]) == len(recs) - 3 and int(valid[1]) == 3 == rejected
 
 
+def test_slice_ingest_is_the_full_group_by_cut_along_key_classes():
+    """ingest_slice against brute force: the classes partition the key space (every key of the
+    brute-force result turns up in exactly one class, with its count and weighted time), the class
+    of a key does not depend on which records carry it, threads and chunking do not matter, and
+    finalize_given_totals reproduces the full oracle's entries bit for bit when handed the totals
+    that direct_totals sums from the records."""
+    spec = make_spec(1, small=True, n=1 << 16)
+    recs = tg.generate(spec)
+    recs[5:9]["phase"] = spec.n_phases          # invalid records must not reach any slice
+    work = spec.work_table()
+    _, full = run_oracle(recs, spec.app_weights, spec.n_phases, work)
+    groups, totals, rejected = brute_force(recs, spec.app_weights, spec.n_phases)
+    modulus = 7
+    classes = oracle.slice_class(full["key"], modulus)
+    assert set(int(c) for c in classes) == set(range(modulus))
+    seen = {}
+    for r in range(modulus):
+        o = oracle.Oracle(spec.app_weights, spec.n_phases)
+        o.set_work(work)
+        for c, th in zip(np.array_split(recs, 3), (1, 3, 2)):
+            assert o.ingest_slice(c, modulus, r, threads=th) == th
+        acc, valid = np.zeros(16, dtype=np.uint64), np.zeros(2, dtype=np.uint64)
+        o.direct_totals(recs, acc, valid)
+        assert int(valid[1]) == rejected == 4
+        got = o.finalize_given_totals(PEAK_BW, PEAK_FLOPS, totals)
+        assert got.tobytes() == full[classes == r].tobytes()       # both key-ascending
+        for e in got:
+            k = int(e["key"])
+            assert k not in seen and [int(e["count"]), entry_wt(e)] == list(groups[k])
+            seen[k] = r
+    assert len(seen) == len(groups)
+    # a second look at the scramble itself: restated with Python integers
+    def py_class(key, m):
+        z = (key + 0x9E3779B97F4A7C15) & (2**64 - 1)
+        z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & (2**64 - 1)
+        z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & (2**64 - 1)
+        return (z ^ (z >> 31)) % m
+    assert [py_class(int(k), 64) for k in full["key"][:200]] == [int(c) for c in oracle.slice_class(full["key"][:200], 64)]
+
+
 # ---------------------------------------------------------------- score aggregation (Eq. 4-6)
 
 def test_score_worked_example(golden_dir):
