@@ -22,7 +22,6 @@ constexpr uint32_t HOT_SAMPLE = 1u << 20;
 constexpr uint32_t CAND_BITS = 17;                     // candidate table of the directory build
 constexpr size_t SKETCH_BYTES = (size_t)4 << 20;        // 2^20 counters (ingest.cu SKETCH_BITS)
 constexpr size_t HOT_SCRATCH_BYTES = SKETCH_BYTES + ((size_t)12 << CAND_BITS);
-constexpr uint32_t APPW_SMEM_MAX = 4096;
 constexpr uint32_t SEL_CAP = ATREX_MAX_TOPK + TOPK_CAND_CAP;
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -81,6 +80,7 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     // workload (half of the records spill) four launches accumulate between drains.
     ull per_buf = (L->sub_launch * 9 / 2) / (((ull)n_sms) << L->lp);
     if (per_buf < 64) per_buf = 64;
+    if (per_buf > 32768) per_buf = 32768;   // the scatter pass counts a buffer's entries in 16 bits, with headroom
     L->cap = (uint32_t)((per_buf + 7) / 8 * 8);
     // entries of one partition whose first look fails wait in a per-CTA queue: room for a quarter of
     // the partition's worst-case stream, at most 32 K entries (the rest is settled in line)
@@ -92,10 +92,7 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     L->Cw = c->max_work_rows ? (uint32_t)((((c->max_work_rows * 3 / 2) >> L->lp) + 64 + 31) / 32 * 32) : 0;
     L->work_slots = (ull)L->Cw << L->lp;
     L->appw_in_smem = c->n_apps <= APPW_SMEM_MAX;
-    size_t appw_smem = L->appw_in_smem ? (size_t)c->n_apps * 4 : 0;
-    size_t fixed = appw_smem + 2048 + ((size_t)4 << L->lp);
-    size_t budget = smem_optin > fixed ? smem_optin - fixed : 0;
-    L->hot_slots = (uint32_t)(budget / 21) & ~15u;  // 21 B per slot in the scatter pass; whole buckets, aligned arrays
+    L->hot_slots = scatter_hot_slots(L->lp);   // what the scatter pass's shared memory holds for this partition count
     if (c->flags & ATREX_FLAG_NO_HOT_DIRECTORY) L->hot_slots = 0;
     size_t o = 0;
     L->off_ctl = o;            o += round_up(sizeof(Control), ALIGN);
@@ -439,6 +436,8 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
     const unsigned char* base = (const unsigned char*)recs;
     uint64_t head = (((uintptr_t)base & 31u) != 0 && n > 0) ? 1 : 0;
     uint64_t n_body = n - head;
+    p.recs = recs;
+    p.n_recs = n;
     p.body = base + head * 16;
     p.n_pairs = n_body / 2;
     p.n_single = 0;
@@ -446,6 +445,7 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
     if (n_body & 1) p.single[p.n_single++] = base + (n - 1) * 16;
     p.n_apps = h->cfg.n_apps;
     p.n_phases = h->cfg.n_phases;
+    p.phase_lim = h->cfg.n_phases << 16;
     p.appw_in_smem = h->L.appw_in_smem ? 1u : 0u;
     p.app_w = h->d_appw;
     p.hot_keys = h->hot_keys;

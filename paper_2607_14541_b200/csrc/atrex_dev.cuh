@@ -90,6 +90,18 @@ __device__ __forceinline__ uint32_t hash32(uint32_t op, uint32_t shape) {
 }
 __device__ __forceinline__ uint32_t hash32(ull key) { return hash32((uint32_t)(key >> 32) & 0xFFFFu, (uint32_t)key); }
 
+// Placement of a key in the scatter pass's hot directory: the high bits of the mixed hash choose the
+// bucket, its low byte is the slot's tag.  The odd multiplier is picked per directory build so that
+// as little sampled weight as possible is lost to crowded buckets.  The table hash `h` leaves the
+// phase out, the directory must not: the phases of a hot (operator, shape) are usually all hot and
+// would otherwise fight over one bucket.
+__device__ __forceinline__ uint32_t dir_mix(uint32_t h, uint32_t phase, uint32_t mult) {
+    return (h + phase * 0x9E3779B9u) * mult;
+}
+__device__ __forceinline__ uint32_t dir_bucket(uint32_t h, uint32_t phase, uint32_t mult, uint32_t n_buckets) {
+    return __umulhi(dir_mix(h, phase, mult), n_buckets);
+}
+
 __device__ __forceinline__ ull pack_key(uint32_t phase, uint32_t op, uint32_t shape) {
     return ((ull)phase << 48) | ((ull)op << 32) | (ull)shape;
 }

@@ -1,23 +1,12 @@
-// Ingest: Eq. 2's group-by sum, streamed, as a two-pass radix-partitioned aggregation.
+// Ingest, everything but the scatter pass (scatter.cu): Eq. 2's group-by sum, streamed, as a
+// two-pass radix-partitioned aggregation.
 //
 // Random read-modify-write into a table far larger than L2 is bound by DRAM latency and by
 // the L2's atomic rate, not by bandwidth, so the hot path avoids global atomics altogether:
 //
-// Pass 1  SCATTER  (one persistent CTA per SM).  Each thread pulls records with 32-byte
-//   vector loads (two 16-byte records per load, several loads in flight, streaming cache
-//   policy), packs the key and multiplies the application's card-hour weight by the duration.
-//   * Keys found in the shared-memory HOT DIRECTORY (the most frequent keys of a sample of the
-//     trace, identical in every CTA, read-only during the pass) are accumulated on the spot
-//     with 32-bit shared-memory atomics in limbs with explicit carries; lanes of a warp that
-//     hit the same slot are first combined with warp reductions.
-//   * Every other record becomes a 16-byte {key, product} entry appended to the CTA's private
-//     buffer for the key's partition.  Appends of one (CTA, partition) pair are sequential in
-//     memory; the next 128-byte line of a buffer is prefetched into L2 shortly before the
-//     appends reach it, because a partial store into a line that is not cached stalls on a fill.
-//   At the end the CTA adds its directory accumulators to its own row of a directory image
-//   ([CTA][slot], plain coalesced read-modify-writes; hot_fold_kernel adds the rows into the table
-//   before results are read) and stores its per-partition cursors: the buffers persist across
-//   launches.
+// Pass 1  SCATTER  (scatter.cu) accumulates the records of hot keys in a shared-memory directory
+//   and appends every other record as a 16-byte {key, product} entry to the CTA's private buffer
+//   of the key's partition.
 //
 // Pass 2  PARTITION  (persistent CTAs, one partition at a time each).  Runs lazily: only when a
 //   buffer is filling up, or when results are about to be read.  The CTA copies its
@@ -41,18 +30,6 @@ constexpr uint32_t NO_SLOT = 0xFFFFFFFFu;
 constexpr uint32_t DIR_WAYS = 4;                   // slots per hot-directory bucket (32 bytes of keys)
 constexpr uint32_t NEW_KEY_FLAG = 0x80000000u;     // partition pass: slot claimed in this launch
 
-// Bucket of the hot directory.  The odd multiplier is picked per build among DIR_MULTS so that
-// as little sampled weight as possible is lost to buckets that more than two hot keys map to.
-// The table hash `h` leaves the phase out, the directory must not: the phases of a hot
-// (operator, shape) are usually all hot and would otherwise fight over one bucket.
-// Directory placement of a key: the high bits of the mixed hash choose the bucket, its low byte is
-// the slot's tag.
-__device__ __forceinline__ uint32_t dir_mix(uint32_t h, uint32_t phase, uint32_t mult) {
-    return (h + phase * 0x9E3779B9u) * mult;
-}
-__device__ __forceinline__ uint32_t dir_bucket(uint32_t h, uint32_t phase, uint32_t mult, uint32_t n_buckets) {
-    return __umulhi(dir_mix(h, phase, mult), n_buckets);
-}
 __device__ __forceinline__ uint32_t dir_bucket_of_key(ull key, uint32_t mult, uint32_t n_buckets) {
     return dir_bucket(hash32(key), (uint32_t)(key >> 48), mult, n_buckets);
 }
@@ -98,29 +75,31 @@ __device__ __forceinline__ uint32_t atoms_exch(uint32_t a, uint32_t v) {
     asm volatile("atom.shared.exch.b32 %0, [%1], %2;" : "=r"(o) : "r"(a), "r"(v) : "memory");
     return o;
 }
+__device__ __forceinline__ uint32_t lds_u32_volatile(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_v2u64(uint32_t a, ull x, ull y) {
+    asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(a), "l"(x), "l"(y) : "memory");
+}
+// zero, in a form the compiler cannot fold: makes one instruction's operand depend on a loaded value
+__device__ __forceinline__ uint32_t zero_after(ull loaded) {
+    uint32_t z;
+    asm volatile("and.b32 %0, %1, 0;" : "=r"(z) : "r"((uint32_t)loaded));
+    return z;
+}
+__device__ __forceinline__ void stg_sector(void* at, ull a, ull b, ull c, ull d) {
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(at), "r"((uint32_t)a), "r"((uint32_t)(a >> 32)),
+                 "r"((uint32_t)b), "r"((uint32_t)(b >> 32)), "r"((uint32_t)c), "r"((uint32_t)(c >> 32)), "r"((uint32_t)d),
+                 "r"((uint32_t)(d >> 32))
+                 : "memory");
+}
 __device__ __forceinline__ ull atoms_cas64(uint32_t a, ull expected, ull desired) {
     ull o;
     asm volatile("atom.shared.cas.b64 %0, [%1], %2, %3;" : "=l"(o) : "r"(a), "l"(expected), "l"(desired) : "memory");
     return o;
 }
-
-// Shared-window byte addresses of the scatter pass's arrays.  The shared-memory data pipe, not
-// instruction issue, is what this kernel runs out of, so a directory look-up first reads one 32-bit
-// word per 4-slot bucket -- an 8-bit tag per slot, taken from hash bits the bucket choice does not
-// use -- and only a lane whose tag matches reads the 8-byte key to confirm.  A wrong tag match
-// (1 in 64 look-ups) fails the confirmation and the record takes the spill path: slower, still exact.
-struct SmemDir {
-    uint32_t keys;    // ull[slots] ~key, 0 = empty
-    uint32_t tag;     // u32[buckets] four 8-bit tags
-    uint32_t a0;      // u32[slots] this launch's weighted time of the slot: bits 0..31 ...
-    uint32_t a1;      // u32[slots] ... and bits 32.. (carries of a0 are added here by the adder)
-    uint32_t cnt;     // u32[slots] this launch's record count of the slot
-    uint32_t cursor;  // u32[P] entries appended to this CTA's buffer of each partition
-    uint32_t appw;    // u32[n_apps] card-hour weights, when they fit in shared memory ...
-    const uint32_t* appw_g;  // ... else they are read from global memory
-    bool appw_shared;
-    uint32_t mult;    // bucket-hash multiplier of this directory image
-};
 
 // Shared-memory accumulation uses native 32-bit atomics only (64-bit shared atomics are
 // compare-and-swap loops).  A slot's weighted time is kept in two limbs: the returning add on
@@ -149,288 +128,6 @@ __device__ __forceinline__ ull limbs_drain(uint32_t a0, uint32_t a1, ull* hi_out
     const ull v = lo + (hi << 32);
     *hi_out = v < lo ? 1ull : 0ull;
     return v;
-}
-
-// Add (count, v) to a directory slot, v < 2^53, count <= 32.
-__device__ __forceinline__ void dir_add(const SmemDir& d, uint32_t slot, ull v, uint32_t count, const TableRef& t,
-                                        uint32_t h) {
-    if (limbs_add(d.a0 + slot * 4, d.a1 + slot * 4, d.cnt + slot * 4, v, count)) {
-        ull hi, lo = limbs_drain(d.a0 + slot * 4, d.a1 + slot * 4, &hi);
-        table_accumulate(t, ~lds_u64(d.keys + slot * 8), h, lo, hi, 0);
-    }
-}
-
-// Process R records held in registers by every lane of the warp (absent ones masked).
-// Written in stages over the R records so that their shared-memory round trips overlap.
-template <bool HOT, bool DEDUPE, bool FULL, int R>
-__device__ __forceinline__ void process(const uint32_t (&w)[R][4], const bool (&present)[R], const IngestParams& p,
-                                        const SmemDir& d, uint32_t& rejected) {
-    uint32_t khi[R], h[R];
-    ull prod[R];
-    bool todo[R];  // valid and not yet accumulated
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        uint32_t app = w[r][0];
-        khi[r] = w[r][1] & 0x00FFFFFFu;                 // phase << 16 | op_id: the key's high word
-        bool ok = (FULL || present[r]) && app < p.n_apps && khi[r] < (p.n_phases << 16);
-        rejected += ((FULL || present[r]) && !ok) ? 1u : 0u;
-        // card-hour weight: from shared memory when the table fits there, else from global
-        uint32_t wgt = d.appw_shared ? lds_u32(d.appw + (ok ? app : 0u) * 4) : __ldg(d.appw_g + (ok ? app : 0u));
-        prod[r] = (ull)wgt * (ull)w[r][3];
-        h[r] = hash32(khi[r] & 0xFFFFu, w[r][2]);
-        todo[r] = ok;
-        // The limb arithmetic below and the 16-byte spill entries assume products below 2^48
-        // (e.g. weights < 2^20, durations < 2^28).  Anything larger is still exact: it goes
-        // straight to the table with full 64-bit adds.
-        if (ok && (prod[r] >> 48) != 0) {
-            table_accumulate(p.t, ((ull)khi[r] << 32) | w[r][2], h[r], prod[r], 0, 1);
-            todo[r] = false;
-        }
-    }
-    if (HOT) {
-        uint32_t slot[R];
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            const uint32_t x = dir_mix(h[r], khi[r] >> 16, d.mult);
-            const uint32_t b = __umulhi(x, p.hot_buckets);
-            const uint32_t eq = __vcmpeq4(lds_u32(d.tag + b * 4), (x & 0xFFu) * 0x01010101u);  // 0xFF per matching byte
-            const uint32_t at = b * DIR_WAYS + (((uint32_t)__ffs(eq) - 1u) >> 3);
-            const ull skey = ~(((ull)khi[r] << 32) | w[r][2]);
-            const bool hit = todo[r] && eq != 0 && lds_u64(d.keys + at * 8) == skey;
-            slot[r] = hit ? at : NO_SLOT;
-        }
-        if (DEDUPE) {
-            // one key dominates the trace: combine the lanes that share the first hitting lane's slot
-            const unsigned lane = threadIdx.x & 31u;
-#pragma unroll
-            for (int r = 0; r < R; ++r) {
-                unsigned hits = __ballot_sync(0xFFFFFFFFu, slot[r] != NO_SLOT);
-                if (hits == 0) continue;
-                int lead = __ffs(hits) - 1;
-                uint32_t ls = __shfl_sync(0xFFFFFFFFu, slot[r], lead);
-                unsigned same = __ballot_sync(0xFFFFFFFFu, slot[r] == ls);
-                if (__popc(same) >= 2 && slot[r] == ls) {
-                    uint32_t s_lo = __reduce_add_sync(same, (uint32_t)prod[r] & 0xFFFFFFu);
-                    uint32_t s_hi = __reduce_add_sync(same, (uint32_t)(prod[r] >> 24));
-                    if (lane == (unsigned)lead)
-                        dir_add(d, ls, (ull)s_lo + ((ull)s_hi << 24), (uint32_t)__popc(same), p.t, h[r]);
-                    slot[r] = NO_SLOT;
-                    todo[r] = false;
-                }
-            }
-        }
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-            if (slot[r] != NO_SLOT) {
-                dir_add(d, slot[r], prod[r], 1u, p.t, h[r]);
-                todo[r] = false;
-            }
-        }
-    }
-    // spill: append {key, product} to this CTA's buffer of the key's partition
-    uint32_t pos[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) pos[r] = todo[r] ? atoms_add(d.cursor + part_of(h[r], p.t.lp) * 4, 1u) : 0u;
-#pragma unroll
-    for (int r = 0; r < R; ++r) {
-        if (todo[r]) {
-            ull key = ((ull)khi[r] << 32) | w[r][2];
-            if (pos[r] < p.cap) {
-                uint32_t idx = ((blockIdx.x << p.t.lp) + part_of(h[r], p.t.lp)) * p.cap + pos[r];
-                unsigned char* at = p.spill + (ull)idx * 16ull;
-                *reinterpret_cast<ulonglong2*>(at) = make_ulonglong2(key, prod[r]);
-                // a 16-byte store into a line that is not in L2 stalls on a write-miss fill; two
-                // entries before this buffer moves on to its next 128-byte line, pull that line in
-                if ((pos[r] & 7u) == 6) asm volatile("prefetch.global.L2 [%0];" ::"l"(at + 32));
-            } else {
-                table_accumulate(p.t, key, h[r], prod[r], 0, 1);  // buffer full: exact slow path
-            }
-        }
-    }
-}
-
-template <bool HOT, bool DEDUPE>
-__device__ __forceinline__ void scatter_body(const IngestParams& p, const SmemDir& d, uint32_t& rejected) {
-    // Each thread keeps two 32-byte loads (four records) in flight: the pair after next is
-    // requested before the current pair is processed.  CTA b handles pairs
-    // (b + k * gridDim) * 1024 + tid; rounds in which every CTA's tile is complete need no
-    // bounds checks, the last (ragged) ones are predicated.
-    const unsigned char* body = reinterpret_cast<const unsigned char*>(p.body);
-    const ull stride = (ull)gridDim.x * INGEST_THREADS;
-    const ull full_rounds = p.n_pairs / stride;                    // rounds complete for every CTA
-    const ull rounds = (p.n_pairs + stride - 1) / stride;
-    const ull first = (ull)blockIdx.x * INGEST_THREADS + threadIdx.x;
-    uint32_t rawA[8], rawB[8];
-    auto fetch = [&](ull round, uint32_t (&raw)[8]) {
-        ull i = first + round * stride;
-        if (round < full_rounds || (round < rounds && i < p.n_pairs)) {
-            ld_stream_256(body + i * 32, raw);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) raw[j] = 0;
-        }
-    };
-    auto consume = [&](ull round, const uint32_t (&raw)[8], auto full_tag) {
-        constexpr bool FULL = decltype(full_tag)::value;
-        uint32_t w[2][4];
-        bool present[2];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            w[0][j] = raw[j];
-            w[1][j] = raw[4 + j];
-        }
-        present[0] = present[1] = FULL || (first + round * stride) < p.n_pairs;
-        process<HOT, DEDUPE, FULL, 2>(w, present, p, d, rejected);
-    };
-    using True = std::integral_constant<bool, true>;
-    using False = std::integral_constant<bool, false>;
-    fetch(0, rawA);
-    fetch(1, rawB);
-    ull round = 0;
-    for (; round + 2 <= full_rounds; round += 2) {
-        uint32_t cur[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) cur[j] = rawA[j];
-        fetch(round + 2, rawA);
-        consume(round, cur, True{});
-#pragma unroll
-        for (int j = 0; j < 8; ++j) cur[j] = rawB[j];
-        fetch(round + 3, rawB);
-        consume(round + 1, cur, True{});
-    }
-    for (; round < rounds; round += 2) {  // ragged tail, predicated
-        uint32_t cur[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) cur[j] = rawA[j];
-        fetch(round + 2, rawA);
-        consume(round, cur, False{});
-#pragma unroll
-        for (int j = 0; j < 8; ++j) cur[j] = rawB[j];
-        fetch(round + 3, rawB);
-        consume(round + 1, cur, False{});
-    }
-    // records that do not form an aligned pair (at most one before and one after the body)
-    if (blockIdx.x == 0 && threadIdx.x < 32) {
-        uint32_t w1[1][4] = {{0, 0, 0, 0}};
-        bool pr[1] = {false};
-        const void* src = threadIdx.x == 0 ? p.single[0] : p.single[1];
-        if (threadIdx.x < p.n_single) {
-            uint4 v = *reinterpret_cast<const uint4*>(src);
-            w1[0][0] = v.x; w1[0][1] = v.y; w1[0][2] = v.z; w1[0][3] = v.w;
-            pr[0] = true;
-        }
-        process<HOT, DEDUPE, false, 1>(w1, pr, p, d, rejected);
-    }
-}
-
-template <bool HOT>
-__global__ void __launch_bounds__(INGEST_THREADS, 1) scatter_kernel(IngestParams p) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    // carve shared memory: directory (keys, limbs, counts), spill cursors, card-hour weights
-    unsigned char* sp = smem_raw;
-    ull* g_keys = reinterpret_cast<ull*>(sp);
-    sp += HOT ? (size_t)p.hot_slots * 8 : 0;
-    uint32_t* g_a0 = reinterpret_cast<uint32_t*>(sp);
-    sp += HOT ? (size_t)p.hot_slots * 4 : 0;
-    uint32_t* g_a1 = reinterpret_cast<uint32_t*>(sp);
-    sp += HOT ? (size_t)p.hot_slots * 4 : 0;
-    uint32_t* g_cnt = reinterpret_cast<uint32_t*>(sp);
-    sp += HOT ? (size_t)p.hot_slots * 4 : 0;
-    unsigned char* g_tag = sp;
-    sp += HOT ? (size_t)p.hot_slots : 0;
-    const uint32_t n_parts = 1u << p.t.lp;
-    uint32_t* g_cursor = reinterpret_cast<uint32_t*>(sp);
-    sp += (size_t)n_parts * 4;
-    uint32_t* g_appw = reinterpret_cast<uint32_t*>(sp);
-
-    SmemDir d;
-    d.a0 = smem_addr(g_a0);
-    d.a1 = smem_addr(g_a1);
-    d.cnt = smem_addr(g_cnt);
-    d.keys = smem_addr(g_keys);
-    d.tag = smem_addr(g_tag);
-    d.cursor = smem_addr(g_cursor);
-    d.appw = smem_addr(g_appw);
-    d.appw_g = p.app_w;
-    d.appw_shared = p.appw_in_smem != 0;
-    d.mult = HOT ? (uint32_t)p.t.ctl->dir_mult : 1u;
-
-    // the buffers persist across launches until the partition pass drains them: resume the cursors
-    for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) g_cursor[i] = p.spill_cnt[((ull)blockIdx.x << p.t.lp) + i];
-    if (p.appw_in_smem)
-        for (uint32_t i = threadIdx.x; i < p.n_apps; i += blockDim.x) g_appw[i] = p.app_w[i];
-    if (HOT) {
-        for (uint32_t i = threadIdx.x; i < p.hot_slots; i += blockDim.x) {
-            const ull image = p.hot_keys[i];  // ~key, 0 = empty
-            g_keys[i] = image;
-            g_tag[i] = (unsigned char)(dir_mix(hash32(~image), (uint32_t)(~image >> 48) & 0xFFu, d.mult) & 0xFFu);
-            g_a0[i] = 0;
-            g_a1[i] = 0;
-            g_cnt[i] = 0;
-        }
-    }
-    __syncthreads();
-
-    uint32_t rejected = 0;
-    if (HOT && p.t.ctl->hot_skew != 0)
-        scatter_body<HOT, true>(p, d, rejected);
-    else
-        scatter_body<HOT, false>(p, d, rejected);
-
-    // rejected counter: one atomic per warp
-    uint32_t rsum = __reduce_add_sync(0xFFFFFFFFu, rejected);
-    if ((threadIdx.x & 31u) == 0 && rsum != 0) atomicAdd(&p.t.ctl->n_rejected, (ull)rsum);
-
-    __syncthreads();
-    uint32_t spilled = 0, overflow = 0, fullest = 0;
-    bool crowded = false;
-    for (uint32_t i = threadIdx.x; i < n_parts; i += blockDim.x) {
-        const ull at = ((ull)blockIdx.x << p.t.lp) + i;
-        uint32_t before = p.spill_cnt[at], c = g_cursor[i];
-        p.spill_cnt[at] = min(c, p.cap);
-        spilled += min(c, p.cap) - before;
-        overflow += c > p.cap ? c - p.cap : 0u;
-        crowded |= c > p.drain_above;
-        fullest = max(fullest, c);
-    }
-    fullest = __reduce_max_sync(0xFFFFFFFFu, fullest);
-    spilled = __reduce_add_sync(0xFFFFFFFFu, spilled);
-    overflow = __reduce_add_sync(0xFFFFFFFFu, overflow);
-    crowded = __any_sync(0xFFFFFFFFu, crowded);
-    if ((threadIdx.x & 31u) == 0) {
-        if (spilled) atomicAdd(&p.t.ctl->n_spilled, (ull)spilled);
-        if (overflow) atomicAdd(&p.t.ctl->n_overflow, (ull)overflow);
-        // a buffer is filling up: have the partition pass that follows this launch drain them
-        if (crowded) atomicMax(&p.t.ctl->drain_seq, p.seq);
-        atomicMax(&p.t.ctl->max_fill, (ull)fullest);
-    }
-    if (HOT) {
-        // This launch's directory sums go to the CTA's own row of the directory image: plain coalesced
-        // read-modify-writes, no atomics (148 CTAs adding the same ~9 K keys into the table at the end
-        // of every launch cost 59 us per launch).  hot_fold_kernel adds the rows into the table before
-        // results are read.
-        ulonglong2* img = p.hot_img + (size_t)blockIdx.x * p.hot_slots;
-        for (uint32_t i0 = threadIdx.x; i0 < p.hot_slots; i0 += 4 * blockDim.x) {  // four slots per thread in flight
-            uint32_t c[4], lo[4], hi[4];
-            ulonglong2 o[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t i = i0 + u * blockDim.x;
-                const bool in = i < p.hot_slots;
-                c[u] = in ? g_cnt[i] : 0u;
-                lo[u] = in ? g_a0[i] : 0u;
-                hi[u] = in ? g_a1[i] : 0u;
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) o[u] = (c[u] | lo[u] | hi[u]) ? img[i0 + u * blockDim.x] : make_ulonglong2(0, 0);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if ((c[u] | lo[u] | hi[u]) == 0) continue;
-                const ull nlo = o[u].x + ((ull)lo[u] | ((ull)hi[u] << 32));
-                img[i0 + u * blockDim.x] = make_ulonglong2(nlo, o[u].y + (ull)c[u] + ((nlo < o[u].x ? 1ull : 0ull) << HI_SHIFT));
-            }
-        }
-    }
 }
 
 // Adds every CTA's directory image row into the table and clears the rows.  A CTA handles 32
@@ -995,22 +692,11 @@ __global__ void __launch_bounds__(256) merge_kernel(const atrex_entry_t* in, ull
 // host launchers
 
 cudaError_t ingest_prepare() {
-    cudaError_t e = cudaFuncSetAttribute(scatter_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(scatter_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
+    cudaError_t e = scatter_prepare();
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(partition_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 2048);
     if (e != cudaSuccess) return e;
     return cudaFuncSetAttribute(hot_select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SELECT_SMEM);
-}
-
-cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream) {
-    size_t smem = (hot ? (size_t)p.hot_slots * 21 : 0) + ((size_t)4 << p.t.lp) + (p.appw_in_smem ? (size_t)p.n_apps * 4 : 0);
-    if (hot)
-        scatter_kernel<true><<<grid, INGEST_THREADS, smem, stream>>>(p);
-    else
-        scatter_kernel<false><<<grid, INGEST_THREADS, smem, stream>>>(p);
-    return cudaGetLastError();
 }
 
 cudaError_t launch_partition(const PartitionParams& q, int n_sms, cudaStream_t stream) {

@@ -4,12 +4,44 @@
 
 namespace atrex {
 
+// Build-time variants of the scatter pass (the defaults are the fastest measured; the others are kept
+// so that the comparison can be repeated):
+//   ATREX_SCATTER_RING   stages of a shared-memory ring that a producer warp fills with bulk
+//                        asynchronous copies of record tiles (0: records are loaded straight into
+//                        registers, two 32-byte loads alternating per thread)
+//   ATREX_SCATTER_PAIR   1: spill entries leave in pairs as whole 32-byte sectors (pairing mailbox per
+//                        partition in shared memory); 0: every entry is stored on its own
+#ifndef ATREX_SCATTER_RING
+#define ATREX_SCATTER_RING 0
+#endif
+#ifndef ATREX_SCATTER_PAIR
+#define ATREX_SCATTER_PAIR 0
+#endif
+
+// Shared memory of the scatter pass (dynamic, one CTA per SM) and what fits in it.  Per partition a
+// cursor word (and a 16-byte pairing mailbox), 16 KB of card-hour weights, the record ring if there
+// is one, then the hot directory: a tag byte, an 8-byte key and 12 bytes of accumulators per slot, in
+// whole 4-way buckets.
+constexpr uint32_t APPW_SMEM_MAX = 4096;
+constexpr uint32_t SCATTER_SMEM_BYTES = 232448 - 1024;
+constexpr uint32_t SCATTER_RING_STAGES = ATREX_SCATTER_RING;
+constexpr uint32_t SCATTER_CONSUMER_WARPS = SCATTER_RING_STAGES ? 31 : 32;
+constexpr uint32_t SCATTER_RING_TILE = SCATTER_CONSUMER_WARPS * 32 * 16;   // one record per consumer thread
+constexpr bool SCATTER_PAIR = ATREX_SCATTER_PAIR != 0;
+constexpr uint32_t scatter_fixed_bytes(uint32_t lp) {
+    return ((SCATTER_PAIR ? 20u : 4u) << lp) + 4u * APPW_SMEM_MAX + SCATTER_RING_STAGES * SCATTER_RING_TILE + 128u;
+}
+constexpr uint32_t scatter_hot_slots(uint32_t lp) { return ((SCATTER_SMEM_BYTES - scatter_fixed_bytes(lp)) / 21u) & ~31u; }
+
 struct IngestParams {
-    const void* body;          // first record of the 32-byte aligned run of record pairs
+    const void* recs;          // all records of this launch (16-byte aligned) ...
+    ull n_recs;
+    const void* body;          // ... and the same split up: first record of the 32-byte aligned run of record pairs
     ull n_pairs;               // pairs in the body
     const void* single[2];     // records outside the body (unaligned head, odd tail)
     uint32_t n_single;
     uint32_t n_apps, n_phases;
+    uint32_t phase_lim;        // n_phases << 16: bound of (phase << 16 | op_id)
     uint32_t appw_in_smem;
     const uint32_t* app_w;     // device copy of the card-hour weights
     const ull* hot_keys;       // directory image, hot_slots entries of ~key (0 = empty)
@@ -99,6 +131,7 @@ struct TopkAllParams {
 };
 
 cudaError_t ingest_prepare();
+cudaError_t scatter_prepare();
 cudaError_t launch_scatter(const IngestParams& p, bool hot, int grid, cudaStream_t stream);
 cudaError_t launch_partition(const PartitionParams& p, int n_sms, cudaStream_t stream);
 cudaError_t launch_hot_build(const HotBuildParams& p, int n_sms, cudaStream_t stream);

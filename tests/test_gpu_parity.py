@@ -384,11 +384,11 @@ def test_topk_requests_in_any_order_and_after_more_records(lib):
 
 
 def test_crowded_small_partitions_overflow_the_deferred_queue(lib):
-    """Tiny partitions (128 slots) at a load factor of 0.76, no hot directory, about 200 K entries per
-    partition in the first drain: more entries fail the first look (45-50 K per partition) than the
-    partition pass's per-CTA queue holds (32 K), so the in-line fallback runs as well.  Still exact."""
+    """Tiny partitions (a few hundred slots, the smallest geometry), no hot directory, about 500 K entries
+    per partition in the first drain: the entries that fail the first look outnumber what the partition
+    pass's per-CTA queue holds (32 K), so the in-line fallback runs as well.  Still exact."""
     rng = np.random.default_rng(77)
-    n, n_keys = 1 << 26, 25_000
+    n, n_keys = 1 << 27, 25_000
     k = rng.integers(0, n_keys, n, dtype=np.uint32)
     recs = np.zeros(n, dtype=RECORD_DTYPE)
     recs["app_id"] = rng.integers(0, 16, n, dtype=np.uint32)
@@ -399,7 +399,7 @@ def test_crowded_small_partitions_overflow_the_deferred_queue(lib):
     weights = rng.integers(1, 1 << 20, 16, dtype=np.uint32)
     agg = gpu_aggregate(lib, recs, weights, 2, max_keys=n_keys, chunks=1, flags=lib.ATREX_FLAG_NO_HOT_DIRECTORY)
     st = agg.stats()
-    assert st["table_slots"] == 256 * 128 and st["n_spilled"] == n and st["n_overflow"] == 0
+    assert st["table_slots"] <= 256 * 256 and st["n_spilled"] == n and st["n_overflow"] == 0
     o = oracle_of(recs, weights, 2, threads=16)
     assert_same_as_oracle(agg, o, 2)
 
