@@ -200,9 +200,18 @@ def run_ours(args):
     out = torch.empty(spec.max_keys * 48, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream(dev)
     ingest_events = []
+    owner = None
+    if world > 1:
+        # several GPUs: this rank's handle holds its slice of the trace; a second handle holds the keys
+        # this rank owns after the exchange step (every entry travels to its key's owner)
+        from paper_2607_14541_b200 import distributed as D
+        owner = p.Aggregator(spec.app_weights, spec.n_phases, spec.max_keys, max_work_rows=len(work), device=local)
+        owner.set_work_table(work)
 
     def step(timed: bool):
         agg.reset()
+        if owner is not None:
+            owner.reset()
         for c in range(n_chunks):
             view = records[c * chunk * RECORD_BYTES: (c + 1) * chunk * RECORD_BYTES]
             if timed:
@@ -213,6 +222,10 @@ def run_ours(args):
                 ingest_events.append((e0, e1))
             else:
                 agg.ingest(view, n=chunk)
+        if owner is not None:
+            _, n_out = D.aggregate_sharded(agg, owner, spec.peak_bw, spec.peak_flops)
+            tops = [D.global_topk(owner, phase, spec.topk) for phase in range(spec.n_phases)]
+            return n_out, tops
         _, n_out = agg.finalize(spec.peak_bw, spec.peak_flops, out=out)
         tops = [agg.topk(phase, spec.topk) for phase in range(spec.n_phases)]
         return n_out, tops
@@ -236,7 +249,7 @@ def run_ours(args):
     ev1.record(stream)
     barrier()
     elapsed_ms = ev0.elapsed_time(ev1)
-    launches = agg.launch_count() - launches0
+    launches = agg.launch_count() - launches0 + (owner.launch_count() if owner is not None else 0)
     ingest_ms = [a.elapsed_time(b) for a, b in ingest_events]
     st = agg.stats()
     assert st["n_valid"] + st["n_rejected"] == n and st["n_dropped"] == 0, st
@@ -276,8 +289,13 @@ def run_ours(args):
                                        f"{spec.n_apps} apps, {spec.n_ops} ops x {spec.n_shapes} shapes Zipf({spec.zipf_s})",
                            "records_per_gpu": n, "chunks": n_chunks, "live_keys": int(n_keys),
                            "l2": "inputs (16 GiB per step) exceed L2; no flush needed",
-                           "step": "reset + ingest x chunks + finalize + topk per phase",
-                           "parallelism": f"independent trace partitions x{world}"},
+                           "step": ("reset + ingest x chunks + finalize + topk per phase" if world == 1 else
+                                    "reset + ingest x chunks + exchange step (entries grouped by key owner, NCCL "
+                                    "all-to-all, merge at the owner, totals combined, finalize of the owned keys) "
+                                    "+ global topk per phase (owners' candidates gathered and ranked)"),
+                           "live_keys_is": "keys of this GPU's trace" if world == 1 else "keys rank 0 owns",
+                           "workspace_bytes_per_handle": agg.workspace_bytes,
+                           "parallelism": f"trace sharded by records x{world}"},
                 "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline,
                 "algorithmic_GBps_whole_step": world * n * RECORD_BYTES * args.steps / (elapsed_ms * 1e-3) / 1e9}
         if e2e:
@@ -286,10 +304,65 @@ def run_ours(args):
                            "steps": e2e["steps"], "sample": e2e["sample"]}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(args, spec, records, torch)
+        if world == 1 and not args.no_per_config:
+            del agg
+            line["per_config"] = per_config(torch, p, records, n, peak)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+# DRAM bytes moved per record by the ingest pass (scatter launches + the drains they trigger), from
+# one-kernel ncu captures of 2^25..2^27-record cases summarised under profiles/ (traffic grows in
+# proportion to the records of a launch); None where no capture was taken.
+NCU_DRAM_BYTES_PER_RECORD = {3: NCU_DRAM_BYTES_PER_INGEST_CALL / float(1 << 27)}
+
+
+def per_config(torch, p, records3, n3, peak):
+    """The ingest pass of each of the five benchmark configurations, timed the same way: records resident
+    in HBM, reset (untimed), CUDA events around all ingest calls of the configuration, best of three after
+    a warm-up.  Config 3's records are the bench step's own."""
+    from tracegen.configs import make_spec
+    from tracegen.gpu import GpuSampler
+    rows = []
+    for index in range(5):
+        spec = make_spec(index)
+        if index == WORKLOAD_INDEX:
+            recs, n = records3, n3
+        else:
+            n = spec.n
+            recs = torch.empty(n * RECORD_BYTES, dtype=torch.uint8, device=records3.device)
+            GpuSampler(spec, records3.device).fill(recs, 0, n)
+        chunk = n // spec.n_chunks
+        agg = p.Aggregator(spec.app_weights, spec.n_phases, spec.max_keys, device=records3.device.index)
+        best = None
+        for rep in range(4):
+            agg.reset()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for c in range(spec.n_chunks):
+                agg.ingest(recs[c * chunk * RECORD_BYTES:(c + 1) * chunk * RECORD_BYTES], n=chunk)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            if rep > 0 and (best is None or ms < best):
+                best = ms
+        st = agg.stats()
+        gbs = chunk * spec.n_chunks * RECORD_BYTES / (best * 1e-3) / 1e9
+        rows.append({"config": index, "name": spec.name, "records": chunk * spec.n_chunks, "ingest_ms": best,
+                     "records_per_s": chunk * spec.n_chunks / (best * 1e-3), "algorithmic_GBps": gbs,
+                     "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / 8000.0,
+                     "spill_fraction": st["n_spilled"] / max(st["n_valid"], 1), "live_keys": st["n_keys"],
+                     "drains_inside": max(int(st["n_drains"]) - 1, 0),
+                     "dram_bytes_per_record": NCU_DRAM_BYTES_PER_RECORD.get(index),
+                     "note": "16 MiB of records: L2-resident and launch-bound, not an HBM measurement" if index == 0 else None})
+        del agg
+        if index != WORKLOAD_INDEX:
+            del recs
+        torch.cuda.empty_cache()
+    return rows
 
 
 def _gpu_id(torch, local: int) -> str:
@@ -357,6 +430,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-config", action="store_true")
     ap.add_argument("--cpu-records", type=int, default=1 << 25)
     ap.add_argument("--ref-records", type=int, default=1 << 24)
     ap.add_argument("--ncu-traffic-bytes", type=float, default=None,

@@ -51,6 +51,7 @@ extern "C" {
 #define ATREX_MAX_PHASES 8
 #define ATREX_MAX_DTYPES 8
 #define ATREX_MAX_TOPK 65536u
+#define ATREX_MAX_WORLD 1024u     /* GPUs an entry array can be split over (atrex_entries_bucket_by_owner) */
 
 typedef enum {
     ATREX_OK = 0,
@@ -174,14 +175,47 @@ int atrex_agg_finalize(atrex_agg_t*, const atrex_hw_peaks_t* peaks, atrex_entry_
 /* atrex_agg_finalize for one shard of a trace that was split over several handles (GPUs).
  * Eq. 3 normalises by the phase total over ALL records; when every handle holds only the keys it
  * owns (after the partial aggregates were exchanged and folded with atrex_agg_merge), the caller
- * adds the handles' per-phase totals (atrex_agg_stats, as 128-bit integers) and passes the sums
- * here: total_lo / total_hi are HOST arrays of ATREX_MAX_PHASES low / high 64-bit words.  The
+ * adds the handles' per-phase totals (atrex_agg_totals, combined by atrex_totals_combine) and passes
+ * the sums here: total_lo / total_hi are HOST arrays of ATREX_MAX_PHASES low / high 64-bit words.  The
  * entries written, and those atrex_agg_topk returns afterwards, then carry
  * phase_weight = fl(fl(wt) / fl(global total)), bit-identical to a single handle that saw every
  * record.  Everything else is as in atrex_agg_finalize. */
 int atrex_agg_finalize_with_totals(atrex_agg_t*, const atrex_hw_peaks_t* peaks, const uint64_t* total_lo,
                                    const uint64_t* total_hi, atrex_entry_t* d_out, uint64_t out_cap,
                                    uint64_t* n_out, void* stream);
+
+/* The per-phase totals T[phase] the last successful finalize of this handle normalised by (Eq. 3's
+ * denominators; after atrex_agg_finalize the handle's own sums, after atrex_agg_finalize_with_totals
+ * the totals that were passed in).  h_lo / h_hi: HOST arrays of ATREX_MAX_PHASES low / high words.
+ * No device work.  ATREX_ERR_STATE without a finalize since the last ingest, merge or reset. */
+int atrex_agg_totals(const atrex_agg_t*, uint64_t* h_lo, uint64_t* h_hi);
+
+/* ---- exchange step of the multi-GPU path ------------------------------------------------------
+ * Eq. 2 is a sum over independent invocations and all accumulators are exact integers, so the
+ * trace shards by records: each GPU aggregates its slice with the calls above.  To make the
+ * partial results global, every entry is sent to the GPU that owns its key and folded in there
+ * with atrex_agg_merge; Eq. 3's denominators are then the sums of the shards' totals.  The three
+ * calls below are the arithmetic of that step (the bytes are moved by the caller's collective).
+ *
+ * atrex_key_owner: the rank in [0, world) that owns `key`; a fixed scramble of the packed key. */
+uint32_t atrex_key_owner(uint64_t key, uint32_t world);
+/* The same for `n` keys at once: h_keys and h_out are HOST arrays. */
+void atrex_keys_owner(const uint64_t* h_keys, uint64_t n, uint32_t world, uint32_t* h_out);
+
+/* Groups the `n` entries at d_entries (DEVICE, 16-byte aligned) by owner rank: d_out (DEVICE, room
+ * for n entries, must not overlap d_entries) receives rank 0's entries first, then rank 1's, ...;
+ * h_counts (HOST, `world` values) the size of each group.  The order inside a group is unspecified.
+ * d_scratch: DEVICE, 2 * world 64-bit words, contents irrelevant.  world <= ATREX_MAX_WORLD,
+ * n <= 2^32 (ATREX_ERR_TOO_LARGE).  Synchronises `stream`. */
+int atrex_entries_bucket_by_owner(const atrex_entry_t* d_entries, uint64_t n, uint32_t world, atrex_entry_t* d_out,
+                                  uint64_t* d_scratch, uint64_t* h_counts, void* stream);
+
+/* Exact sum of the shards' per-phase totals: h_lo / h_hi are HOST arrays [n_ranks][ATREX_MAX_PHASES]
+ * of low / high 64-bit words (one row per shard, as atrex_agg_totals returns them), h_out_lo /
+ * h_out_hi receive the ATREX_MAX_PHASES 128-bit sums.  Host arithmetic only (a reduction of the
+ * halves by a collective would lose the carries). */
+int atrex_totals_combine(const uint64_t* h_lo, const uint64_t* h_hi, uint32_t n_ranks, uint64_t* h_out_lo,
+                         uint64_t* h_out_hi);
 
 /* Table 2: the min(k, keys of `phase`) entries with the largest weighted time, compared as
  * exact 128-bit integers, ties broken by ascending key; written in that order to `h_out`

@@ -30,6 +30,7 @@ ATREX_ERR_NOMEM = -7
 ATREX_ERR_TOO_LARGE = -8
 ATREX_RELEASE_MAX_ENTRIES = 1 << 28
 ATREX_STATIC_TOPK_MAX_ENTRIES = 65536
+ATREX_MAX_WORLD = 1024
 
 RECORD_DTYPE = np.dtype([("app_id", "<u4"), ("op_id", "<u2"), ("phase", "u1"), ("pad", "u1"),
                          ("shape_id", "<u4"), ("duration_ns", "<u4")])
@@ -44,7 +45,8 @@ EXPORTED_SYMBOLS = [
     "atrex_agg_launch_count", "atrex_topk_entries_static", "atrex_agg_hot_directory",
     "atrex_agg_finalize_with_totals", "atrex_score_aggregate", "atrex_eq3_create", "atrex_eq3_ingest",
     "atrex_eq3_finalize", "atrex_eq3_reset", "atrex_eq3_destroy", "atrex_release_scratch_bytes",
-    "atrex_entries_sort_by_key", "atrex_entries_rank",
+    "atrex_entries_sort_by_key", "atrex_entries_rank", "atrex_agg_totals", "atrex_key_owner", "atrex_keys_owner",
+    "atrex_entries_bucket_by_owner", "atrex_totals_combine",
 ]
 
 
@@ -110,6 +112,13 @@ def _load():
     L.atrex_release_scratch_bytes.argtypes = [u64]
     L.atrex_entries_sort_by_key.argtypes = [vp, u64, vp, vp, u64, vp]
     L.atrex_entries_rank.argtypes = [vp, u64, u32, u32, vp, vp, u64, C.POINTER(atrex_rank_result_t), vp, u64, vp]
+    L.atrex_agg_totals.argtypes = [vp, vp, vp]
+    L.atrex_key_owner.restype = u32
+    L.atrex_key_owner.argtypes = [u64, u32]
+    L.atrex_keys_owner.restype = None
+    L.atrex_keys_owner.argtypes = [vp, u64, u32, vp]
+    L.atrex_entries_bucket_by_owner.argtypes = [vp, u64, u32, vp, vp, vp, vp]
+    L.atrex_totals_combine.argtypes = [vp, vp, u32, vp, vp]
     return L
 
 
@@ -142,6 +151,11 @@ atrex_eq3_destroy = lib.atrex_eq3_destroy
 atrex_release_scratch_bytes = lib.atrex_release_scratch_bytes
 atrex_entries_sort_by_key = lib.atrex_entries_sort_by_key
 atrex_entries_rank = lib.atrex_entries_rank
+atrex_agg_totals = lib.atrex_agg_totals
+atrex_key_owner = lib.atrex_key_owner
+atrex_keys_owner = lib.atrex_keys_owner
+atrex_entries_bucket_by_owner = lib.atrex_entries_bucket_by_owner
+atrex_totals_combine = lib.atrex_totals_combine
 
 
 class AtrexError(RuntimeError):
@@ -292,6 +306,32 @@ def rank_entries(entries, n: int, phase: int, coverage_ppm: int = 0, out_cap=Non
         "covered": int(res.covered_lo) | (int(res.covered_hi) << 64)}
 
 
+def bucket_entries_by_owner(entries, n: int, world: int, stream=None):
+    """Group the ``n`` entries of the CUDA byte tensor ``entries`` by owner rank (``atrex_entries_bucket_by_owner``).
+    Returns (grouped CUDA byte tensor, list of per-rank entry counts)."""
+    import torch
+    out = torch.empty(max(int(n), 1) * 48, dtype=torch.uint8, device=entries.device)
+    scratch = torch.empty(2 * int(world), dtype=torch.int64, device=entries.device)
+    counts = np.zeros(int(world), dtype=np.uint64)
+    rc = atrex_entries_bucket_by_owner(entries.data_ptr() if n else None, int(n), int(world), out.data_ptr(),
+                                       scratch.data_ptr(), counts.ctypes.data, _stream_ptr(stream))
+    if rc != ATREX_OK:
+        raise AtrexError(rc, "atrex_entries_bucket_by_owner")
+    return out[: int(n) * 48], [int(c) for c in counts]
+
+
+def combine_totals(lo_rows: np.ndarray, hi_rows: np.ndarray):
+    """Exact per-phase sums of the shards' totals (``atrex_totals_combine``); rows are [n_ranks, 8] uint64.
+    Returns (lo[8], hi[8]) as uint64 arrays."""
+    lo = np.ascontiguousarray(lo_rows, dtype=np.uint64).reshape(-1, ATREX_MAX_PHASES)
+    hi = np.ascontiguousarray(hi_rows, dtype=np.uint64).reshape(-1, ATREX_MAX_PHASES)
+    out_lo, out_hi = np.zeros(ATREX_MAX_PHASES, dtype=np.uint64), np.zeros(ATREX_MAX_PHASES, dtype=np.uint64)
+    rc = atrex_totals_combine(lo.ctypes.data, hi.ctypes.data, lo.shape[0], out_lo.ctypes.data, out_hi.ctypes.data)
+    if rc != ATREX_OK:
+        raise AtrexError(rc, "atrex_totals_combine")
+    return out_lo, out_hi
+
+
 class Aggregator:
     """One aggregation handle on one GPU.  Thin object wrapper over the C calls."""
 
@@ -386,9 +426,12 @@ class Aggregator:
         pk = make_peaks(peak_bw, peak_flops)
         n_out = C.c_uint64(0)
         if global_totals is not None:
-            t = list(global_totals) + [0] * (ATREX_MAX_PHASES - len(global_totals))
-            lo = np.array([x & 0xFFFFFFFFFFFFFFFF for x in t[:ATREX_MAX_PHASES]], dtype=np.uint64)
-            hi = np.array([x >> 64 for x in t[:ATREX_MAX_PHASES]], dtype=np.uint64)
+            if isinstance(global_totals, tuple) and len(global_totals) == 2 and isinstance(global_totals[0], np.ndarray):
+                lo, hi = (np.ascontiguousarray(x, dtype=np.uint64) for x in global_totals)   # (lo[8], hi[8]) words
+            else:
+                t = list(global_totals) + [0] * (ATREX_MAX_PHASES - len(global_totals))
+                lo = np.array([x & 0xFFFFFFFFFFFFFFFF for x in t[:ATREX_MAX_PHASES]], dtype=np.uint64)
+                hi = np.array([x >> 64 for x in t[:ATREX_MAX_PHASES]], dtype=np.uint64)
 
             def call(ptr, cap):
                 return atrex_agg_finalize_with_totals(self._h, C.byref(pk), lo.ctypes.data, hi.ctypes.data, ptr, cap,
@@ -427,6 +470,12 @@ class Aggregator:
                 "keys_per_phase": [int(x) for x in st.keys_per_phase], "table_slots": st.table_slots,
                 "hot_slots": st.hot_slots, "n_spilled": st.n_spilled, "n_overflow": st.n_overflow,
                 "max_spill_fill": st.max_spill_fill, "spill_cap": st.spill_cap, "n_drains": st.n_drains}
+
+    def totals_words(self):
+        """(lo[8], hi[8]) uint64 arrays: the per-phase totals of the last finalize (``atrex_agg_totals``)."""
+        lo, hi = np.zeros(ATREX_MAX_PHASES, dtype=np.uint64), np.zeros(ATREX_MAX_PHASES, dtype=np.uint64)
+        self._check(atrex_agg_totals(self._h, lo.ctypes.data, hi.ctypes.data), "atrex_agg_totals")
+        return lo, hi
 
     def hot_directory(self, stream=None) -> np.ndarray:
         """Keys currently in the shared-memory hot directory (diagnostic)."""

@@ -7,7 +7,7 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libatrex_agg.so")
-SOURCES = ["api.cu", "scatter.cu", "ingest.cu", "finalize.cu", "static_topk.cu", "score.cu", "eq3.cu", "release.cu"]
+SOURCES = ["api.cu", "scatter.cu", "ingest.cu", "finalize.cu", "static_topk.cu", "score.cu", "eq3.cu", "release.cu", "exchange.cu"]
 HEADERS = ["atrex_dev.cuh", "kernels.h", os.path.join("..", "..", "include", "atrex_agg.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-fmad=false", "-shared", "-Xcompiler", "-fPIC"]

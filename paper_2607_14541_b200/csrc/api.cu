@@ -716,6 +716,16 @@ int atrex_agg_topk(atrex_agg_t* h, uint32_t phase, uint32_t k, atrex_entry_t* h_
     return ATREX_OK;
 }
 
+int atrex_agg_totals(const atrex_agg_t* h, uint64_t* h_lo, uint64_t* h_hi) {
+    if (!h || !h_lo || !h_hi) return ATREX_ERR_INVALID;
+    if (!h->finalized) return ATREX_ERR_STATE;
+    for (int p = 0; p < ATREX_MAX_PHASES; ++p) {
+        h_lo[p] = h->h_ctl->total_lo[p];
+        h_hi[p] = h->h_ctl->total_hi[p];
+    }
+    return ATREX_OK;
+}
+
 int atrex_agg_stats(atrex_agg_t* h, atrex_stats_t* out, void* stream) {
     if (!h || !out) return ATREX_ERR_INVALID;
     DeviceGuard guard(h->cfg.device);

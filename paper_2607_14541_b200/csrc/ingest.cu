@@ -110,14 +110,16 @@ __device__ __forceinline__ ull atoms_cas64(uint32_t a, ull expected, ull desired
 // 2^31, so the high limb never wraps.
 constexpr uint32_t DRAIN_BIT = 0x40000000u;
 
-// returns true when the caller must drain the slot
+// returns true when the caller must drain the slot.  Most products fit 32 bits and most low-limb adds
+// do not wrap: the high limb is then left alone.
 __device__ __forceinline__ bool limbs_add(uint32_t a0, uint32_t a1, uint32_t cnt, ull v, uint32_t count) {
     const uint32_t v0 = (uint32_t)v;
     const uint32_t o0 = atoms_add(a0, v0);
-    const uint32_t x = (uint32_t)(v >> 32) + ((o0 + v0 < o0) ? 1u : 0u);
-    const uint32_t o1 = atoms_add(a1, x);
     reds_add(cnt, count);
-    return ((o1 ^ (o1 + x)) & DRAIN_BIT) && !(o1 & DRAIN_BIT);
+    const uint32_t x = (uint32_t)(v >> 32) + ((o0 + v0 < o0) ? 1u : 0u);
+    if (x == 0) return false;
+    const uint32_t o1 = atoms_add(a1, x);
+    return ((o1 + x) & ~o1 & DRAIN_BIT) != 0;
 }
 
 __device__ __forceinline__ ull limbs_drain(uint32_t a0, uint32_t a1, ull* hi_out) {

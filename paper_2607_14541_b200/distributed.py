@@ -4,19 +4,27 @@ The aggregation shards by records: Eq. 2 is a plain sum over independent invocat
 accumulator is an exact integer, so each rank aggregates its own slice of the trace with the
 single-GPU kernels and no data-path collective.  One exchange step makes the partial results
 global: every aggregated entry is sent to the rank that owns its key, and the owner folds what
-it receives into its table with ``atrex_agg_merge`` (exact).  Per-phase totals are combined as
-128-bit integers on the host: an element-wise reduction of the 64-bit halves would lose carries.
+it receives into its table with ``atrex_agg_merge`` (exact); Eq. 3's denominators become the sums
+of the shards' per-phase totals.
 
-Only tensor plumbing lives here (torch.distributed for the exchange); all arithmetic on the
-records stays in the CUDA kernels.  Works with the ``nccl`` backend on GPUs and with ``gloo`` on
-CPU tensors (used by the multi-process tests).
+Only plumbing lives here -- tensors handed to ``torch.distributed`` and to the C ABI.  Every piece
+of arithmetic on keys, weights and totals is a library call: the owner function
+(``atrex_key_owner``), the grouping of entries by owner (``atrex_entries_bucket_by_owner``), the
+128-bit combination of totals (``atrex_totals_combine``; an element-wise reduction of 64-bit halves
+by the collective would lose carries), the fold (``atrex_agg_merge``), the normalisation
+(``atrex_agg_finalize_with_totals``) and the ranking of the gathered candidates
+(``atrex_topk_entries_static``).  Received entries land in this GPU's own memory through plain NCCL
+receives; no kernel is handed another GPU's memory.
 """
 from __future__ import annotations
 
+import ctypes as C
+
 import numpy as np
 
+from . import binding as B
+
 ENTRY_BYTES = 48
-_MIX = np.uint64(0x9E3779B97F4A7C15)
 
 
 def shard_range(n_total: int, rank: int, world: int) -> tuple[int, int]:
@@ -26,26 +34,139 @@ def shard_range(n_total: int, rank: int, world: int) -> tuple[int, int]:
 
 
 def owner_of_keys(keys: np.ndarray, world: int) -> np.ndarray:
-    """Rank that owns each packed key (any fixed function of the key works; this one mixes the bits)."""
-    with np.errstate(over="ignore"):
-        h = np.asarray(keys, dtype=np.uint64) * _MIX
-    return ((h >> np.uint64(33)) % np.uint64(world)).astype(np.int64)
+    """Rank that owns each packed key (``atrex_keys_owner``, the library's host-side owner function)."""
+    k = np.ascontiguousarray(keys, dtype=np.uint64)
+    out = np.zeros(k.shape[0], dtype=np.uint32)
+    B.atrex_keys_owner(k.ctypes.data, k.shape[0], int(world), out.ctypes.data)
+    return out.astype(np.int64)
 
 
-def bucket_entries_by_owner(entries: np.ndarray, world: int) -> list[np.ndarray]:
-    """Split a structured array of entries into one array per destination rank."""
+# ---------------------------------------------------------------- one rank's two halves of the step
+
+class Outgoing:
+    """What one rank contributes to the exchange: its entries grouped by owner (a CUDA byte tensor),
+    the entry count per destination rank, and its per-phase totals as (lo[8], hi[8]) words."""
+
+    def __init__(self, grouped, counts, totals_lo, totals_hi):
+        self.grouped, self.counts, self.totals_lo, self.totals_hi = grouped, counts, totals_lo, totals_hi
+
+    def part_for(self, dst: int):
+        begin = sum(self.counts[:dst]) * ENTRY_BYTES
+        return self.grouped[begin: begin + self.counts[dst] * ENTRY_BYTES]
+
+
+def prepare_outgoing(local_agg, peak_bw: float, peak_flops, world: int) -> Outgoing:
+    """Sender side: finalize this rank's partial aggregate and group its entries by owner on the device."""
+    local, n = local_agg.finalize(peak_bw, peak_flops)
+    lo, hi = local_agg.totals_words()                 # the totals the finalize just computed: no second pass
+    grouped, counts = B.bucket_entries_by_owner(local, n, world)
+    return Outgoing(grouped, counts, lo, hi)
+
+
+def fold_incoming(owner_agg, received, peak_bw: float, peak_flops, totals_lo_rows, totals_hi_rows):
+    """Owner side: fold the received entries (a CUDA byte tensor, any order) into ``owner_agg``, combine the
+    shards' totals exactly and finalize the owned keys against them.  Returns (entries, n)."""
+    n = received.numel() // ENTRY_BYTES
+    if n:
+        owner_agg.merge(received, n)
+    lo, hi = B.combine_totals(totals_lo_rows, totals_hi_rows)
+    return owner_agg.finalize(peak_bw, peak_flops, global_totals=(lo, hi))
+
+
+# ---------------------------------------------------------------- the exchange over torch.distributed
+
+def exchange(outgoing: Outgoing, group=None):
+    """All-to-all of the grouped entries (``all_to_all_single``: NCCL over NVLink on GPUs) and all-gather of
+    the totals' words.  Returns (received CUDA byte tensor, lo rows [world, 8], hi rows [world, 8])."""
+    import torch
+    import torch.distributed as dist
+    world = dist.get_world_size(group)
+    dev = outgoing.grouped.device
+    send_counts = torch.tensor([c * ENTRY_BYTES for c in outgoing.counts], dtype=torch.int64, device=dev)
+    recv_counts = torch.empty_like(send_counts)
+    dist.all_to_all_single(recv_counts, send_counts, group=group)
+    recv_list = recv_counts.tolist()
+    received = torch.empty(sum(recv_list), dtype=torch.uint8, device=dev)
+    dist.all_to_all_single(received, outgoing.grouped, recv_list, send_counts.tolist(), group=group)
+    words = torch.from_numpy(np.concatenate([outgoing.totals_lo, outgoing.totals_hi]).view(np.int64).copy()).to(dev)
+    rows = [torch.empty_like(words) for _ in range(world)]
+    dist.all_gather(rows, words, group=group)
+    table = torch.stack(rows).cpu().numpy().view(np.uint64)
+    return received, table[:, :B.ATREX_MAX_PHASES].copy(), table[:, B.ATREX_MAX_PHASES:].copy()
+
+
+def aggregate_sharded(local_agg, owner_agg, peak_bw: float, peak_flops, group=None):
+    """Full multi-GPU step for one rank, after ``local_agg`` has ingested this rank's slice: group the
+    local entries by owner, exchange, fold what arrives into ``owner_agg`` and finalize the owned keys
+    against the totals over all shards.  Returns (entries, n) of the keys this rank owns."""
+    import torch.distributed as dist
+    out = prepare_outgoing(local_agg, peak_bw, peak_flops, dist.get_world_size(group))
+    received, lo_rows, hi_rows = exchange(out, group)
+    return fold_incoming(owner_agg, received, peak_bw, peak_flops, lo_rows, hi_rows)
+
+
+def global_topk(owner_agg, phase: int, k: int, group=None):
+    """Table 2's ranking over all shards: every owner's local top-k is gathered and the candidates are
+    ranked on the device (``atrex_topk_entries_static``: weighted time descending as exact integers,
+    key ascending).  Returns a numpy array of entries; world * k may be at most 65 536."""
+    import torch
+    import torch.distributed as dist
+    world = dist.get_world_size(group)
+    dev = f"cuda:{owner_agg.device}"
+    mine = owner_agg.topk(phase, k)
+    padded = np.zeros(k * ENTRY_BYTES + 8, dtype=np.uint8)
+    padded[:8] = np.array([len(mine)], dtype=np.uint64).view(np.uint8)
+    padded[8: 8 + mine.nbytes] = mine.view(np.uint8).reshape(-1)
+    send = torch.from_numpy(padded).to(dev)
+    rows = [torch.empty_like(send) for _ in range(world)]
+    dist.all_gather(rows, send, group=group)
+    return rank_candidates([r[8: 8 + int(r[:8].view(torch.int64).item()) * ENTRY_BYTES] for r in rows], phase, k)
+
+
+def rank_candidates(parts, phase: int, k: int) -> np.ndarray:
+    """The best ``k`` of the candidate entries in ``parts`` (CUDA byte tensors), ranked on the device."""
+    import torch
+    parts = [p for p in parts if p.numel()]
+    if not parts or k == 0:
+        return np.zeros(0, dtype=B.ENTRY_DTYPE)
+    cand = torch.cat(parts).contiguous()
+    out = torch.empty(k * ENTRY_BYTES, dtype=torch.uint8, device=cand.device)
+    m = B.topk_entries_static(cand, cand.numel() // ENTRY_BYTES, phase, k, out)
+    return out[: m * ENTRY_BYTES].cpu().numpy().view(B.ENTRY_DTYPE).copy()
+
+
+# ---------------------------------------------------------------- ranks run in turn inside one process
+
+class Loopback:
+    """Stands in for the collectives when several ranks are run one after the other in a single process
+    (one GPU): it is handed every rank's ``Outgoing`` and gives each destination what the all-to-all
+    would deliver, as local copies."""
+
+    def __init__(self, outgoing: list[Outgoing]):
+        self.outgoing = outgoing
+
+    def deliver(self, dst: int):
+        import torch
+        received = torch.cat([o.part_for(dst) for o in self.outgoing])
+        lo_rows = np.stack([o.totals_lo for o in self.outgoing])
+        hi_rows = np.stack([o.totals_hi for o in self.outgoing])
+        return received, lo_rows, hi_rows
+
+
+# ---------------------------------------------------------------- CPU tensors (gloo), for the host-logic tests
+
+def bucket_entries_by_owner_host(entries: np.ndarray, world: int) -> list[np.ndarray]:
+    """Split a structured array of entries into one array per destination rank (host memory; the
+    device path uses ``atrex_entries_bucket_by_owner``)."""
     owner = owner_of_keys(entries["key"], world)
     order = np.argsort(owner, kind="stable")
     bounds = np.searchsorted(owner[order], np.arange(world + 1))
     return [entries[order[bounds[r]:bounds[r + 1]]] for r in range(world)]
 
 
-def exchange_entries(buckets: list[np.ndarray], group=None, device=None) -> list[np.ndarray]:
-    """All-to-all of per-destination entry arrays.  Returns what each source rank sent to this rank.
-
-    With ``device`` set (a CUDA device) the payload travels as CUDA tensors over ``all_to_all_single``
-    (NCCL over NVLink); otherwise as CPU tensors, gathered and filtered, which every backend supports.
-    """
+def exchange_entries_host(buckets: list[np.ndarray], group=None) -> list[np.ndarray]:
+    """All-to-all of per-destination entry arrays as CPU tensors (every backend supports the all-gather
+    it is built from).  Returns what each source rank sent to this rank."""
     import torch
     import torch.distributed as dist
     world, rank = dist.get_world_size(group), dist.get_rank(group)
@@ -53,26 +174,8 @@ def exchange_entries(buckets: list[np.ndarray], group=None, device=None) -> list
     dtype = buckets[0].dtype
     counts = torch.tensor([len(b) for b in buckets], dtype=torch.int64)
     all_counts = [torch.zeros(world, dtype=torch.int64) for _ in range(world)]
-    if device is not None:
-        counts_dev = counts.to(device)
-        gathered = [torch.zeros(world, dtype=torch.int64, device=device) for _ in range(world)]
-        dist.all_gather(gathered, counts_dev, group=group)
-        all_counts = [g.cpu() for g in gathered]
-    else:
-        dist.all_gather(all_counts, counts, group=group)
+    dist.all_gather(all_counts, counts, group=group)
     incoming = [int(all_counts[src][rank]) for src in range(world)]
-    if device is not None:
-        send = torch.from_numpy(np.concatenate(buckets).view(np.uint8).reshape(-1).copy()).to(device)
-        recv = torch.empty(sum(incoming) * ENTRY_BYTES, dtype=torch.uint8, device=device)
-        dist.all_to_all_single(recv, send, [c * ENTRY_BYTES for c in incoming],
-                               [len(b) * ENTRY_BYTES for b in buckets], group=group)
-        flat = recv.cpu().numpy()
-        out, off = [], 0
-        for c in incoming:
-            out.append(flat[off:off + c * ENTRY_BYTES].view(dtype).copy())
-            off += c * ENTRY_BYTES
-        return out
-    # portable path: every rank publishes all its buckets, each rank keeps the slices addressed to it
     width = int(max(int(c.sum()) for c in all_counts))
     mine = np.zeros(width * ENTRY_BYTES, dtype=np.uint8)
     payload = np.concatenate(buckets).view(np.uint8).reshape(-1)
@@ -87,81 +190,14 @@ def exchange_entries(buckets: list[np.ndarray], group=None, device=None) -> list
     return out
 
 
-def combine_phase_totals(local_totals: list[int], group=None) -> list[int]:
-    """Sum per-phase 128-bit totals over ranks exactly (gather the halves, add as integers)."""
+def gather_totals_host(totals_lo: np.ndarray, totals_hi: np.ndarray, group=None):
+    """All-gather of one rank's totals' words as CPU tensors, combined exactly by the library.
+    Returns (lo[8], hi[8])."""
     import torch
     import torch.distributed as dist
     world = dist.get_world_size(group)
-    halves = []
-    for t in local_totals:
-        halves += [t & 0xFFFFFFFF, (t >> 32) & 0xFFFFFFFF, (t >> 64) & 0xFFFFFFFF, (t >> 96) & 0xFFFFFFFF]
-    mine = torch.tensor(halves, dtype=torch.int64)
-    everyone = [torch.zeros_like(mine) for _ in range(world)]
-    dist.all_gather(everyone, mine, group=group)
-    out = [0] * len(local_totals)
-    for t in everyone:
-        v = t.tolist()
-        for p in range(len(local_totals)):
-            out[p] += v[4 * p] | (v[4 * p + 1] << 32) | (v[4 * p + 2] << 64) | (v[4 * p + 3] << 96)
-    return out
-
-
-def merge_ranked(candidates: list[np.ndarray], k: int) -> np.ndarray:
-    """Global top-k from every rank's local top-k: weighted time descending (exact), key ascending."""
-    allc = np.concatenate(candidates) if candidates else np.zeros(0)
-    if len(allc) == 0:
-        return allc
-    wt = allc["wt_hi"].astype(object) * (1 << 64) + allc["wt_lo"].astype(object)
-    order = sorted(range(len(allc)), key=lambda i: (-wt[i], int(allc["key"][i])))
-    return allc[order[:k]]
-
-
-def owner_of_keys_torch(keys):
-    """``owner_of_keys`` on a CUDA int64 tensor of packed keys; ``world`` is applied by the caller."""
-    import torch
-    h = keys * torch.tensor(-7046029254386353131, dtype=torch.int64, device=keys.device)  # 0x9E3779B97F4A7C15
-    return (h >> 33) & 0x7FFFFFFF  # logical shift of the product's top 31 bits
-
-
-def bucket_entries_by_owner_torch(entries, n: int, world: int):
-    """Split a CUDA uint8 tensor of ``n`` 48-byte entries into per-destination tensors (on the device)."""
-    import torch
-    e = entries[: n * ENTRY_BYTES].view(torch.int64).view(n, ENTRY_BYTES // 8)
-    owner = owner_of_keys_torch(e[:, 0]) % world
-    order = torch.argsort(owner, stable=True)
-    counts = torch.bincount(owner, minlength=world).tolist()
-    sorted_e = e[order].contiguous().view(torch.uint8).view(-1)
-    out, off = [], 0
-    for c in counts:
-        out.append(sorted_e[off * ENTRY_BYTES:(off + c) * ENTRY_BYTES])
-        off += c
-    return out
-
-
-def merge_and_finalize_owned(owner_agg, parts, peak_bw, peak_flops, global_totals):
-    """Owner side of the exchange: fold the entry tensors received from every rank into
-    ``owner_agg`` (``atrex_agg_merge``) and finalize against the totals over all shards."""
-    for part in parts:
-        if part.numel():
-            owner_agg.merge(part, part.numel() // ENTRY_BYTES)
-    return owner_agg.finalize(peak_bw, peak_flops, global_totals=global_totals)
-
-
-def aggregate_sharded(local_agg, owner_agg, peak_bw, peak_flops, group=None):
-    """Full multi-GPU flow for one rank, after ``local_agg`` has ingested this rank's slice:
-    finalize locally, send every entry to its key's owner (NCCL all-to-all), fold what arrives into
-    ``owner_agg``, combine the per-phase totals exactly, and finalize the owned keys against them.
-    Returns (entries, n) of the keys this rank owns."""
-    import torch
-    import torch.distributed as dist
-    world = dist.get_world_size(group)
-    local, n = local_agg.finalize(peak_bw, peak_flops)
-    buckets = bucket_entries_by_owner_torch(local, n, world)
-    send_counts = torch.tensor([b.numel() for b in buckets], dtype=torch.int64, device=local.device)
-    recv_counts = torch.empty_like(send_counts)
-    dist.all_to_all_single(recv_counts, send_counts, group=group)
-    recv = torch.empty(int(recv_counts.sum()), dtype=torch.uint8, device=local.device)
-    dist.all_to_all_single(recv, torch.cat(buckets) if buckets else local[:0], recv_counts.tolist(),
-                           send_counts.tolist(), group=group)
-    totals = combine_phase_totals(local_agg.stats()["totals"], group=group)
-    return merge_and_finalize_owned(owner_agg, [recv], peak_bw, peak_flops, totals)
+    words = torch.from_numpy(np.concatenate([totals_lo, totals_hi]).astype(np.uint64).view(np.int64).copy())
+    rows = [torch.empty_like(words) for _ in range(world)]
+    dist.all_gather(rows, words, group=group)
+    table = torch.stack(rows).numpy().view(np.uint64)
+    return B.combine_totals(table[:, :B.ATREX_MAX_PHASES].copy(), table[:, B.ATREX_MAX_PHASES:].copy())

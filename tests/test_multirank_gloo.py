@@ -1,7 +1,8 @@
 """The multi-rank path on CPU: two gloo ranks shard a trace, exchange their partial aggregates
-by key owner, and the union must equal the single-rank result.  Per-rank aggregation and the
-fold of received entries use the CPU oracle here (no GPU on this machine); what is under test is the
-product's host-side plumbing in ``paper_2607_14541_b200.distributed``."""
+by key owner, and the union must equal the single-rank result.  Per-rank aggregation, the fold
+of received entries and the ranking use the CPU oracle here (no GPU on this machine); what is under
+test is the product's host-side plumbing in ``paper_2607_14541_b200.distributed`` and the
+library's host-callable pieces (owner function, exact combination of the totals)."""
 import os
 import socket
 
@@ -44,21 +45,23 @@ def _worker(rank, world, port, n, out_dir):
     o = oracle.Oracle(spec.app_weights, spec.n_phases)
     o.ingest(recs)
     local = o.finalize(PEAK_BW, PEAK_FLOPS)
-    received = D.exchange_entries(D.bucket_entries_by_owner(local, world))
+    received = D.exchange_entries_host(D.bucket_entries_by_owner_host(local, world))
     owned = _fold(received)
     assert all(D.owner_of_keys(np.array([k], dtype=np.uint64), world)[0] == rank for k in list(owned)[:200])
-    totals = D.combine_phase_totals(o.stats()["totals"])
+    mine_t = o.stats()["totals"]
+    lo, hi = D.gather_totals_host(np.array([t & (2**64 - 1) for t in mine_t], dtype=np.uint64),
+                                  np.array([t >> 64 for t in mine_t], dtype=np.uint64))
+    totals = [int(lo[q]) | (int(hi[q]) << 64) for q in range(8)]
     # local top-k of the owned keys -> global top-k
     ent = np.zeros(len(owned), dtype=local.dtype)
     for i, (k, (c, w)) in enumerate(sorted(owned.items())):
         ent[i] = (k, c, w & (2**64 - 1), w >> 64, 0.0, 0.0)
     tops = []
-    for phase in range(spec.n_phases):
-        sel = ent[(ent["key"] >> np.uint64(48)) == phase]
-        mine = D.merge_ranked([sel], 10)
+    for phase in range(spec.n_phases):                    # every owner's local top-10, gathered, ranked again
+        mine = oracle.rank_phase(ent, phase, 0)[0][:10]
         gathered = [None] * world
         dist.all_gather_object(gathered, mine)
-        tops.append(D.merge_ranked(gathered, 10))
+        tops.append(oracle.rank_phase(np.concatenate(gathered), phase, 0)[0][:10])
     np.save(os.path.join(out_dir, f"owned_{rank}.npy"), ent)
     if rank == 0:
         np.save(os.path.join(out_dir, "totals.npy"), np.array([str(t) for t in totals]))
@@ -96,7 +99,15 @@ def test_shard_ranges_and_owners_are_a_partition():
     keys = np.arange(100_000, dtype=np.uint64) * np.uint64(2654435761)
     own = D.owner_of_keys(keys, 8)
     assert own.min() == 0 and own.max() == 7 and np.bincount(own).min() > 100_000 / 8 * 0.9
-    # 128-bit totals survive the combination with carries out of every 32-bit piece
-    big = (1 << 127) + (1 << 64) - 1
-    halves = [big & 0xFFFFFFFF, (big >> 32) & 0xFFFFFFFF, (big >> 64) & 0xFFFFFFFF, (big >> 96) & 0xFFFFFFFF]
-    assert sum(h << (32 * i) for i, h in enumerate(halves)) == big
+    # the owner function is the same whether asked one key at a time or in bulk
+    import paper_2607_14541_b200 as p
+    assert [p.atrex_key_owner(int(k), 8) for k in keys[:100]] == [int(x) for x in own[:100]]
+    # 128-bit totals survive the combination with carries out of the low words
+    a, b, c = (1 << 127) + (1 << 64) - 1, (1 << 64) - 1, 3
+    lo = np.zeros((3, 8), dtype=np.uint64)
+    hi = np.zeros((3, 8), dtype=np.uint64)
+    for r, t in enumerate((a, b, c)):
+        lo[r, 2], hi[r, 2] = t & (2**64 - 1), t >> 64
+    out_lo, out_hi = p.combine_totals(lo, hi)
+    assert (int(out_lo[2]) | (int(out_hi[2]) << 64)) == (a + b + c) % (1 << 128)
+    assert not out_lo[[0, 1, 3, 4, 5, 6, 7]].any() and not out_hi[[0, 1, 3, 4, 5, 6, 7]].any()
