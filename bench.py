@@ -179,6 +179,15 @@ def run_ours(args):
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device(f"cuda:{local}"))
+    elif args.force_exchange:
+        # one GPU, but the step of a multi-GPU run: a process group of one rank (exercises the exchange path)
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                                device_id=torch.device(f"cuda:{local}"))
+    sharded = world > 1 or args.force_exchange
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
 
@@ -201,7 +210,7 @@ def run_ours(args):
     stream = torch.cuda.current_stream(dev)
     ingest_events = []
     owner = None
-    if world > 1:
+    if sharded:
         # several GPUs: this rank's handle holds its slice of the trace; a second handle holds the keys
         # this rank owns after the exchange step (every entry travels to its key's owner)
         from paper_2607_14541_b200 import distributed as D
@@ -289,11 +298,11 @@ def run_ours(args):
                                        f"{spec.n_apps} apps, {spec.n_ops} ops x {spec.n_shapes} shapes Zipf({spec.zipf_s})",
                            "records_per_gpu": n, "chunks": n_chunks, "live_keys": int(n_keys),
                            "l2": "inputs (16 GiB per step) exceed L2; no flush needed",
-                           "step": ("reset + ingest x chunks + finalize + topk per phase" if world == 1 else
+                           "step": ("reset + ingest x chunks + finalize + topk per phase" if not sharded else
                                     "reset + ingest x chunks + exchange step (entries grouped by key owner, NCCL "
                                     "all-to-all, merge at the owner, totals combined, finalize of the owned keys) "
                                     "+ global topk per phase (owners' candidates gathered and ranked)"),
-                           "live_keys_is": "keys of this GPU's trace" if world == 1 else "keys rank 0 owns",
+                           "live_keys_is": "keys of this GPU's trace" if not sharded else "keys rank 0 owns",
                            "workspace_bytes_per_handle": agg.workspace_bytes,
                            "parallelism": f"trace sharded by records x{world}"},
                 "clocks": clocks, "gpu_launches": int(launches), "roofline": roofline,
@@ -304,12 +313,13 @@ def run_ours(args):
                            "steps": e2e["steps"], "sample": e2e["sample"]}
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(args, spec, records, torch)
-        if world == 1 and not args.no_per_config:
+        if world == 1 and not args.no_per_config and not sharded:
             del agg
             line["per_config"] = per_config(torch, p, records, n, peak)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
+    if sharded:
         dist.destroy_process_group()
 
 
@@ -431,6 +441,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-config", action="store_true")
+    ap.add_argument("--force-exchange", action="store_true",
+                    help="with one GPU: run the step of a multi-GPU run (exchange, merge, global top-k) in a process group of one rank")
     ap.add_argument("--cpu-records", type=int, default=1 << 25)
     ap.add_argument("--ref-records", type=int, default=1 << 24)
     ap.add_argument("--ncu-traffic-bytes", type=float, default=None,
