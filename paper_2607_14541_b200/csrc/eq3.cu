@@ -6,8 +6,12 @@
 //          w_i = wtilde_i / sum over retained j of wtilde_j
 //
 // The group-by runs over (operator, application, phase) cells, a space of at most a few million
-// cells that stays resident in L2, so ingest is one 64-bit atomic add per record (plus a counted
-// carry into a second limb).  The floating-point part sums in ascending phase, application and
+// cells that stays resident in L2.  With uniformly spread applications no subset of the cells is hot
+// and equal cells hardly ever meet inside a warp, so there is nothing to pre-aggregate: ingest is one
+// 64-bit reduction per record into L2, and what matters is that it does not return a value.  While
+// fewer than 2^32 records have been ingested no cell can overflow 64 bits (durations are below 2^32),
+// so the reduction is fire-and-forget; from then on every add returns the old value and wraps are
+// counted in a second limb.  The floating-point part sums in ascending phase, application and
 // operator order with every operation rounded once, which gives one bit pattern.
 #include <cmath>
 #include <new>
@@ -28,6 +32,7 @@ struct atrex_eq3 {
     uint8_t* d_ret = nullptr;     // [n_ops] retained flags
     ull* d_rejected = nullptr;
     size_t cells = 0;
+    ull n_ingested = 0;           // records handed to ingest since create/reset (decides the carry handling)
 };
 
 namespace {
@@ -43,20 +48,56 @@ struct Guard {
     }
 };
 
-__global__ void __launch_bounds__(512) eq3_ingest_kernel(const uint4* __restrict__ recs, ull n, uint32_t n_apps, uint32_t n_ops,
-                                                         uint32_t n_phases, ull* lo, ull* hi, ull* rejected) {
-    uint32_t bad = 0;
-    for (ull i = (ull)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (ull)gridDim.x * blockDim.x) {
-        const uint4 r = __ldcs(recs + i);
-        const uint32_t app = r.x, op = r.y & 0xFFFFu, phase = (r.y >> 16) & 0xFFu;
-        if (app >= n_apps || op >= n_ops || phase >= n_phases) {
-            ++bad;
-            continue;
-        }
-        const size_t cell = ((size_t)phase * n_ops + op) * n_apps + app;
-        const ull d = r.w;
-        const ull old = atomicAdd(&lo[cell], d);
+__device__ __forceinline__ void red_add_u64(ull* p, ull v) {
+    asm volatile("red.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// One record's duration into its cell.  CARRY: the low limb may wrap, so the add returns the old value.
+template <bool CARRY>
+__device__ __forceinline__ uint32_t eq3_add(uint32_t app, uint32_t w1, uint32_t dur, uint32_t n_apps, uint32_t n_ops,
+                                            uint32_t n_phases, ull* lo, ull* hi) {
+    const uint32_t op = w1 & 0xFFFFu, phase = (w1 >> 16) & 0xFFu;
+    if (app >= n_apps || op >= n_ops || phase >= n_phases) return 1u;
+    const size_t cell = ((size_t)phase * n_ops + op) * n_apps + app;
+    if (CARRY) {
+        const ull d = dur, old = atomicAdd(&lo[cell], d);
         if (old + d < old) atomicAdd(&hi[cell], 1ull);
+    } else {
+        red_add_u64(&lo[cell], (ull)dur);
+    }
+    return 0u;
+}
+
+// Two records per 32-byte load, two loads in flight per thread.
+template <bool CARRY>
+__global__ void __launch_bounds__(512) eq3_ingest_kernel(const unsigned char* __restrict__ body, ull n_pairs, const uint4* head,
+                                                         const uint4* tail, uint32_t n_apps, uint32_t n_ops, uint32_t n_phases,
+                                                         ull* lo, ull* hi, ull* rejected) {
+    uint32_t bad = 0;
+    const ull stride = (ull)gridDim.x * blockDim.x;
+    for (ull i = (ull)blockIdx.x * blockDim.x + threadIdx.x; i < n_pairs; i += 2 * stride) {
+        uint32_t a[8], b[8];
+        const bool second = i + stride < n_pairs;
+        asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]), "=r"(a[4]), "=r"(a[5]), "=r"(a[6]), "=r"(a[7])
+                     : "l"(body + i * 32));
+        if (second)
+            asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(b[0]), "=r"(b[1]), "=r"(b[2]), "=r"(b[3]), "=r"(b[4]), "=r"(b[5]), "=r"(b[6]), "=r"(b[7])
+                         : "l"(body + (i + stride) * 32));
+        bad += eq3_add<CARRY>(a[0], a[1], a[3], n_apps, n_ops, n_phases, lo, hi);
+        bad += eq3_add<CARRY>(a[4], a[5], a[7], n_apps, n_ops, n_phases, lo, hi);
+        if (second) {
+            bad += eq3_add<CARRY>(b[0], b[1], b[3], n_apps, n_ops, n_phases, lo, hi);
+            bad += eq3_add<CARRY>(b[4], b[5], b[7], n_apps, n_ops, n_phases, lo, hi);
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 2) {   // records outside the 32-byte aligned body
+        const uint4* one = threadIdx.x == 0 ? head : tail;
+        if (one) {
+            const uint4 r = *one;
+            bad += eq3_add<CARRY>(r.x, r.y, r.w, n_apps, n_ops, n_phases, lo, hi);
+        }
     }
     bad = __reduce_add_sync(0xFFFFFFFFu, bad);
     if ((threadIdx.x & 31u) == 0 && bad) atomicAdd(rejected, (ull)bad);
@@ -79,28 +120,47 @@ __global__ void eq3_app_totals_kernel(const ull* lo, const ull* hi, uint32_t n_a
     tot[2 * idx + 1] = s_hi;
 }
 
-// wtilde_i: one warp per operator finds Phi_i in parallel, then lane 0 sums over the
-// applications in order (the order is part of the result)
-__global__ void __launch_bounds__(32) eq3_wtilde_kernel(const ull* lo, const ull* hi, const ull* tot, const uint32_t* appw,
-                                                        uint32_t n_apps, uint32_t n_ops, uint32_t n_phases, double* wt) {
-    const uint32_t i = blockIdx.x, lane = threadIdx.x;
-    uint32_t present = 0;  // bit phi: operator i has time in phase phi
-    for (uint32_t p = 0; p < n_phases; ++p) {
-        bool any = false;
-        for (uint32_t a = lane; a < n_apps; a += 32) {
-            const size_t cell = ((size_t)p * n_ops + i) * n_apps + a;
-            any |= (lo[cell] | hi[cell]) != 0;
-        }
-        if (__any_sync(0xFFFFFFFFu, any)) present |= 1u << p;
+// wtilde_i: one CTA per operator.  The CTA finds Phi_i, then every thread works out the terms
+// p_a * (1/|Phi_i|) * sum_phi D[i][a][phi] / D_a[phi] of its applications (each a fixed sequence of
+// rounded operations, independent of the others) into shared memory in chunks; only the running sum
+// over the applications, whose order is part of the result, is left to one thread.
+constexpr int WT_THREADS = 256;
+constexpr uint32_t WT_CHUNK = 2048;   // terms held in shared memory at a time
+
+__global__ void __launch_bounds__(WT_THREADS) eq3_wtilde_kernel(const ull* lo, const ull* hi, const ull* tot, const uint32_t* appw,
+                                                                uint32_t n_apps, uint32_t n_ops, uint32_t n_phases, double* wt) {
+    __shared__ double s_term[WT_CHUNK];
+    __shared__ uint32_t s_present;
+    __shared__ ull s_weights;
+    const uint32_t i = blockIdx.x;
+    if (threadIdx.x == 0) {
+        s_present = 0;
+        s_weights = 0;
     }
-    if (lane != 0) return;
-    ull c_lo = 0;
-    for (uint32_t a = 0; a < n_apps; ++a) c_lo += appw[a];  // < 2^64: n_apps < 2^32 weights < 2^32
-    double acc = 0.0;
+    __syncthreads();
+    uint32_t present = 0;  // bit phi: operator i has time in phase phi
+    ull c_part = 0;
+    for (uint32_t a = threadIdx.x; a < n_apps; a += WT_THREADS) {
+        c_part += appw[a];  // < 2^64 in total: fewer than 2^32 weights below 2^32
+        for (uint32_t p = 0; p < n_phases; ++p) {
+            const size_t cell = ((size_t)p * n_ops + i) * n_apps + a;
+            if ((lo[cell] | hi[cell]) != 0) present |= 1u << p;
+        }
+    }
+    if (present) atomicOr(&s_present, present);
+    atomicAdd(&s_weights, c_part);
+    __syncthreads();
+    present = s_present;
+    const ull c_lo = s_weights;
     const int n_phi = __popc(present);
-    if (n_phi != 0 && c_lo != 0) {
-        const double c_total = __ull2double_rn(c_lo), d_phi = (double)n_phi;
-        for (uint32_t a = 0; a < n_apps; ++a) {
+    if (n_phi == 0 || c_lo == 0) {
+        if (threadIdx.x == 0) wt[i] = 0.0;
+        return;
+    }
+    const double c_total = __ull2double_rn(c_lo), d_phi = (double)n_phi;
+    double acc = 0.0;   // thread 0's
+    for (uint32_t a0 = 0; a0 < n_apps; a0 += WT_CHUNK) {
+        for (uint32_t a = a0 + threadIdx.x; a < min(a0 + WT_CHUNK, n_apps); a += WT_THREADS) {
             double inner = 0.0;
             for (uint32_t p = 0; p < n_phases; ++p) {
                 if (!(present & (1u << p))) continue;
@@ -112,10 +172,14 @@ __global__ void __launch_bounds__(32) eq3_wtilde_kernel(const ull* lo, const ull
             }
             const double avg = __ddiv_rn(inner, d_phi);
             const double p_a = __ddiv_rn(__ull2double_rn((ull)appw[a]), c_total);
-            acc = __dadd_rn(acc, __dmul_rn(p_a, avg));
+            s_term[a - a0] = __dmul_rn(p_a, avg);
         }
+        __syncthreads();
+        if (threadIdx.x == 0)
+            for (uint32_t a = a0; a < min(a0 + WT_CHUNK, n_apps); ++a) acc = __dadd_rn(acc, s_term[a - a0]);
+        __syncthreads();
     }
-    wt[i] = acc;
+    if (threadIdx.x == 0) wt[i] = acc;
 }
 
 __global__ void eq3_normalise_kernel(const double* wt, const uint8_t* retained, uint32_t n_ops, double* w) {
@@ -185,6 +249,7 @@ int atrex_eq3_reset(atrex_eq3_t* h, void* stream) {
     if (cudaMemsetAsync(h->d_lo, 0, h->cells * 8, s) != cudaSuccess || cudaMemsetAsync(h->d_hi, 0, h->cells * 8, s) != cudaSuccess ||
         cudaMemsetAsync(h->d_rejected, 0, 8, s) != cudaSuccess)
         return ATREX_ERR_CUDA;
+    h->n_ingested = 0;
     return ATREX_OK;
 }
 
@@ -193,10 +258,24 @@ int atrex_eq3_ingest(atrex_eq3_t* h, const atrex_record_t* d_records, uint64_t n
     if (n == 0) return ATREX_OK;
     if (!d_records || ((uintptr_t)d_records & 15u)) return ATREX_ERR_INVALID;
     Guard g(h->device);
-    ull blocks = (n + 511) / 512;
+    // the 32-byte aligned body as record pairs; at most one record before and one after it
+    const unsigned char* base = (const unsigned char*)d_records;
+    const uint64_t head = ((uintptr_t)base & 31u) ? 1 : 0;
+    const uint64_t n_body = n - head, n_pairs = n_body / 2;
+    const uint4* head_rec = head ? (const uint4*)base : nullptr;
+    const uint4* tail_rec = (n_body & 1) ? (const uint4*)(base + (n - 1) * 16) : nullptr;
+    ull blocks = (n_pairs + 1023) / 1024;
     if (blocks > (ull)h->n_sms * 4) blocks = (ull)h->n_sms * 4;
-    eq3_ingest_kernel<<<(unsigned)blocks, 512, 0, (cudaStream_t)stream>>>((const uint4*)d_records, n, h->n_apps, h->n_ops,
-                                                                         h->n_phases, h->d_lo, h->d_hi, h->d_rejected);
+    if (blocks == 0) blocks = 1;
+    // below 2^32 records in total no cell's 64-bit sum can wrap: fire-and-forget reductions
+    const bool carry = h->n_ingested + n >= (1ull << 32);
+    h->n_ingested += n;
+    if (carry)
+        eq3_ingest_kernel<true><<<(unsigned)blocks, 512, 0, (cudaStream_t)stream>>>(base + head * 16, n_pairs, head_rec, tail_rec, h->n_apps,
+                                                                                    h->n_ops, h->n_phases, h->d_lo, h->d_hi, h->d_rejected);
+    else
+        eq3_ingest_kernel<false><<<(unsigned)blocks, 512, 0, (cudaStream_t)stream>>>(base + head * 16, n_pairs, head_rec, tail_rec, h->n_apps,
+                                                                                     h->n_ops, h->n_phases, h->d_lo, h->d_hi, h->d_rejected);
     return cudaGetLastError() == cudaSuccess ? ATREX_OK : ATREX_ERR_CUDA;
 }
 
@@ -217,7 +296,7 @@ int atrex_eq3_finalize(atrex_eq3_t* h, const uint8_t* h_retained, double* h_w, d
     if (e != cudaSuccess) return ATREX_ERR_CUDA;
     const size_t pa = (size_t)h->n_phases * h->n_apps;
     eq3_app_totals_kernel<<<(unsigned)((pa + 255) / 256), 256, 0, s>>>(h->d_lo, h->d_hi, h->n_apps, h->n_ops, h->n_phases, h->d_tot);
-    eq3_wtilde_kernel<<<h->n_ops, 32, 0, s>>>(h->d_lo, h->d_hi, h->d_tot, h->d_appw, h->n_apps, h->n_ops, h->n_phases, h->d_wt);
+    eq3_wtilde_kernel<<<h->n_ops, WT_THREADS, 0, s>>>(h->d_lo, h->d_hi, h->d_tot, h->d_appw, h->n_apps, h->n_ops, h->n_phases, h->d_wt);
     eq3_normalise_kernel<<<1, 256, 0, s>>>(h->d_wt, h->d_ret, h->n_ops, h->d_w);
     if (cudaGetLastError() != cudaSuccess) return ATREX_ERR_CUDA;
     e = cudaMemcpyAsync(h_w, h->d_w, (size_t)h->n_ops * 8, cudaMemcpyDeviceToHost, s);

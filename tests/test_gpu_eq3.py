@@ -48,3 +48,36 @@ def test_eq3_parity(index, n):
     ow.reset()
     w, wt, rej = ow.finalize()
     assert not w.any() and not wt.any() and rej == 0
+
+
+def test_eq3_beyond_two_to_the_32_records_switches_to_counted_carries():
+    """Below 2^32 ingested records no 64-bit cell sum can wrap and ingest uses fire-and-forget
+    reductions; from the 2^32-th record on every add returns the old value and wraps are counted.
+    A 2^26-record trace is ingested 64 times (the 64th pass crosses the line) and a second trace once
+    more.  Cell sums are linear in the durations, so the oracle gets the equivalent trace: the first
+    one with every duration multiplied by 64 (they stay below 2^32), followed by the second."""
+    import torch
+    import paper_2607_14541_b200 as p
+    rng = np.random.default_rng(2024)
+    n_apps, n_ops, n_phases, n_x, n_y = 64, 16, 2, 1 << 26, (1 << 20) + 3
+
+    def trace(n):
+        r = np.zeros(n, dtype=tg.RECORD_DTYPE)
+        r["app_id"] = rng.integers(0, n_apps, n, dtype=np.uint32)
+        r["op_id"] = rng.integers(0, n_ops, n).astype(np.uint16)
+        r["phase"] = rng.integers(0, n_phases, n).astype(np.uint8)
+        r["shape_id"] = rng.integers(0, 1 << 20, n, dtype=np.uint32)
+        r["duration_ns"] = rng.integers(1, 1 << 26, n, dtype=np.uint32)
+        return r
+    x, y = trace(n_x), trace(n_y)
+    weights = rng.integers(1, 1 << 20, n_apps, dtype=np.uint32)
+    ow = p.OperatorWeights(weights, n_ops, n_phases)
+    dx, dy = to_dev(x), to_dev(y)
+    for _ in range(64):
+        ow.ingest(dx, n=n_x)
+    ow.ingest(dy, n=n_y)
+    w, wt, rej = ow.finalize()
+    x["duration_ns"] *= np.uint32(64)
+    ew, ewt, erej = oracle.eq3_weights(np.concatenate([x, y]), weights, n_ops, n_phases)
+    assert rej == erej == 0
+    assert wt.tobytes() == ewt.tobytes() and w.tobytes() == ew.tobytes()
