@@ -62,7 +62,8 @@ typedef enum {
     ATREX_ERR_TIMEOUT = -5,        /* a bounded device-side wait gave up                                */
     ATREX_ERR_STATE = -6,          /* call order: topk before finalize, or > 2^40 records               */
     ATREX_ERR_NOMEM = -7,          /* workspace too small / allocation failed                           */
-    ATREX_ERR_TOO_LARGE = -8       /* input larger than a fixed-size internal buffer can take           */
+    ATREX_ERR_TOO_LARGE = -8,      /* input larger than a fixed-size internal buffer can take           */
+    ATREX_ERR_BOUNDS = -9          /* checked build only: a kernel computed an index outside its array  */
 } atrex_status_t;
 
 /* One observed device-kernel invocation (Sec. 3.1; the d_{a,phi,r,l} of Eq. 2). 16 bytes. */
@@ -216,6 +217,12 @@ int atrex_entries_bucket_by_owner(const atrex_entry_t* d_entries, uint64_t n, ui
  * halves by a collective would lose the carries). */
 int atrex_totals_combine(const uint64_t* h_lo, const uint64_t* h_hi, uint32_t n_ranks, uint64_t* h_out_lo,
                          uint64_t* h_out_hi);
+
+/* 1 if this library was built with -DATREX_DEBUG_BOUNDS, else 0.  In that build every index the
+ * ingest kernels form into the key table, the spill buffers and their shared-memory arrays is range
+ * checked; a violation substitutes a valid index, latches a status bit and makes the next finalize /
+ * stats return ATREX_ERR_BOUNDS (nothing traps).  The regular build has no such checks. */
+int atrex_build_has_bounds_checks(void);
 
 /* Table 2: the min(k, keys of `phase`) entries with the largest weighted time, compared as
  * exact 128-bit integers, ties broken by ascending key; written in that order to `h_out`

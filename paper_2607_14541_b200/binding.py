@@ -12,7 +12,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libatrex_agg.so")
+# ATREX_AGG_LIBRARY selects another build of the same library (e.g. the bounds-checked one)
+LIB_PATH = os.environ.get("ATREX_AGG_LIBRARY") or os.path.join(_HERE, "libatrex_agg.so")
 
 ATREX_MAX_PHASES = 8
 ATREX_MAX_DTYPES = 8
@@ -28,6 +29,7 @@ ATREX_ERR_TIMEOUT = -5
 ATREX_ERR_STATE = -6
 ATREX_ERR_NOMEM = -7
 ATREX_ERR_TOO_LARGE = -8
+ATREX_ERR_BOUNDS = -9
 ATREX_RELEASE_MAX_ENTRIES = 1 << 28
 ATREX_STATIC_TOPK_MAX_ENTRIES = 65536
 ATREX_MAX_WORLD = 1024
@@ -46,7 +48,7 @@ EXPORTED_SYMBOLS = [
     "atrex_agg_finalize_with_totals", "atrex_score_aggregate", "atrex_eq3_create", "atrex_eq3_ingest",
     "atrex_eq3_finalize", "atrex_eq3_reset", "atrex_eq3_destroy", "atrex_release_scratch_bytes",
     "atrex_entries_sort_by_key", "atrex_entries_rank", "atrex_agg_totals", "atrex_key_owner", "atrex_keys_owner",
-    "atrex_entries_bucket_by_owner", "atrex_totals_combine",
+    "atrex_entries_bucket_by_owner", "atrex_totals_combine", "atrex_build_has_bounds_checks",
 ]
 
 
@@ -112,6 +114,7 @@ def _load():
     L.atrex_release_scratch_bytes.argtypes = [u64]
     L.atrex_entries_sort_by_key.argtypes = [vp, u64, vp, vp, u64, vp]
     L.atrex_entries_rank.argtypes = [vp, u64, u32, u32, vp, vp, u64, C.POINTER(atrex_rank_result_t), vp, u64, vp]
+    L.atrex_build_has_bounds_checks.argtypes = []
     L.atrex_agg_totals.argtypes = [vp, vp, vp]
     L.atrex_key_owner.restype = u32
     L.atrex_key_owner.argtypes = [u64, u32]
@@ -152,6 +155,7 @@ atrex_release_scratch_bytes = lib.atrex_release_scratch_bytes
 atrex_entries_sort_by_key = lib.atrex_entries_sort_by_key
 atrex_entries_rank = lib.atrex_entries_rank
 atrex_agg_totals = lib.atrex_agg_totals
+atrex_build_has_bounds_checks = lib.atrex_build_has_bounds_checks
 atrex_key_owner = lib.atrex_key_owner
 atrex_keys_owner = lib.atrex_keys_owner
 atrex_entries_bucket_by_owner = lib.atrex_entries_bucket_by_owner

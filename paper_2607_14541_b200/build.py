@@ -31,5 +31,19 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+DEBUG_LIB = os.path.join(_HERE, "libatrex_agg_checked.so")
+
+
+def build_checked(force: bool = False) -> str:
+    """The same library with -DATREX_DEBUG_BOUNDS: every kernel index is range checked (see
+    atrex_build_has_bounds_checks in the header).  Select it with ATREX_AGG_LIBRARY=<path>."""
+    srcs = [os.path.join(CSRC, s) for s in SOURCES]
+    deps = srcs + [os.path.normpath(os.path.join(CSRC, h)) for h in HEADERS]
+    if force or _stale(DEBUG_LIB, deps):
+        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+        subprocess.check_call([nvcc] + NVCC_FLAGS + ["-DATREX_DEBUG_BOUNDS", "-o", DEBUG_LIB] + srcs)
+    return DEBUG_LIB
+
+
 if __name__ == "__main__":
     print(build(force=True, verbose=True))

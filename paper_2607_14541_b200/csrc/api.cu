@@ -217,6 +217,7 @@ struct atrex_agg {
     } while (0)
 
 static int device_status_to_error(const Control* c) {
+    if (c->status & ST_BOUNDS) return ATREX_ERR_BOUNDS;
     if (c->status & ST_TIMEOUT) return ATREX_ERR_TIMEOUT;
     if (c->status & ST_TABLE_FULL) return ATREX_ERR_CAPACITY;
     return ATREX_OK;
@@ -794,8 +795,17 @@ const char* atrex_strerror(int status) {
         case ATREX_ERR_STATE: return "call not valid in this state";
         case ATREX_ERR_NOMEM: return "workspace too small or allocation failed";
         case ATREX_ERR_TOO_LARGE: return "input larger than the fixed internal buffer";
+        case ATREX_ERR_BOUNDS: return "checked build: a kernel index was out of range";
         default: return "unknown status";
     }
+}
+
+int atrex_build_has_bounds_checks(void) {
+#ifdef ATREX_DEBUG_BOUNDS
+    return 1;
+#else
+    return 0;
+#endif
 }
 
 int atrex_agg_last_cuda_error(const atrex_agg_t* h) { return h ? h->last_cuda_error : 0; }

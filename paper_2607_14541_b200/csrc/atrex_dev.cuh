@@ -46,6 +46,7 @@ constexpr ull ST_WORK_DUP = 2;
 constexpr ull ST_WORK_FULL = 4;
 constexpr ull ST_WORK_DTYPE = 8;
 constexpr ull ST_TIMEOUT = 16;
+constexpr ull ST_BOUNDS = 32;   // debug build: an index was outside its array
 
 constexpr int TOPK_BINS = 4096;       // 12-bit digits
 constexpr int TOPK_DIGITS = 12;       // 144-bit composite = 88-bit weighted time, 56-bit ~key
@@ -106,6 +107,23 @@ __device__ __forceinline__ ull pack_key(uint32_t phase, uint32_t op, uint32_t sh
     return ((ull)phase << 48) | ((ull)op << 32) | (ull)shape;
 }
 
+// Debug build (-DATREX_DEBUG_BOUNDS): every index into the key table, the work table, the spill buffers
+// and the kernels' shared-memory arrays goes through ATREX_INDEX, which latches ST_BOUNDS in the control
+// block and substitutes index 0 when the index is outside [0, limit) -- the access then touches valid
+// memory and the violation is reported as ATREX_ERR_BOUNDS by the next finalize / stats (nothing traps).
+// In the regular build the macro is the index itself.
+#ifdef ATREX_DEBUG_BOUNDS
+template <typename I, typename L>
+__device__ __forceinline__ I checked_index(I i, L limit, ull* status) {
+    if ((ull)i < (ull)limit) return i;
+    atomicOr(status, ST_BOUNDS);
+    return (I)0;
+}
+#define ATREX_INDEX(i, limit, ctl) atrex::checked_index((i), (limit), &(ctl)->status)
+#else
+#define ATREX_INDEX(i, limit, ctl) (i)
+#endif
+
 __device__ __forceinline__ ull ld_relaxed(const ull* p) {
     ull v;
     asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p));
@@ -151,7 +169,7 @@ __device__ __forceinline__ ull find_or_claim(const TableRef& t, ull key, uint32_
     uint32_t s = local_of(h, (uint32_t)(key >> 48), t.C) & ~1u;
     const uint32_t advance = 2u * stride_of(t, stride_index(h));
     for (uint32_t probe = 0; probe < t.C; ++probe) {
-        ull* kp = t.keys + base + s;
+        ull* kp = t.keys + ATREX_INDEX(base + s, (ull)t.C << t.lp, t.ctl);
         ull k = ld_relaxed(kp);
         if (k == skey) return base + s;
         if (k == 0) {
@@ -171,7 +189,7 @@ __device__ __forceinline__ ull find_or_claim(const TableRef& t, ull key, uint32_
 // Exact, order-independent accumulation of (count, v_hi * 2^64 + v_lo) into a slot: the
 // thread whose add wraps `lo` is unique, and it alone adds the carry.
 __device__ __forceinline__ void slot_add(const TableRef& t, ull idx, ull v_lo, ull v_hi, ull count) {
-    ull* v = reinterpret_cast<ull*>(t.vals + idx);
+    ull* v = reinterpret_cast<ull*>(t.vals + ATREX_INDEX(idx, (ull)t.C << t.lp, t.ctl));
     ull carry = 0;
     if (v_lo != 0) {
         ull old = atomicAdd(v, v_lo);

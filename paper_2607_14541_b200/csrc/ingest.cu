@@ -199,7 +199,7 @@ __device__ __forceinline__ uint32_t probe_general(const PartSmem& m, ull skey, u
     uint32_t steps = 0;
     while (__any_sync(0xFFFFFFFFu, busy)) {
         if (busy) {
-            const ulonglong2 kk = lds_v2u64(m.keys + slot * 8);
+            const ulonglong2 kk = lds_v2u64(m.keys + ATREX_INDEX(slot, C - 1u, ctl) * 8);
             const bool hit1 = kk.y == skey;
             if (kk.x == skey || hit1) {
                 slot += hit1 ? 1u : 0u;
@@ -230,7 +230,8 @@ __device__ __forceinline__ uint32_t probe_general(const PartSmem& m, ull skey, u
 
 // One entry's product and count into its slot's limbs; the adder that fills the high limb moves the
 // slot's sums to HBM (this CTA owns the slot, so those adds are exact; the write-back adds on top).
-__device__ __forceinline__ void part_accumulate(const PartSmem& m, uint32_t slot, ull v, ulonglong2* vals_of_partition) {
+__device__ __forceinline__ void part_accumulate(const PartSmem& m, uint32_t slot, ull v, ulonglong2* vals_of_partition, uint32_t C, Control* ctl) {
+    slot = ATREX_INDEX(slot, C, ctl);
     if (limbs_add(m.a0 + slot * 4, m.a1 + slot * 4, m.cnt + slot * 4, v, 1u)) {
         ull hi, lo = limbs_drain(m.a0 + slot * 4, m.a1 + slot * 4, &hi);
         ull* vp = reinterpret_cast<ull*>(vals_of_partition + slot);
@@ -349,7 +350,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 // of slots of their probe sequence, and most new keys find room there.
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const ulonglong2 kk = lds_v2u64(m.keys + slot[u] * 8);
+                    const ulonglong2 kk = lds_v2u64(m.keys + ATREX_INDEX(slot[u], C - 1u, q.t.ctl) * 8);
                     const bool hit1 = kk.y == skey[u];
                     if (hit1) slot[u] += 1;
                     if (kk.x == skey[u] || hit1) {
@@ -382,7 +383,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         if (searching[u] && qbase + before[u] < queue_cap_w) {
-                            my_queue[qbase + before[u]] = make_ulonglong2(~skey[u], v[u]);
+                            my_queue[ATREX_INDEX(qbase + before[u], queue_cap_w, q.t.ctl)] = make_ulonglong2(~skey[u], v[u]);
                             searching[u] = false;
                             ok[u] = false;
                         }
@@ -433,7 +434,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (ok[u]) part_accumulate(m, slot[u], v[u], q.t.vals + base);
+                    if (ok[u]) part_accumulate(m, slot[u], v[u], q.t.vals + base, C, q.t.ctl);
             }
         }
         {   // this warp's queued entries, one per lane (other warps may still be streaming: the general
@@ -445,7 +446,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 const uint32_t hh = hash32(ent.x);
                 const uint32_t start = local_of(hh, (uint32_t)(ent.x >> 48), C) & ~1u;
                 const uint32_t found = probe_general(m, ~ent.x, start, 2u * stride_of(q.t, stride_index(hh)), serving, C, q.t.ctl);
-                if (serving && found != PROBE_FAILED) part_accumulate(m, found, ent.y, q.t.vals + base);
+                if (serving && found != PROBE_FAILED) part_accumulate(m, found, ent.y, q.t.vals + base, C, q.t.ctl);
             }
         }
         __syncthreads();

@@ -147,7 +147,7 @@ __device__ __noinline__ void table_route(TableRef t, ull key, uint32_t h, ull pr
 template <uint32_t LP>
 __device__ __forceinline__ void dir_add(const IngestParams& p, const Ctx& c, uint32_t slot, ull v, uint32_t count, ull key,
                                         uint32_t h) {
-    const uint32_t acc = c.sb + Smem<LP>::ACC + slot * 12u;
+    const uint32_t acc = c.sb + Smem<LP>::ACC + ATREX_INDEX(slot, Smem<LP>::SLOTS, p.t.ctl) * 12u;
     const uint32_t v0 = (uint32_t)v;
     const uint32_t o0 = atoms_add(acc, v0);
     reds_add(acc + 8, count);
@@ -173,7 +173,7 @@ __device__ __forceinline__ void spill_turn(const IngestParams& p, const Ctx& c, 
     if (pos & 1u) {
         const ulonglong2 first = lds_v2u64(mb);                    // shared-memory accesses of a thread are performed
         reds_add(cw, 0x10000u + zero_after(first.x));              // in program order; frees the mailbox only after the load
-        stg_sector(c.my_spill + (size_t)(part * p.cap + pos - 1u) * 16u, first.x, first.y, key, prod);
+        stg_sector(c.my_spill + (size_t)ATREX_INDEX(part * p.cap + pos - 1u, (p.cap << LP) - 1u, p.t.ctl) * 16u, first.x, first.y, key, prod);
     } else {
         sts_v2u64(mb, key, prod);
         reds_add(cw, 0x10000u);
@@ -192,7 +192,7 @@ constexpr uint32_t SPILL_WAIT_ROUNDS = 1u << 20;
 // Called by all lanes of a warp together; `todo` lanes append.
 template <uint32_t LP, bool PAIR>
 __device__ __forceinline__ void spill_append(const IngestParams& p, Ctx& c, bool todo, ull key, ull prod, uint32_t h) {
-    const uint32_t part = h >> (32 - LP);
+    const uint32_t part = ATREX_INDEX(h >> (32 - LP), Smem<LP>::P, p.t.ctl);
     const uint32_t cw = c.sb + Smem<LP>::CUR + part * 4u;
     if (PAIR) {
         uint32_t tk = 0;
@@ -227,7 +227,7 @@ __device__ __forceinline__ void spill_append(const IngestParams& p, Ctx& c, bool
         // that line is pulled into L2 (a partial store into a line that is not cached stalls on a fill)
         const uint32_t tk = atoms_add(cw, 1u);
         if (tk < p.cap) {
-            unsigned char* at = c.my_spill + (size_t)(part * p.cap + tk) * 16u;
+            unsigned char* at = c.my_spill + (size_t)ATREX_INDEX(part * p.cap + tk, p.cap << LP, p.t.ctl) * 16u;
             *reinterpret_cast<ulonglong2*>(at) = make_ulonglong2(key, prod);
             if ((tk & 7u) == 6) asm volatile("prefetch.global.L2 [%0];" ::"l"(at + 32));
         } else {
@@ -266,10 +266,10 @@ __device__ __forceinline__ void one_record(const IngestParams& p, Ctx& c, uint32
         // 8-byte key.  A wrong tag match (1 in 64 look-ups) fails the confirmation and the record takes
         // the spill path: slower, still exact.
         const uint32_t x = dir_mix(h, khi >> 16, c.mult);
-        const uint32_t b = __umulhi(x, L::NB);
+        const uint32_t b = ATREX_INDEX(__umulhi(x, L::NB), L::NB, p.t.ctl);
         const uint32_t t = lds_u32(c.sb + L::TAG + b * 4u) ^ __byte_perm(x, 0, 0);   // 0 in the bytes that match
         const uint32_t m = (t - 0x01010101u) & ~t & 0x80808080u;                      // lowest flagged byte is exact
-        const uint32_t at = b * DIR_WAYS + ((uint32_t)__clz((int)__brev(m)) >> 3);
+        const uint32_t at = ATREX_INDEX(b * DIR_WAYS + ((uint32_t)__clz((int)__brev(m)) >> 3), L::SLOTS + DIR_WAYS, p.t.ctl);
         bool hit = todo && m != 0 && lds_u64(c.sb + L::KEYS + at * 8u) == key;
         if (DEDUPE) {
             // one key dominates the trace: combine the lanes that share the first hitting lane's slot
