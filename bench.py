@@ -30,10 +30,13 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "trace records aggregated/sec"
-# DRAM bytes (read + written) per 2^27-record ingest call of this workload, from the ncu captures
-# summarised under profiles/: scatter_kernel 4.47 GB per launch plus
-# the two real partition drains of a step (12.20 GB) spread over its eight calls.
-NCU_DRAM_BYTES_PER_INGEST_CALL = 5.99e9
+# DRAM bytes (read + written) per 2^27-record ingest call of this workload, from the one-kernel ncu
+# captures of the 2^25-record case summarised under profiles/ (traffic grows in proportion to the
+# records of a launch, so refresh this constant from the small case, never from a full-size capture):
+# scatter_kernel 4 x 1.1426 GB per 2^27-record launch, plus the two drains inside a step's eight calls
+# (557 M spilled entries x 16 B read, and per drain 1.2 GB of table reads and write-backs) spread over
+# the eight calls.
+NCU_DRAM_BYTES_PER_INGEST_CALL = 4 * 1.1426e9 + (557e6 * 16 + 2 * 1.2e9) / 8
 UNIT = "records/s"
 WORKLOAD_INDEX = 3
 RECORD_BYTES = 16
@@ -336,8 +339,10 @@ def per_config(torch, p, records3, n3, peak):
     from tracegen.configs import make_spec
     from tracegen.gpu import GpuSampler
     rows = []
-    for index in range(5):
-        spec = make_spec(index)
+    # the five configurations, then the tiny configuration's law at 2^28 records: every one of its 4096
+    # keys sits in the shared-memory directory, which shows the rate of the path when nothing spills
+    for index, n_override in ((0, None), (1, None), (2, None), (3, None), (4, None), (0, 1 << 28)):
+        spec = make_spec(index) if n_override is None else make_spec(index, n=n_override)
         if index == WORKLOAD_INDEX:
             recs, n = records3, n3
         else:
@@ -361,13 +366,15 @@ def per_config(torch, p, records3, n3, peak):
                 best = ms
         st = agg.stats()
         gbs = chunk * spec.n_chunks * RECORD_BYTES / (best * 1e-3) / 1e9
-        rows.append({"config": index, "name": spec.name, "records": chunk * spec.n_chunks, "ingest_ms": best,
+        rows.append({"config": index, "name": spec.name if n_override is None else f"{spec.name} law, {n_override} records",
+                     "records": chunk * spec.n_chunks, "ingest_ms": best,
                      "records_per_s": chunk * spec.n_chunks / (best * 1e-3), "algorithmic_GBps": gbs,
                      "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / 8000.0,
                      "spill_fraction": st["n_spilled"] / max(st["n_valid"], 1), "live_keys": st["n_keys"],
-                     "drains_inside": max(int(st["n_drains"]) - 1, 0),
+                     "drains": int(st["n_drains"]),
                      "dram_bytes_per_record": NCU_DRAM_BYTES_PER_RECORD.get(index),
-                     "note": "16 MiB of records: L2-resident and launch-bound, not an HBM measurement" if index == 0 else None})
+                     "note": "16 MiB of records: L2-resident and launch-bound, not an HBM measurement"
+                             if index == 0 and n_override is None else None})
         del agg
         if index != WORKLOAD_INDEX:
             del recs

@@ -8,7 +8,7 @@
  *          invocations; here kept per (operator, shape, phase) key and scaled by the
  *          application's card-hour weight (Eq. 3's p_a) as an exact 128-bit integer;
  *   Eq. 3  normalisation so that weights sum to 1, taken separately for each serving
- *          phase (Sec. 3.1 "computed separately for the serving phases");
+ *          phase (Sec. 3.1: each serving phase gets its own set of weights);
  *   Eq. 1  roofline time max(F / P_dtype, M / beta) per (operator, shape) unit;
  *   Table 2  ranking of units by weight (deterministic top-k).
  *
