@@ -45,5 +45,19 @@ def build_checked(force: bool = False) -> str:
     return DEBUG_LIB
 
 
+def build_variant(name: str, flags) -> str:
+    """The library with extra nvcc flags, as libatrex_agg_<name>.so beside the regular one -- e.g. the
+    scatter pass's build-time variants (-DATREX_SCATTER_RING=4, -DATREX_SCATTER_PAIR=1).  Select it with
+    ATREX_AGG_LIBRARY=<path>."""
+    out = os.path.join(_HERE, f"libatrex_agg_{name}.so")
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    subprocess.check_call([nvcc] + NVCC_FLAGS + list(flags) + ["-o", out] + [os.path.join(CSRC, s) for s in SOURCES])
+    return out
+
+
 if __name__ == "__main__":
-    print(build(force=True, verbose=True))
+    import sys
+    if len(sys.argv) >= 3 and sys.argv[1] == "--variant":      # build.py --variant NAME [nvcc flags...]
+        print(build_variant(sys.argv[2], sys.argv[3:]))
+    else:
+        print(build(force=True, verbose=True))
