@@ -81,12 +81,32 @@ int atrex_entries_bucket_by_owner(const atrex_entry_t* d_entries, uint64_t n, ui
     if (!d_entries || !d_out || ((uintptr_t)d_entries & 15u) || ((uintptr_t)d_out & 15u) || ((uintptr_t)d_scratch & 7u))
         return ATREX_ERR_INVALID;
     if (n > (1ull << 32)) return ATREX_ERR_TOO_LARGE;
+    // the entries live on some device: run there
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, d_entries) != cudaSuccess || attr.type != cudaMemoryTypeDevice) {
+        cudaGetLastError();
+        return ATREX_ERR_INVALID;
+    }
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+    if (prev != attr.device && cudaSetDevice(attr.device) != cudaSuccess) {
+        cudaGetLastError();
+        return ATREX_ERR_CUDA;
+    }
+    struct Restore {
+        int dev;
+        ~Restore() {
+            if (dev >= 0) cudaSetDevice(dev);
+        }
+    } restore{prev != attr.device ? prev : -1};
+    int n_sms = 148;
+    if (cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, attr.device) != cudaSuccess || n_sms <= 0) n_sms = 148;
     cudaStream_t s = (cudaStream_t)stream;
     ull* counts = (ull*)d_scratch;
     ull* cursors = counts + world;
     const ull tile = (ull)BUCKET_THREADS * BUCKET_PER_THREAD;
     int grid = (int)((n + tile - 1) / tile);
-    if (grid > 148 * 8) grid = 148 * 8;
+    if (grid > n_sms * 8) grid = n_sms * 8;
     const size_t smem = (size_t)world * 16;
     if (cudaMemsetAsync(counts, 0, (size_t)world * 8, s) != cudaSuccess) return ATREX_ERR_CUDA;
     bucket_kernel<<<grid, BUCKET_THREADS, smem, s>>>(d_entries, n, world, d_out, counts, cursors, 1);
