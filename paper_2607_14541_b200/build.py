@@ -45,6 +45,32 @@ def build_checked(force: bool = False) -> str:
     return DEBUG_LIB
 
 
+# the scatter pass's build-time variants that the test-suite runs the parity cases under
+VARIANTS = {"ring4": ["-DATREX_SCATTER_RING=4"], "pair": ["-DATREX_SCATTER_PAIR=1"]}
+
+
+def variant_path(name: str) -> str:
+    return os.path.join(_HERE, f"libatrex_agg_{name}.so")
+
+
+def build_variant_if_stale(name: str, flags) -> str:
+    srcs = [os.path.join(CSRC, s) for s in SOURCES]
+    deps = srcs + [os.path.normpath(os.path.join(CSRC, h)) for h in HEADERS]
+    if _stale(variant_path(name), deps):
+        build_variant(name, flags)
+    return variant_path(name)
+
+
+def build_all(force: bool = True) -> None:
+    """The regular library, the bounds-checked one and the tested variants, compiled side by side."""
+    from concurrent.futures import ThreadPoolExecutor
+    jobs = [lambda: build(force=force), lambda: build_checked(force=force)]
+    jobs += [(lambda n=n, f=f: build_variant(n, f) if force else build_variant_if_stale(n, f)) for n, f in VARIANTS.items()]
+    with ThreadPoolExecutor(max_workers=len(jobs)) as pool:
+        for fut in [pool.submit(j) for j in jobs]:
+            fut.result()
+
+
 def build_variant(name: str, flags) -> str:
     """The library with extra nvcc flags, as libatrex_agg_<name>.so beside the regular one -- e.g. the
     scatter pass's build-time variants (-DATREX_SCATTER_RING=4, -DATREX_SCATTER_PAIR=1).  Select it with

@@ -241,6 +241,140 @@ __device__ __forceinline__ void part_accumulate(const PartSmem& m, uint32_t slot
     }
 }
 
+// One batch of 128 entries of a sub-buffer, four per lane.  FULL: the batch is complete (no masks).
+// Entry state is two bit sets per lane -- `open` (present, slot not known yet) and `hit` (slot known).
+template <bool FULL>
+__device__ __forceinline__ void stream_batch(const PartitionParams& q, const PartSmem& m, const ulonglong2* src, uint32_t e0,
+                                             uint32_t n_e, uint32_t C, ull base, ulonglong2* my_queue, uint32_t queue_cap_w,
+                                             uint32_t& qn_w, unsigned char* s_owner_w, uint32_t lane) {
+    ull key[4], v[4];
+    uint32_t slot[4];
+    uint32_t open = 0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const uint32_t e = e0 + u * 32 + lane;
+        if (FULL || e < n_e) {
+            const ulonglong2 ent = __ldcs(src + e);
+            key[u] = ent.x;
+            v[u] = ent.y;
+            open |= 1u << u;
+        } else {
+            key[u] = 0;
+            v[u] = 0;
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) slot[u] = local_of(hash32(key[u]), (uint32_t)(key[u] >> 48), C) & ~1u;  // first pair of the probe sequence
+    // First look, straight-line for all four entries: most keys sit in the first pair of slots of
+    // their probe sequence.
+    uint32_t hit = 0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const ulonglong2 kk = lds_v2u64(m.keys + ATREX_INDEX(slot[u], C - 1u, q.t.ctl) * 8);
+        const ull skey = ~key[u];
+        const bool h1 = kk.y == skey;
+        if (h1) slot[u] |= 1u;
+        if (kk.x == skey || h1) hit |= 1u << u;
+    }
+    hit &= open;     // (an absent entry reads as key 0, which may exist)
+    open &= ~hit;
+    if (__any_sync(0xFFFFFFFFu, open != 0)) {
+        // A new key whose first pair has room is inserted at once, so that its later occurrences find
+        // it there; losing the slot to another key defers the entry.
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (open & (1u << u)) {
+                const ulonglong2 kk = lds_v2u64(m.keys + slot[u] * 8);
+                const ull skey = ~key[u];
+                if (kk.x == skey || kk.y == skey) {            // it appeared meanwhile
+                    slot[u] += kk.x == skey ? 0u : 1u;
+                    hit |= 1u << u;
+                    open &= ~(1u << u);
+                } else if (kk.x == 0 || kk.y == 0) {
+                    const uint32_t at = slot[u] + (kk.x == 0 ? 0u : 1u);
+                    const ull old = atoms_cas64(m.keys + at * 8, 0ull, skey);
+                    if (old == 0) reds_or(m.cnt + at * 4, NEW_KEY_FLAG);
+                    if (old == 0 || old == skey) {
+                        slot[u] = at;
+                        hit |= 1u << u;
+                        open &= ~(1u << u);
+                    }
+                }
+            }
+        }
+        // The rest (collisions, keys further down their probe sequence: a few per batch) is not settled
+        // here, where the fixed cost of a general probe round would be paid for a handful of entries: it
+        // goes to this warp's queue and is settled after the partition's stream, 32 entries per warp round.
+        uint32_t pend[4], before[4], total = 0;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            pend[u] = __ballot_sync(0xFFFFFFFFu, (open >> u) & 1u);
+            before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
+            total += __popc(pend[u]);
+        }
+        if (total != 0) {
+            uint32_t qbase = qn_w;
+            qn_w = min(qn_w + total, queue_cap_w);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if ((open & (1u << u)) && qbase + before[u] < queue_cap_w) {
+                    my_queue[ATREX_INDEX(qbase + before[u], queue_cap_w, q.t.ctl)] = make_ulonglong2(key[u], v[u]);
+                    open &= ~(1u << u);
+                }
+            }
+            // Queue full (a partition made of new keys only): settle the remainder in line.  The pending
+            // entries are handed out one per lane: each one's owner publishes (round, lane) at the entry's
+            // position; lane t serves position t.
+            while (qbase + total > queue_cap_w) {
+                total = 0;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    pend[u] = __ballot_sync(0xFFFFFFFFu, (open >> u) & 1u);
+                    before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
+                    total += __popc(pend[u]);
+                }
+                if (total == 0) break;
+                qbase = queue_cap_w;  // stay in this loop until nothing is pending
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if ((open & (1u << u)) && before[u] < 32) s_owner_w[before[u]] = (unsigned char)((u << 5) | lane);
+                __syncwarp();
+                const bool serving = lane < total;
+                const uint32_t code = serving ? s_owner_w[lane] : lane;
+                const uint32_t from = code & 31u, su = code >> 5;
+                ull key_s = 0;
+                uint32_t slot_s = 0;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const ull k = __shfl_sync(0xFFFFFFFFu, key[u], from);
+                    const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u] & ~1u, from);
+                    if (su == (uint32_t)u) {
+                        key_s = k;
+                        slot_s = sl;
+                    }
+                }
+                const uint32_t found_s = probe_general(m, ~key_s, slot_s, 2u * stride_of(q.t, stride_index(hash32(key_s))), serving, C,
+                                                       q.t.ctl);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t found = __shfl_sync(0xFFFFFFFFu, found_s, before[u] & 31u);
+                    if ((open & (1u << u)) && before[u] < 32) {
+                        open &= ~(1u << u);
+                        if (found != PROBE_FAILED) {
+                            slot[u] = found;
+                            hit |= 1u << u;
+                        }
+                    }
+                }
+                __syncwarp();  // the owner table is rewritten in the next round
+            }
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+        if (hit & (1u << u)) part_accumulate(m, slot[u], v[u], q.t.vals + base, C, q.t.ctl);
+}
+
 __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionParams q) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t C = q.t.C;
@@ -331,110 +465,10 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
             for (uint32_t e0 = 0; e0 < n_e; e0 += 128) {
                 if (lane < 16 && (e0 + 256u + lane * 8u) < n_e)
                     prefetch_l2(reinterpret_cast<const unsigned char*>(src) + (e0 + 256u) * 16u + lane * 128u);
-                ull skey[4], v[4];
-                uint32_t slot[4], strides = 0;  // strides: each entry's stride index, one byte each
-                bool searching[4], ok[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    uint32_t e = e0 + u * 32 + lane;
-                    ok[u] = e < n_e;
-                    ulonglong2 ent = ok[u] ? __ldcs(src + e) : make_ulonglong2(0, 0);
-                    skey[u] = ~ent.x;
-                    v[u] = ent.y;
-                    const uint32_t hh = hash32(ent.x);
-                    slot[u] = local_of(hh, (uint32_t)(ent.x >> 48), C) & ~1u;  // first pair of the probe sequence
-                    strides |= stride_index(hh) << (8 * u);
-                    searching[u] = ok[u];
-                }
-                // First look, straight-line for all four entries: most keys sit in the first pair
-                // of slots of their probe sequence, and most new keys find room there.
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const ulonglong2 kk = lds_v2u64(m.keys + ATREX_INDEX(slot[u], C - 1u, q.t.ctl) * 8);
-                    const bool hit1 = kk.y == skey[u];
-                    if (hit1) slot[u] += 1;
-                    if (kk.x == skey[u] || hit1) {
-                        searching[u] = false;
-                    } else if (searching[u] && (kk.x == 0 || kk.y == 0)) {
-                        // a new key whose first pair has room is inserted at once, so that its later
-                        // occurrences find it here; losing the slot to another key defers the entry
-                        const uint32_t at = slot[u] + (kk.x == 0 ? 0u : 1u);
-                        const ull old = atoms_cas64(m.keys + at * 8, 0ull, skey[u]);
-                        if (old == 0) reds_or(m.cnt + at * 4, NEW_KEY_FLAG);
-                        if (old == 0 || old == skey[u]) {
-                            slot[u] = at;
-                            searching[u] = false;
-                        }
-                    }
-                }
-                // The rest (new keys, collisions: a few per batch) is not settled here, where the fixed
-                // cost of a general probe round would be paid for a handful of entries: it goes to this
-                // CTA's queue and is settled after the partition's stream, 32 entries per warp round.
-                uint32_t pend[4], before[4], total = 0;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    pend[u] = __ballot_sync(0xFFFFFFFFu, searching[u]);
-                    before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
-                    total += __popc(pend[u]);
-                }
-                if (total != 0) {
-                    uint32_t qbase = qn_w;
-                    qn_w = min(qn_w + total, queue_cap_w);
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if (searching[u] && qbase + before[u] < queue_cap_w) {
-                            my_queue[ATREX_INDEX(qbase + before[u], queue_cap_w, q.t.ctl)] = make_ulonglong2(~skey[u], v[u]);
-                            searching[u] = false;
-                            ok[u] = false;
-                        }
-                    }
-                    // Queue full (a partition made of new keys only): settle the remainder in line.
-                    // The pending entries are handed out one per lane: each one's owner publishes
-                    // (round, lane) at the entry's position; lane t serves position t.
-                    while (qbase + total > queue_cap_w) {
-                        total = 0;
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            pend[u] = __ballot_sync(0xFFFFFFFFu, searching[u]);
-                            before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
-                            total += __popc(pend[u]);
-                        }
-                        if (total == 0) break;
-                        qbase = queue_cap_w;  // stay in this loop until nothing is pending
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            if (searching[u] && before[u] < 32) s_owner[warp][before[u]] = (unsigned char)((u << 5) | lane);
-                        __syncwarp();
-                        const bool serving = lane < total;
-                        const uint32_t code = serving ? s_owner[warp][lane] : lane;
-                        const uint32_t from = code & 31u, su = code >> 5;
-                        ull key_s = 0;
-                        uint32_t slot_s = 0;
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const ull k = __shfl_sync(0xFFFFFFFFu, skey[u], from);
-                            const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u] | (((strides >> (8 * u)) & 7u) << 16), from);
-                            if (su == (uint32_t)u) {
-                                key_s = k;
-                                slot_s = sl;
-                            }
-                        }
-                        const uint32_t found_s = probe_general(m, key_s, slot_s & 0xFFFFu, 2u * stride_of(q.t, slot_s >> 16),
-                                                               serving, C, q.t.ctl);
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const uint32_t found = __shfl_sync(0xFFFFFFFFu, found_s, before[u] & 31u);
-                            if (searching[u] && before[u] < 32) {
-                                searching[u] = false;
-                                if (found == PROBE_FAILED) ok[u] = false; else slot[u] = found;
-                            }
-                        }
-                        __syncwarp();  // the owner table is rewritten in the next round
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (ok[u]) part_accumulate(m, slot[u], v[u], q.t.vals + base, C, q.t.ctl);
+                if (e0 + 128u <= n_e)
+                    stream_batch<true>(q, m, src, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
+                else
+                    stream_batch<false>(q, m, src, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
             }
         }
         {   // this warp's queued entries, one per lane (other warps may still be streaming: the general

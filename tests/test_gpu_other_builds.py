@@ -30,6 +30,25 @@ def test_parity_cases_under_the_bounds_checked_build():
     assert " passed" in run.stdout
 
 
+@pytest.mark.parametrize("variant", ["ring4", "pair"])
+def test_parity_cases_under_the_scatter_variants(variant):
+    """The scatter pass's build-time variants -- the shared-memory record ring filled by bulk asynchronous
+    copies, and spill entries leaving as whole sectors through the pairing mailboxes -- are slower than
+    the default and therefore not what ships, but they are kept buildable and exact: the same parity
+    cases, bit for bit against the oracle."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("atrex_build", os.path.join(ROOT, "paper_2607_14541_b200", "build.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    lib = mod.build_variant_if_stale(variant, mod.VARIANTS[variant])
+    env = dict(os.environ, ATREX_AGG_LIBRARY=lib)
+    run = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "-x", "-q", "-k",
+                          "five_configs or misaligned or carry or invalid_records or full_u32 or many_small_calls"],
+                         cwd=ROOT, env=env, capture_output=True, text=True, timeout=1200)
+    assert run.returncode == 0, run.stdout[-3000:] + run.stderr[-2000:]
+    assert " passed" in run.stdout
+
+
 def test_the_regular_build_has_no_checks():
     import paper_2607_14541_b200 as p
     assert p.atrex_build_has_bounds_checks() == 0 or os.environ.get("ATREX_AGG_LIBRARY")
