@@ -3,7 +3,8 @@
 // operators ordered by weight, a "Cum." column beside them).
 //
 // Both are built on one primitive, a stable least-significant-digit radix sort of
-// (64-bit word, 32-bit entry index) pairs with 8-bit digits.  The ranking order
+// (64-bit word, 32-bit entry index) pairs with 8-bit digits (tiles reordered in shared memory, so
+// that every pass writes contiguous runs).  The ranking order
 // (weighted time descending, key ascending) is a 3-word composite; since the sort is stable it
 // is produced word by word, least significant first: key, then ~wt_lo, then ~wt_hi, each word
 // gathered through the current permutation.  A digit on which all words agree (the bitwise OR
@@ -12,6 +13,8 @@
 //
 // The running sum is an exact 128-bit prefix sum in rank order (block sums, a scan of the block
 // sums, a block-local scan), rounded once per row when the share is formed.
+#include <mutex>
+
 #include "kernels.h"
 
 using namespace atrex;
@@ -190,18 +193,30 @@ __global__ void __launch_bounds__(SCAN_BLOCK) radix_scan_kernel(uint32_t* hist, 
 
 // Stable: item order inside a tile is (warp, round, lane) = input order; a lane's rank among
 // equal digits is (items of earlier warps) + (earlier rounds of its warp) + (lower lanes of its
-// round), and tiles are ordered by the scanned (digit, tile) counters.
+// round), and tiles are ordered by the scanned (digit, tile) counters.  The tile is first put in
+// digit order in shared memory and then written out run by run, so that the global stores are
+// contiguous per digit (about 32 items per digit and tile) instead of one scattered 12-byte piece
+// per item.
+constexpr size_t SCATTER_SMEM = (size_t)SORT_TILE * 12;   // words (8 B) and indices (4 B) of one tile
+
 __global__ void __launch_bounds__(SORT_WARPS * 32) radix_scatter_kernel(const ull* words_in, const uint32_t* idx_in,
                                                                         ull* words_out, uint32_t* idx_out, uint32_t m,
                                                                         int shift, const uint32_t* hist,
                                                                         uint32_t n_tiles, const uint32_t* bin_total) {
+    extern __shared__ __align__(16) unsigned char sort_smem[];
+    ull* s_words = reinterpret_cast<ull*>(sort_smem);                          // [SORT_TILE] the tile in digit order
+    uint32_t* s_idx = reinterpret_cast<uint32_t*>(sort_smem + (size_t)SORT_TILE * 8);
     __shared__ uint32_t wh[SORT_WARPS][256];
-    __shared__ uint32_t bin_base[256];  // exclusive scan of the digit totals
+    __shared__ uint32_t bin_base[256];   // exclusive scan of the digit totals (global)
     __shared__ uint32_t bin_warp[8];
+    __shared__ uint32_t tile_base[256];  // first position of digit d inside this tile's digit order
+    __shared__ uint32_t tile_warp[8];
+    __shared__ uint32_t out_base[256];   // global position of this tile's first item of digit d
     for (uint32_t j = threadIdx.x; j < SORT_WARPS * 256; j += SORT_WARPS * 32) (&wh[0][0])[j] = 0;
     __syncthreads();
     const uint32_t w = threadIdx.x >> 5, lane = threadIdx.x & 31, lt = (1u << lane) - 1u;
-    const uint32_t first = blockIdx.x * SORT_TILE + w * (SORT_ROUNDS * 32) + lane;
+    const uint32_t tile_start = blockIdx.x * SORT_TILE;
+    const uint32_t first = tile_start + w * (SORT_ROUNDS * 32) + lane;
     uint32_t packed[SORT_ROUNDS];  // digit | rank inside the warp << 9
 #pragma unroll
     for (int r = 0; r < SORT_ROUNDS; ++r) {
@@ -215,37 +230,62 @@ __global__ void __launch_bounds__(SORT_WARPS * 32) radix_scatter_kernel(const ul
         __syncwarp();
         packed[r] = d | ((base + __popc(same & lt)) << 9);
     }
-    if (threadIdx.x < 256) {
-        const uint32_t c = bin_total[threadIdx.x];
-        uint32_t incl = c;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t o = __shfl_up_sync(FULL, incl, d);
-            if (lane >= (uint32_t)d) incl += o;
-        }
-        if (lane == 31) bin_warp[w] = incl;
-        bin_base[threadIdx.x] = incl - c;
-    }
     __syncthreads();
+    uint32_t tile_count = 0;
     if (threadIdx.x < 256) {
-        uint32_t run = bin_base[threadIdx.x] + hist[(size_t)threadIdx.x * n_tiles + blockIdx.x];
-        for (uint32_t k = 0; k < w; ++k) run += bin_warp[k];
+        // this digit's items in the tile, per warp -> running offsets; the digit totals -> global bases
 #pragma unroll
         for (int k = 0; k < SORT_WARPS; ++k) {
             const uint32_t c = wh[k][threadIdx.x];
-            wh[k][threadIdx.x] = run;
-            run += c;
+            wh[k][threadIdx.x] = tile_count;     // items of this digit in earlier warps
+            tile_count += c;
         }
+        const uint32_t c = bin_total[threadIdx.x];
+        uint32_t incl = c, tincl = tile_count;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t o = __shfl_up_sync(FULL, incl, d), to = __shfl_up_sync(FULL, tincl, d);
+            if (lane >= (uint32_t)d) {
+                incl += o;
+                tincl += to;
+            }
+        }
+        if (lane == 31) {
+            bin_warp[w] = incl;
+            tile_warp[w] = tincl;
+        }
+        bin_base[threadIdx.x] = incl - c;
+        tile_base[threadIdx.x] = tincl - tile_count;
+    }
+    __syncthreads();
+    if (threadIdx.x < 256) {
+        uint32_t g = bin_base[threadIdx.x] + hist[(size_t)threadIdx.x * n_tiles + blockIdx.x], t = tile_base[threadIdx.x];
+        for (uint32_t k = 0; k < w; ++k) {
+            g += bin_warp[k];
+            t += tile_warp[k];
+        }
+        out_base[threadIdx.x] = g;
+        tile_base[threadIdx.x] = t;
     }
     __syncthreads();
 #pragma unroll
     for (int r = 0; r < SORT_ROUNDS; ++r) {
         const uint32_t i = first + r * 32;
         if (i < m) {
-            const uint32_t pos = wh[w][packed[r] & 511u] + (packed[r] >> 9);
-            words_out[pos] = words_in[i];
-            idx_out[pos] = idx_in[i];
+            const uint32_t d = packed[r] & 511u;
+            const uint32_t at = tile_base[d] + wh[w][d] + (packed[r] >> 9);
+            s_words[at] = words_in[i];
+            s_idx[at] = idx_in[i];
         }
+    }
+    __syncthreads();
+    const uint32_t tile_n = min(SORT_TILE, m - tile_start);
+    for (uint32_t j = threadIdx.x; j < tile_n; j += SORT_WARPS * 32) {
+        const ull word = s_words[j];
+        const uint32_t d = (uint32_t)(word >> shift) & 255u;
+        const uint32_t pos = out_base[d] + (j - tile_base[d]);
+        words_out[pos] = word;
+        idx_out[pos] = s_idx[j];
     }
 }
 
@@ -425,13 +465,32 @@ int reset_or_and(const Scratch& sc, cudaStream_t s) {
 
 // Sorts the m pairs in buffer `cur` by the digits of the word on which the words differ.
 // Returns the buffer that holds the result, or a negative status.
+// The scatter kernel keeps a whole tile in shared memory: raise its dynamic shared-memory limit once per
+// device (the caller has made the entries' device current).
+int prepare_sort_kernels() {
+    static std::mutex lock;
+    static bool prepared[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ATREX_ERR_CUDA;
+    std::lock_guard<std::mutex> hold(lock);
+    if (!prepared[dev]) {
+        if (cudaFuncSetAttribute(radix_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SCATTER_SMEM) != cudaSuccess) {
+            cudaGetLastError();
+            return ATREX_ERR_CUDA;
+        }
+        prepared[dev] = true;
+    }
+    return ATREX_OK;
+}
+
 int sort_by_word(const Scratch& sc, int cur, uint32_t m, ull differing_bits, cudaStream_t s) {
     const uint32_t tiles = (m + SORT_TILE - 1) / SORT_TILE;
+    if (prepare_sort_kernels() != ATREX_OK) return ATREX_ERR_CUDA;
     for (int shift = 0; shift < 64; shift += 8) {
         if (((differing_bits >> shift) & 255u) == 0) continue;
         radix_hist_kernel<<<tiles, SORT_WARPS * 32, 0, s>>>(sc.words[cur], m, shift, sc.hist, tiles);
         radix_scan_kernel<<<256, SCAN_BLOCK, 0, s>>>(sc.hist, tiles, sc.bin_total);
-        radix_scatter_kernel<<<tiles, SORT_WARPS * 32, 0, s>>>(sc.words[cur], sc.idx[cur], sc.words[cur ^ 1],
+        radix_scatter_kernel<<<tiles, SORT_WARPS * 32, SCATTER_SMEM, s>>>(sc.words[cur], sc.idx[cur], sc.words[cur ^ 1],
                                                                 sc.idx[cur ^ 1], m, shift, sc.hist, tiles,
                                                                 sc.bin_total);
         if (cudaGetLastError() != cudaSuccess) return ATREX_ERR_CUDA;
