@@ -1,21 +1,21 @@
 // Pass 1 of the ingest (Eq. 2's group-by sum, streamed): SCATTER, one persistent CTA per SM.
 //
-// Each thread pulls records with 32-byte vector loads (two 16-byte records per load, two loads per thread
-// alternating so that one is in flight while the other is consumed, streaming cache policy), validates, packs the key and
-// multiplies the application's card-hour weight by the duration.
+// Each thread pulls records with 32-byte vector loads (two 16-byte records per load, three loads
+// rotating per thread so that two are in flight while one is consumed, streaming cache policy),
+// validates, packs the key and multiplies the application's card-hour weight by the duration.
 //   * Keys found in the shared-memory HOT DIRECTORY (the most frequent keys of a sample of the
 //     trace, identical in every CTA, read-only during the pass) are accumulated on the spot with
 //     32-bit shared-memory atomics in limbs with explicit carries.
 //   * Every other record becomes a 16-byte {key, product} entry appended to the CTA's private
-//     buffer of the key's partition; entries leave in pairs, as whole 32-byte sectors (see
-//     spill_append).
+//     buffer of the key's partition (see spill_append: stored on its own with the next line of the
+//     buffer prefetched into L2, or -- build-time variant -- paired into whole 32-byte sectors).
 // At the end the CTA adds its directory accumulators to its own row of a directory image
 // ([CTA][slot], plain coalesced read-modify-writes; hot_fold_kernel adds the rows into the table
 // before results are read) and stores its per-partition cursors: the buffers persist across launches
 // until the partition pass drains them.
 //
-// The kernel is bound by instruction issue and by the shared-memory pipe, not by DRAM, so the hot
-// loop is written for a low instruction count: the shared-memory layout is a compile-time function
+// The kernel runs out of issue slots, shared-memory pipe cycles and latency-hiding warps long before
+// it runs out of DRAM bandwidth, so the hot loop is written for a low instruction count: the shared-memory layout is a compile-time function
 // of the partition count (every array address is a register plus an immediate), rarely taken
 // branches (products of 2^48 and more, a full buffer, a wait for another lane's turn, a drain of a
 // directory slot) are calls to functions that are not inlined, and the three load buffers rotate by
@@ -400,8 +400,8 @@ __device__ __forceinline__ void process(const IngestParams& p, Ctx& c, const uin
 
 template <uint32_t LP, bool HOT, bool DEDUPE, bool PAIR>
 __device__ __forceinline__ void scatter_body(const IngestParams& p, Ctx& c) {
-    // CTA b handles record pairs (b + k * gridDim) * 1024 + tid, k = 0, 1, ...  Two 32-byte loads
-    // alternate per thread: while one is consumed the next is in flight.  Rounds in which every
+    // CTA b handles record pairs (b + k * gridDim) * 1024 + tid, k = 0, 1, ...  Three 32-byte loads
+    // rotate per thread: while one is consumed the next two are in flight.  Rounds in which every
     // CTA's tile is complete need no bounds checks; the last (ragged) ones are predicated.
     const unsigned char* body = reinterpret_cast<const unsigned char*>(p.body);
     const uint32_t stride = gridDim.x * SCATTER_THREADS;                  // pairs per round
