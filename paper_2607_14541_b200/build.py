@@ -45,8 +45,8 @@ def build_checked(force: bool = False) -> str:
     return DEBUG_LIB
 
 
-# the scatter pass's build-time variants that the test-suite runs the parity cases under
-VARIANTS = {"ring4": ["-DATREX_SCATTER_RING=4"], "pair": ["-DATREX_SCATTER_PAIR=1"]}
+# the scatter pass's build-time variant that the test-suite runs the parity cases under
+VARIANTS = {"ring4": ["-DATREX_SCATTER_RING=4"]}
 
 
 def variant_path(name: str) -> str:
@@ -73,7 +73,7 @@ def build_all(force: bool = True) -> None:
 
 def build_variant(name: str, flags) -> str:
     """The library with extra nvcc flags, as libatrex_agg_<name>.so beside the regular one -- e.g. the
-    scatter pass's build-time variants (-DATREX_SCATTER_RING=4, -DATREX_SCATTER_PAIR=1).  Select it with
+    scatter pass's build-time variant (-DATREX_SCATTER_RING=4).  Select it with
     ATREX_AGG_LIBRARY=<path>."""
     out = os.path.join(_HERE, f"libatrex_agg_{name}.so")
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")

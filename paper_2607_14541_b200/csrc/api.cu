@@ -81,7 +81,7 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     ull per_buf = (L->sub_launch * 9 / 2) / (((ull)n_sms) << L->lp);
     if (per_buf < 64) per_buf = 64;
     if (per_buf > 32768) per_buf = 32768;   // the scatter pass counts a buffer's entries in 16 bits, with headroom
-    L->cap = (uint32_t)((per_buf + 7) / 8 * 8);
+    L->cap = (uint32_t)((per_buf + 31) / 32 * 32);   // a buffer is a whole number of 128-byte lines
     // entries of one partition whose first look fails wait in a per-CTA queue: room for a quarter of
     // the partition's worst-case stream, at most 32 K entries (the rest is settled in line)
     {
@@ -110,7 +110,7 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     L->off_hot_scratch = o;    o += round_up(HOT_SCRATCH_BYTES, ALIGN);
     L->off_queue = o;          o += round_up((size_t)L->n_groups * L->queue_cap * 16, ALIGN);
     L->off_spill_cnt = o;      o += round_up(((size_t)L->n_groups << L->lp) * 4, ALIGN);
-    L->off_spill = o;          o += round_up(((size_t)L->n_groups << L->lp) * L->cap * 16, ALIGN) + ALIGN;  // + prefetch overrun
+    L->off_spill = o;          o += round_up(((size_t)L->n_groups << L->lp) * L->cap * SPILL_ENTRY_BYTES, ALIGN) + ALIGN;  // + prefetch overrun
     L->total = o;
 }
 

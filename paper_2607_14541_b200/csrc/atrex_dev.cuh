@@ -12,10 +12,10 @@
 //                 find_or_claim below).  C is chosen so that one partition's
 //                 keys and per-launch accumulators fit in one SM's shared memory: the
 //                 aggregation pass owns a partition per CTA and needs no global atomics.
-//   spill bufs  : [G][P][cap] 16-byte {key, weighted duration} entries and [G][P] counts,
+//   spill bufs  : [G][P][cap] 12-byte entries -- an 8-byte word {weighted duration, operator}
+//                 and a 4-byte word {phase, low hash bits} -- and [G][P] counts,
 //                 written by CTA g of the scatter pass (its buffers are contiguous, which keeps
-//                 the scattered 16-byte appends within a few pages), read by CTA p of the
-//                 partition pass
+//                 the scattered appends within a few pages), read by CTA p of the partition pass
 //   work table  : the same P partitions (by the same hash of op_id and shape_id) of Cw 32-byte
 //                 slots {~(op_id << 32 | shape_id), flops, bytes, dtype}, probed inside the partition
 //   control     : counters, per-phase totals, top-k histogram
@@ -82,12 +82,29 @@ struct Control {
 // more.  The top bits pick the partition, the bits below them the start slot inside it.  The
 // phase is deliberately left out: a key's partition is then also the partition of its
 // (operator, shape) row in the work table, which keeps the roofline pass's look-ups local.
+constexpr uint32_t HASH_A = 0x9E3779B1u, HASH_B = 0x85EBCA77u, HASH_C = 0x2C1B3C6Du;
 __device__ __forceinline__ uint32_t hash32(uint32_t op, uint32_t shape) {
-    uint32_t h = (shape * 0x9E3779B1u) ^ (op * 0x85EBCA77u);
+    uint32_t h = (shape * HASH_A) ^ (op * HASH_B);
     h ^= h >> 15;
-    h *= 0x2C1B3C6Du;
+    h *= HASH_C;
     h ^= h >> 13;
     return h;
+}
+// For a given operator the hash is a bijection of the shape (odd multipliers, xor-shifts), so inside a
+// partition the triple (phase, operator, hash) identifies a key as well as (phase, operator, shape) does.
+// The inverse: undo the xor-shifts, multiply by the multipliers' inverses modulo 2^32.
+constexpr uint32_t mod_inverse_u32(uint32_t a) {   // a odd; Newton's iteration doubles the correct bits
+    uint32_t x = a;
+    for (int i = 0; i < 5; ++i) x *= 2u - a * x;
+    return x;
+}
+constexpr uint32_t HASH_A_INV = mod_inverse_u32(HASH_A), HASH_C_INV = mod_inverse_u32(HASH_C);
+static_assert(HASH_A * HASH_A_INV == 1u && HASH_C * HASH_C_INV == 1u, "modular inverses");
+__host__ __device__ __forceinline__ uint32_t shape_of_hash(uint32_t h, uint32_t op) {
+    uint32_t x = h ^ (h >> 13) ^ (h >> 26);
+    x *= HASH_C_INV;
+    x = x ^ (x >> 15) ^ (x >> 30);
+    return (x ^ (op * HASH_B)) * HASH_A_INV;
 }
 __device__ __forceinline__ uint32_t hash32(ull key) { return hash32((uint32_t)(key >> 32) & 0xFFFFu, (uint32_t)key); }
 
@@ -101,6 +118,25 @@ __device__ __forceinline__ uint32_t dir_mix(uint32_t h, uint32_t phase, uint32_t
 }
 __device__ __forceinline__ uint32_t dir_bucket(uint32_t h, uint32_t phase, uint32_t mult, uint32_t n_buckets) {
     return __umulhi(dir_mix(h, phase, mult), n_buckets);
+}
+
+// The partition pass's own form of a key, unique inside a partition: bit 63 set (so that 0 can mean
+// an empty slot), phase << 16 | operator in bits 32..55, the 32-bit hash below.
+constexpr ull CKEY_MARK = 1ull << 63;
+__device__ __forceinline__ ull ckey_of(uint32_t khi24, uint32_t h) { return CKEY_MARK | ((ull)khi24 << 32) | h; }
+__device__ __forceinline__ ull ckey_of_key(ull key) { return ckey_of((uint32_t)(key >> 32) & 0x00FFFFFFu, hash32((uint32_t)(key >> 32) & 0xFFFFu, (uint32_t)key)); }
+__device__ __forceinline__ uint32_t ckey_phase(ull ckey) { return (uint32_t)(ckey >> 48) & 0xFFu; }
+__device__ __forceinline__ ull key_of_ckey(ull ckey) {
+    const uint32_t khi24 = (uint32_t)(ckey >> 32) & 0x00FFFFFFu;
+    return ((ull)khi24 << 32) | shape_of_hash((uint32_t)ckey, khi24 & 0xFFFFu);
+}
+// The two words of a spill entry (12 bytes): a = product (48 bits) | operator << 48,
+// b = phase << 24 | the hash bits below the partition's log2 P (at most 24: there are at least 2^8 partitions).
+constexpr uint32_t SPILL_ENTRY_BYTES = 12;
+__device__ __forceinline__ ull spill_word_a(ull prod, uint32_t op) { return prod | ((ull)op << 48); }
+__device__ __forceinline__ uint32_t spill_word_b(uint32_t phase, uint32_t h, uint32_t lp) { return (phase << 24) | (h & (0xFFFFFFFFu >> lp)); }
+__device__ __forceinline__ ull ckey_of_spill(ull a, uint32_t b, uint32_t part, uint32_t lp) {
+    return ckey_of(((b >> 24) << 16) | (uint32_t)(a >> 48), (part << (32 - lp)) | (b & (0xFFFFFFFFu >> lp)));
 }
 
 __device__ __forceinline__ ull pack_key(uint32_t phase, uint32_t op, uint32_t shape) {

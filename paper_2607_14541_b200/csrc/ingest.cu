@@ -26,7 +26,6 @@
 namespace atrex {
 
 constexpr int INGEST_THREADS = 1024;
-constexpr uint32_t NO_SLOT = 0xFFFFFFFFu;
 constexpr uint32_t DIR_WAYS = 4;                   // slots per hot-directory bucket (32 bytes of keys)
 constexpr uint32_t NEW_KEY_FLAG = 0x80000000u;     // partition pass: slot claimed in this launch
 
@@ -178,7 +177,8 @@ __global__ void __launch_bounds__(FOLD_WARPS * 32) hot_fold_kernel(const ull* ho
 // Pass 2: a CTA aggregates one partition at a time entirely in shared memory.  CTAs are
 // persistent and take partitions blockIdx.x, blockIdx.x + gridDim.x, ...; while one partition
 // is processed, the next one's keys and spill entries are pulled into L2.  Per partition: copy the
-// keys in; stream the entries of all scatter CTAs, four per lane, and settle each with one look at
+// keys in, each in the pass's own 64-bit form (phase, operator, 32-bit hash: unique inside a
+// partition, and what a spill entry carries); stream the entries of all scatter CTAs, four per lane, and settle each with one look at
 // the first pair of its probe sequence (hit, or a new key with room there); entries that need more
 // than that wait in the warp's segment of a per-CTA queue in global memory and are settled, 32 per
 // round, once the warp's share of the stream is through; then write the deltas back.
@@ -241,42 +241,59 @@ __device__ __forceinline__ void part_accumulate(const PartSmem& m, uint32_t slot
     }
 }
 
-// One batch of 128 entries of a sub-buffer, four per lane.  FULL: the batch is complete (no masks).
+// The first 256 entries (24 lines) of sub-buffer `sb` towards L2, as far as it holds that many.
+__device__ __forceinline__ void prefetch_entries(const PartitionParams& q, ull sb, uint32_t lane) {
+    const uint32_t bytes = q.spill_cnt[sb] * SPILL_ENTRY_BYTES;
+    if (lane < 24 && lane * 128u < bytes) prefetch_l2(q.spill + sb * q.cap * SPILL_ENTRY_BYTES + lane * 128u);
+}
+
+// One batch of 128 entries of a sub-buffer, four consecutive ones (48 bytes) per lane.  FULL: the
+// batch is complete (no masks).
 // Entry state is two bit sets per lane -- `open` (present, slot not known yet) and `hit` (slot known).
 template <bool FULL>
-__device__ __forceinline__ void stream_batch(const PartitionParams& q, const PartSmem& m, const ulonglong2* src, uint32_t e0,
-                                             uint32_t n_e, uint32_t C, ull base, ulonglong2* my_queue, uint32_t queue_cap_w,
-                                             uint32_t& qn_w, unsigned char* s_owner_w, uint32_t lane) {
-    ull key[4], v[4];
+__device__ __forceinline__ void stream_batch(const PartitionParams& q, const PartSmem& m, const unsigned char* src,
+                                             uint32_t part, uint32_t e0, uint32_t n_e, uint32_t C, ull base, ulonglong2* my_queue,
+                                             uint32_t queue_cap_w, uint32_t& qn_w, unsigned char* s_owner_w, uint32_t lane) {
+    ull key[4], v[4];   // key: the partition pass's form (ckey_of)
     uint32_t slot[4];
     uint32_t open = 0;
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-        const uint32_t e = e0 + u * 32 + lane;
+    {
+        // the lane's entries e, e + 1, e + 2, e + 3 (e a multiple of 4) as twelve words; in an even
+        // entry the 8-byte word comes first, in an odd one last.  A buffer's capacity is a multiple
+        // of 4, so a lane that holds any entry may read all 48 bytes.
+        const uint32_t e = e0 + 4u * lane;
+        uint4 w[3];
         if (FULL || e < n_e) {
-            const ulonglong2 ent = __ldcs(src + e);
-            key[u] = ent.x;
-            v[u] = ent.y;
-            open |= 1u << u;
+            const uint4* at = reinterpret_cast<const uint4*>(src + (size_t)e * SPILL_ENTRY_BYTES);
+#pragma unroll
+            for (int j = 0; j < 3; ++j) w[j] = __ldcs(at + j);
+            open = FULL ? 0xFu : (0xFu >> (4u - min(n_e - e, 4u)));
         } else {
-            key[u] = 0;
-            v[u] = 0;
+#pragma unroll
+            for (int j = 0; j < 3; ++j) w[j] = make_uint4(0, 0, 0, 0);
+        }
+        const ull a[4] = {w[0].x | ((ull)w[0].y << 32), w[1].x | ((ull)w[1].y << 32), w[1].z | ((ull)w[1].w << 32), w[2].z | ((ull)w[2].w << 32)};
+        const uint32_t b[4] = {w[0].z, w[0].w, w[2].x, w[2].y};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            key[u] = ckey_of_spill(a[u], b[u], part, q.t.lp);
+            v[u] = a[u] & 0x0000FFFFFFFFFFFFull;
         }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) slot[u] = local_of(hash32(key[u]), (uint32_t)(key[u] >> 48), C) & ~1u;  // first pair of the probe sequence
+    for (int u = 0; u < 4; ++u) slot[u] = local_of((uint32_t)key[u], ckey_phase(key[u]), C) & ~1u;  // first pair of the probe sequence
     // First look, straight-line for all four entries: most keys sit in the first pair of slots of
     // their probe sequence.
     uint32_t hit = 0;
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
         const ulonglong2 kk = lds_v2u64(m.keys + ATREX_INDEX(slot[u], C - 1u, q.t.ctl) * 8);
-        const ull skey = ~key[u];
+        const ull skey = key[u];
         const bool h1 = kk.y == skey;
         if (h1) slot[u] |= 1u;
         if (kk.x == skey || h1) hit |= 1u << u;
     }
-    hit &= open;     // (an absent entry reads as key 0, which may exist)
+    hit &= open;     // (an absent entry is a well-formed key too)
     open &= ~hit;
     if (__any_sync(0xFFFFFFFFu, open != 0)) {
         // A new key whose first pair has room is inserted at once, so that its later occurrences find
@@ -285,7 +302,7 @@ __device__ __forceinline__ void stream_batch(const PartitionParams& q, const Par
         for (int u = 0; u < 4; ++u) {
             if (open & (1u << u)) {
                 const ulonglong2 kk = lds_v2u64(m.keys + slot[u] * 8);
-                const ull skey = ~key[u];
+                const ull skey = key[u];
                 if (kk.x == skey || kk.y == skey) {            // it appeared meanwhile
                     slot[u] += kk.x == skey ? 0u : 1u;
                     hit |= 1u << u;
@@ -353,7 +370,7 @@ __device__ __forceinline__ void stream_batch(const PartitionParams& q, const Par
                         slot_s = sl;
                     }
                 }
-                const uint32_t found_s = probe_general(m, ~key_s, slot_s, 2u * stride_of(q.t, stride_index(hash32(key_s))), serving, C,
+                const uint32_t found_s = probe_general(m, key_s, slot_s, 2u * stride_of(q.t, stride_index((uint32_t)key_s)), serving, C,
                                                        q.t.ctl);
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -436,7 +453,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
             for (int u = 0; u < 4; ++u) {
                 const uint32_t i = i0 + u * blockDim.x;
                 if (i < C) {
-                    s_keys[i] = k[u];
+                    s_keys[i] = k[u] == 0 ? 0ull : ckey_of_key(~k[u]);   // the table stores complemented keys, 0 = empty
                     s_a0[i] = 0;
                     s_a1[i] = 0;
                     s_cnt[i] = 0;
@@ -453,22 +470,18 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
         for (uint32_t g = warp; g < q.n_used; g += n_warps) {
             const ull sb = ((ull)g << q.t.lp) + part;
             const uint32_t n_e = q.spill_cnt[sb];
-            const ulonglong2* src = reinterpret_cast<const ulonglong2*>(q.spill) + sb * q.cap;
-            // Short-distance L2 prefetch, a fixed 4 KB window per warp (a longer reach gets evicted
-            // before use: all warps of all CTAs together must stay well inside L2): the head of this
-            // warp's next sub-buffer now, and inside the loop the lines two batches ahead.
-            if (g + n_warps < q.n_used) {
-                const ull nb = ((ull)(g + n_warps) << q.t.lp) + part;
-                const uint32_t bytes = q.spill_cnt[nb] * 16u;
-                if (lane * 128u < bytes) prefetch_l2(q.spill + nb * q.cap * 16ull + lane * 128u);
-            }
+            const unsigned char* buf = q.spill + sb * q.cap * SPILL_ENTRY_BYTES;
+            // Short-distance L2 prefetch, a fixed window of 256 entries per warp (a longer reach gets
+            // evicted before use: all warps of all CTAs together must stay well inside L2): the head of
+            // this warp's next sub-buffer now, and inside the loop the lines two batches ahead.
+            if (g + n_warps < q.n_used) prefetch_entries(q, ((ull)(g + n_warps) << q.t.lp) + part, lane);
             for (uint32_t e0 = 0; e0 < n_e; e0 += 128) {
-                if (lane < 16 && (e0 + 256u + lane * 8u) < n_e)
-                    prefetch_l2(reinterpret_cast<const unsigned char*>(src) + (e0 + 256u) * 16u + lane * 128u);
+                if (lane < 12 && (e0 + 256u) * SPILL_ENTRY_BYTES + lane * 128u < n_e * SPILL_ENTRY_BYTES)
+                    prefetch_l2(buf + (e0 + 256u) * SPILL_ENTRY_BYTES + lane * 128u);
                 if (e0 + 128u <= n_e)
-                    stream_batch<true>(q, m, src, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
+                    stream_batch<true>(q, m, buf, part, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
                 else
-                    stream_batch<false>(q, m, src, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
+                    stream_batch<false>(q, m, buf, part, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
             }
         }
         {   // this warp's queued entries, one per lane (other warps may still be streaming: the general
@@ -477,9 +490,9 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
             for (uint32_t i0 = 0; i0 < qn_w; i0 += 32u) {
                 const bool serving = i0 + lane < qn_w;
                 const ulonglong2 ent = serving ? __ldcg(my_queue + i0 + lane) : make_ulonglong2(0, 0);
-                const uint32_t hh = hash32(ent.x);
-                const uint32_t start = local_of(hh, (uint32_t)(ent.x >> 48), C) & ~1u;
-                const uint32_t found = probe_general(m, ~ent.x, start, 2u * stride_of(q.t, stride_index(hh)), serving, C, q.t.ctl);
+                const uint32_t hh = (uint32_t)ent.x;
+                const uint32_t start = local_of(hh, ckey_phase(ent.x), C) & ~1u;
+                const uint32_t found = probe_general(m, ent.x, start, 2u * stride_of(q.t, stride_index(hh)), serving, C, q.t.ctl);
                 if (serving && found != PROBE_FAILED) part_accumulate(m, found, ent.y, q.t.vals + base, C, q.t.ctl);
             }
         }
@@ -489,11 +502,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
             if (next < n_parts) {
                 const unsigned char* nk = reinterpret_cast<const unsigned char*>(q.t.keys + (ull)next * C);
                 for (uint32_t off = threadIdx.x * 128u; off < C * 8u; off += blockDim.x * 128u) prefetch_l2(nk + off);
-                if (warp < q.n_used) {
-                    const ull nb = ((ull)warp << q.t.lp) + next;
-                    const uint32_t bytes = q.spill_cnt[nb] * 16u;
-                    if (lane * 128u < bytes) prefetch_l2(q.spill + nb * q.cap * 16ull + lane * 128u);
-                }
+                if (warp < q.n_used) prefetch_entries(q, ((ull)warp << q.t.lp) + next, lane);
             }
         }
         // read-modify-write of the touched slots, four per thread in flight (the loads miss L1 by
@@ -521,7 +530,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 const ull nlo = old[u].x + ((ull)s_a0[i] | ((ull)s_a1[i] << 32));
                 const ull cnthi = old[u].y + (ull)(c[u] & ~NEW_KEY_FLAG) + ((nlo < old[u].x ? 1ull : 0ull) << HI_SHIFT);
                 q.t.vals[base + i] = make_ulonglong2(nlo, cnthi);
-                if (c[u] & NEW_KEY_FLAG) q.t.keys[base + i] = s_keys[i];
+                if (c[u] & NEW_KEY_FLAG) q.t.keys[base + i] = ~key_of_ckey(s_keys[i]);
             }
         }
         // this partition's buffers are empty again

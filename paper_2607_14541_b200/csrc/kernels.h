@@ -4,22 +4,17 @@
 
 namespace atrex {
 
-// Build-time variants of the scatter pass (the defaults are the fastest measured; the others are kept
-// so that the comparison can be repeated):
+// Build-time variant of the scatter pass (the default is the fastest measured; the other is kept so
+// that the comparison can be repeated):
 //   ATREX_SCATTER_RING   stages of a shared-memory ring that a producer warp fills with bulk
 //                        asynchronous copies of record tiles (0: records are loaded straight into
 //                        registers, two 32-byte loads alternating per thread)
-//   ATREX_SCATTER_PAIR   1: spill entries leave in pairs as whole 32-byte sectors (pairing mailbox per
-//                        partition in shared memory); 0: every entry is stored on its own
 #ifndef ATREX_SCATTER_RING
 #define ATREX_SCATTER_RING 0
 #endif
-#ifndef ATREX_SCATTER_PAIR
-#define ATREX_SCATTER_PAIR 0
-#endif
 
 // Shared memory of the scatter pass (dynamic, one CTA per SM) and what fits in it.  Per partition a
-// cursor word (and a 16-byte pairing mailbox), 16 KB of card-hour weights, the record ring if there
+// cursor word, 16 KB of card-hour weights, the record ring if there
 // is one, then the hot directory: a tag byte, an 8-byte key and 12 bytes of accumulators per slot, in
 // whole 4-way buckets.
 constexpr uint32_t APPW_SMEM_MAX = 4096;
@@ -27,9 +22,8 @@ constexpr uint32_t SCATTER_SMEM_BYTES = 232448 - 1024;
 constexpr uint32_t SCATTER_RING_STAGES = ATREX_SCATTER_RING;
 constexpr uint32_t SCATTER_CONSUMER_WARPS = SCATTER_RING_STAGES ? 31 : 32;
 constexpr uint32_t SCATTER_RING_TILE = SCATTER_CONSUMER_WARPS * 32 * 16;   // one record per consumer thread
-constexpr bool SCATTER_PAIR = ATREX_SCATTER_PAIR != 0;
 constexpr uint32_t scatter_fixed_bytes(uint32_t lp) {
-    return ((SCATTER_PAIR ? 20u : 4u) << lp) + 4u * APPW_SMEM_MAX + SCATTER_RING_STAGES * SCATTER_RING_TILE + 128u;
+    return (4u << lp) + 4u * APPW_SMEM_MAX + SCATTER_RING_STAGES * SCATTER_RING_TILE + 128u;
 }
 constexpr uint32_t scatter_hot_slots(uint32_t lp) { return ((SCATTER_SMEM_BYTES - scatter_fixed_bytes(lp)) / 21u) & ~31u; }
 
@@ -49,11 +43,12 @@ struct IngestParams {
     uint32_t hot_buckets;      // hot_slots / 4
     ulonglong2* hot_img;       // [n_groups][hot_slots] each CTA's directory sums since the last fold, {lo, count | hi << 40}
     TableRef t;
-    // spill buffers: entry i of scatter CTA g for partition p at spill + ((g * P + p) * cap + i) * 16 bytes
+    // spill buffers: entry i of scatter CTA g for partition p at spill + ((g * P + p) * cap + i) * 12 bytes: an 8-byte
+    // word {product, operator} and a 4-byte word {phase, low hash bits}, the 8-byte word at the 8-byte aligned end
     unsigned char* spill;
     uint32_t* spill_cnt;       // [n_groups][P]
     uint32_t n_groups;         // G, row pitch of the buffers (= CTAs of the widest scatter launch)
-    uint32_t cap;              // entries per (partition, CTA) buffer
+    uint32_t cap;              // entries per (partition, CTA) buffer, a multiple of 32 (whole 128-byte lines)
     uint32_t drain_above;      // ask for a drain when a buffer holds more entries than this
     ull seq;                   // sequence number of this launch
 };

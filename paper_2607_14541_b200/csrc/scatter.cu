@@ -6,9 +6,8 @@
 //   * Keys found in the shared-memory HOT DIRECTORY (the most frequent keys of a sample of the
 //     trace, identical in every CTA, read-only during the pass) are accumulated on the spot with
 //     32-bit shared-memory atomics in limbs with explicit carries.
-//   * Every other record becomes a 16-byte {key, product} entry appended to the CTA's private
-//     buffer of the key's partition (see spill_append: stored on its own with the next line of the
-//     buffer prefetched into L2, or -- build-time variant -- paired into whole 32-byte sectors).
+//   * Every other record becomes a 12-byte entry {product, operator, phase, hash bits} appended to
+//     the CTA's private buffer of the key's partition (see spill_append).
 // At the end the CTA adds its directory accumulators to its own row of a directory image
 // ([CTA][slot], plain coalesced read-modify-writes; hot_fold_kernel adds the rows into the table
 // before results are read) and stores its per-partition cursors: the buffers persist across launches
@@ -17,8 +16,7 @@
 // The kernel runs out of issue slots, shared-memory pipe cycles and latency-hiding warps long before
 // it runs out of DRAM bandwidth, so the hot loop is written for a low instruction count: the shared-memory layout is a compile-time function
 // of the partition count (every array address is a register plus an immediate), rarely taken
-// branches (products of 2^48 and more, a full buffer, a wait for another lane's turn, a drain of a
-// directory slot) are calls to functions that are not inlined, and the three load buffers rotate by
+// branches (products of 2^48 and more, a full buffer, a drain of a directory slot) are calls to functions that are not inlined, and the three load buffers rotate by
 // name instead of being copied.
 #include "atrex_dev.cuh"
 #include "kernels.h"
@@ -41,8 +39,7 @@ struct Smem {
     static constexpr uint32_t SLOTS = scatter_hot_slots(LP);   // directory slots, whole 4-way buckets
     static constexpr uint32_t NB = SLOTS / DIR_WAYS;
     static constexpr uint32_t RING = 0;                         // record ring: SCATTER_RING_STAGES tiles
-    static constexpr uint32_t MBOX = RING + SCATTER_RING_STAGES * SCATTER_RING_TILE;   // ulonglong2[P]  first entry of a pair, waiting for the second
-    static constexpr uint32_t CUR = MBOX + (SCATTER_PAIR ? 16u * P : 0u);   // u32[P]  tickets handed out (bits 0..15), appends completed (16..31)
+    static constexpr uint32_t CUR = RING + SCATTER_RING_STAGES * SCATTER_RING_TILE;   // u32[P]  entries appended to this CTA's buffer of each partition
     static constexpr uint32_t APPW = CUR + 4u * P;              // u32[APPW_SMEM_MAX]  card-hour weights
     static constexpr uint32_t TAG = APPW + 4u * APPW_SMEM_MAX;  // u32[NB + 1]  four 8-bit tags per bucket (+ one pad bucket)
     static constexpr uint32_t KEYS = (TAG + 4u * (NB + 1u) + 7u) & ~7u;   // ull[SLOTS + 4]  key, all ones = empty
@@ -65,23 +62,10 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
     asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
     return v;
 }
-__device__ __forceinline__ uint32_t lds_u32_volatile(uint32_t a) {
-    uint32_t v;
-    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
-    return v;
-}
 __device__ __forceinline__ ull lds_u64(uint32_t a) {
     ull v;
     asm("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(a));
     return v;
-}
-__device__ __forceinline__ ulonglong2 lds_v2u64(uint32_t a) {
-    ulonglong2 v;
-    asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ void sts_v2u64(uint32_t a, ull x, ull y) {
-    asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(a), "l"(x), "l"(y) : "memory");
 }
 __device__ __forceinline__ uint32_t atoms_add(uint32_t a, uint32_t v) {
     uint32_t o;
@@ -96,20 +80,11 @@ __device__ __forceinline__ uint32_t atoms_exch(uint32_t a, uint32_t v) {
     asm volatile("atom.shared.exch.b32 %0, [%1], %2;" : "=r"(o) : "r"(a), "r"(v) : "memory");
     return o;
 }
-// zero, in a form the compiler cannot fold: makes an instruction's operand depend on a loaded value
-__device__ __forceinline__ uint32_t zero_after(ull loaded) {
-    uint32_t z;
-    asm volatile("and.b32 %0, %1, 0;" : "=r"(z) : "r"((uint32_t)loaded));
-    return z;
+__device__ __forceinline__ void stg_u64(void* at, ull v, ull policy) {
+    asm volatile("st.global.L2::cache_hint.u64 [%0], %1, %2;" ::"l"(at), "l"(v), "l"(policy) : "memory");
 }
-__device__ __forceinline__ void stg_entry(void* at, ull key, ull prod, ull policy) {
-    asm volatile("st.global.L2::cache_hint.v2.u64 [%0], {%1, %2}, %3;" ::"l"(at), "l"(key), "l"(prod), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void stg_sector(void* at, ull a, ull b, ull c, ull d, ull policy) {
-    asm volatile("st.global.L2::cache_hint.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8}, %9;" ::"l"(at), "r"((uint32_t)a),
-                 "r"((uint32_t)(a >> 32)), "r"((uint32_t)b), "r"((uint32_t)(b >> 32)), "r"((uint32_t)c), "r"((uint32_t)(c >> 32)),
-                 "r"((uint32_t)d), "r"((uint32_t)(d >> 32)), "l"(policy)
-                 : "memory");
+__device__ __forceinline__ void stg_u32(void* at, uint32_t v, ull policy) {
+    asm volatile("st.global.L2::cache_hint.u32 [%0], %1, %2;" ::"l"(at), "r"(v), "l"(policy) : "memory");
 }
 
 // What the hot loop keeps in registers (everything else is read from the kernel's parameter block,
@@ -162,28 +137,6 @@ __device__ __forceinline__ void dir_add(const IngestParams& p, const Ctx& c, uin
     }
 }
 
-// Spill: append {key, product} to this CTA's buffer of the key's partition, two entries at a time.
-// A 16-byte store into a 32-byte sector that is not in L2 makes the L2 read the sector from DRAM first
-// (a quarter of this pass's DRAM traffic when every entry was stored on its own), so entries are
-// paired in shared memory and leave as whole sectors.  Each partition has a cursor word -- tickets
-// handed out in bits 0..15, appends completed in bits 16..31 -- and a 16-byte mailbox.  A ticket
-// holder acts when the completed count has reached its ticket: an even ticket puts its entry into the
-// mailbox, the odd ticket after it takes that entry out and stores both to positions (ticket - 1,
-// ticket).  Every transition has exactly one owner, so nothing is claimed twice.
-template <uint32_t LP>
-__device__ __forceinline__ void spill_turn(const IngestParams& p, const Ctx& c, uint32_t part, uint32_t pos, ull key, ull prod) {
-    const uint32_t mb = c.sb + Smem<LP>::MBOX + part * 16u;
-    const uint32_t cw = c.sb + Smem<LP>::CUR + part * 4u;
-    if (pos & 1u) {
-        const ulonglong2 first = lds_v2u64(mb);                    // shared-memory accesses of a thread are performed
-        reds_add(cw, 0x10000u + zero_after(first.x));              // in program order; frees the mailbox only after the load
-        stg_sector(c.my_spill + (size_t)ATREX_INDEX(part * p.cap + pos - 1u, (p.cap << LP) - 1u, p.t.ctl) * 16u, first.x, first.y, key, prod, c.keep);
-    } else {
-        sts_v2u64(mb, key, prod);
-        reds_add(cw, 0x10000u);
-    }
-}
-
 // (rare) The buffer is full: the ticket is handed back and the record takes the exact slow path.
 template <uint32_t LP>
 __device__ __noinline__ void spill_overflow(TableRef t, uint32_t cw, ull key, ull prod, uint32_t h) {
@@ -191,61 +144,42 @@ __device__ __noinline__ void spill_overflow(TableRef t, uint32_t cw, ull key, ul
     table_accumulate(t, key, h, prod, 0, 1);
 }
 
-constexpr uint32_t SPILL_WAIT_ROUNDS = 1u << 20;
-
-// Called by all lanes of a warp together; `todo` lanes append.
-template <uint32_t LP, bool PAIR>
-__device__ __forceinline__ void spill_append(const IngestParams& p, Ctx& c, bool todo, ull key, ull prod, uint32_t h) {
+// Spill: the record becomes a 12-byte entry in this CTA's buffer of the key's partition -- an 8-byte
+// word {product (48 bits), operator} and a 4-byte word {phase, the hash bits below the partition's},
+// kept as two arrays per buffer.  Inside its partition (the hash's top bits) the pair (phase,
+// operator, hash) identifies the key: for a given operator the hash is a bijection of the shape
+// (shape_of_hash).  Each word is stored on its own; two entries before a buffer's 8-byte array reaches
+// its next 128-byte line (and likewise for the 4-byte array) that line is pulled into L2 -- a partial
+// store into a line that is not cached stalls on a fill -- and the stores ask the L2 to evict their
+// lines last: a buffer's current lines are written to 16 and 32 times over tens of thousands of cycles
+// while 16 GiB of records stream through the same cache.
+template <uint32_t LP>
+__device__ __forceinline__ void spill_append(const IngestParams& p, Ctx& c, bool todo, uint32_t khi, uint32_t shape, ull prod,
+                                             uint32_t h) {
+    if (!todo) return;
     const uint32_t part = ATREX_INDEX(h >> (32 - LP), Smem<LP>::P, p.t.ctl);
     const uint32_t cw = c.sb + Smem<LP>::CUR + part * 4u;
-    if (PAIR) {
-        uint32_t tk = 0;
-        if (todo) tk = atoms_add(cw, 1u);
-        const uint32_t pos = tk & 0xFFFFu;
-        if (todo && pos >= p.cap) {
-            spill_overflow<LP>(p.t, cw, key, prod, h);
-            count_one(&p.t.ctl->n_overflow);
-            todo = false;
-        }
-        // Turns.  Nearly always the completed count already equals the ticket.  Otherwise a smaller
-        // ticket of the same partition has not finished -- often a lane of this very warp that took its
-        // ticket in the same instruction -- so the lanes whose turn it is act, then the warp votes (which
-        // also keeps a waiting lane from spinning ahead of the lane it waits for), then the waiting lanes
-        // look again.  The holder of the smallest unfinished ticket never waits, so this ends; it is
-        // bounded all the same and latches ST_TIMEOUT when it gives up.
-        uint32_t seen = tk >> 16;
-        for (uint32_t rounds = 0;; ++rounds) {
-            if (todo && seen == pos) {
-                spill_turn<LP>(p, c, part, pos, key, prod);
-                todo = false;
-            }
-            if (!__any_sync(0xFFFFFFFFu, todo)) break;
-            if (rounds >= SPILL_WAIT_ROUNDS) {
-                if (todo) atomicOr(&p.t.ctl->status, ST_TIMEOUT);
-                break;
-            }
-            if (todo) seen = lds_u32_volatile(cw) >> 16;
-        }
-    } else if (todo) {
-        // every entry stored on its own; two entries before the buffer reaches its next 128-byte line,
-        // that line is pulled into L2 (a partial store into a line that is not cached stalls on a fill),
-        // and the stores ask the L2 to evict their lines last: a buffer's current line is written to 8
-        // times over ~30 K cycles while 16 GiB of records stream through the same cache
-        const uint32_t tk = atoms_add(cw, 1u);
-        if (tk < p.cap) {
-            unsigned char* at = c.my_spill + (size_t)ATREX_INDEX(part * p.cap + tk, p.cap << LP, p.t.ctl) * 16u;
-            stg_entry(at, key, prod, c.keep);
-            if ((tk & 7u) == 6) asm volatile("prefetch.global.L2 [%0];" ::"l"(at + 32));
-        } else {
-            spill_overflow<LP>(p.t, cw, key, prod, h);
-            count_one(&p.t.ctl->n_overflow);
-        }
+    const uint32_t tk = atoms_add(cw, 1u);
+    if (tk < p.cap) {
+        // Entry tk occupies bytes [12 tk, 12 tk + 12) of the buffer; its 8-byte word sits at whichever
+        // end is 8-byte aligned.  Two or three entries before the buffer reaches its next 128-byte
+        // line, that line is pulled into L2 (a partial store into a line that is not cached stalls on a
+        // fill), and the stores ask the L2 to evict their lines last: a buffer's current line is
+        // written to some 20 times over ~40 K cycles while 16 GiB of records stream through the same cache.
+        unsigned char* at = c.my_spill + ((size_t)part * p.cap + ATREX_INDEX(tk, p.cap, p.t.ctl)) * SPILL_ENTRY_BYTES;
+        const uint32_t odd = tk & 1u;
+        stg_u64(at + odd * 4u, spill_word_a(prod, khi & 0xFFFFu), c.keep);
+        stg_u32(at + 8u - odd * 8u, spill_word_b(khi >> 16, h, LP), c.keep);
+        if (((tk * SPILL_ENTRY_BYTES) & 127u) - 96u < 12u) asm volatile("prefetch.global.L2 [%0];" ::"l"(at + 64));
+    } else {
+        spill_overflow<LP>(p.t, cw, ((ull)khi << 32) | shape, prod, h);
+        count_one(&p.t.ctl->n_overflow);
     }
 }
 
 // One record, start to finish (the register-staged loop has no registers to spare for working on
 // two records at once).  Called by all lanes of a warp together (absent records masked by `present`).
-template <uint32_t LP, bool HOT, bool DEDUPE, bool PAIR, bool FULL>
+template <uint32_t LP, bool HOT, bool DEDUPE, bool FULL>
 __device__ __forceinline__ void one_record(const IngestParams& p, Ctx& c, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3,
                                            bool present) {
     using L = Smem<LP>;
@@ -300,14 +234,14 @@ __device__ __forceinline__ void one_record(const IngestParams& p, Ctx& c, uint32
             todo = false;
         }
     }
-    spill_append<LP, PAIR>(p, c, todo, key, prod, h);
+    spill_append<LP>(p, c, todo, khi, w2, prod, h);
 }
 
 // The same for R records per lane at once (used with the shared-memory record ring, where the
 // registers allow it; w[r] = the record's four words).  Called by all lanes of a
 // warp together (absent records masked by `present`).  Written in stages over the R records so that
 // their shared-memory round trips overlap: all look-ups are issued before the first result is used.
-template <uint32_t LP, bool HOT, bool DEDUPE, bool PAIR, bool FULL, int R>
+template <uint32_t LP, bool HOT, bool DEDUPE, bool FULL, int R>
 __device__ __forceinline__ void process(const IngestParams& p, Ctx& c, const uint32_t (&w)[R][4], bool present) {
     using L = Smem<LP>;
     uint32_t khi[R], h[R], wgt[R], x[R], tags[R];
@@ -401,10 +335,10 @@ __device__ __forceinline__ void process(const IngestParams& p, Ctx& c, const uin
         }
     }
 #pragma unroll
-    for (int r = 0; r < R; ++r) spill_append<LP, PAIR>(p, c, todo[r], ((ull)khi[r] << 32) | w[r][2], prod[r], h[r]);
+    for (int r = 0; r < R; ++r) spill_append<LP>(p, c, todo[r], khi[r], w[r][2], prod[r], h[r]);
 }
 
-template <uint32_t LP, bool HOT, bool DEDUPE, bool PAIR>
+template <uint32_t LP, bool HOT, bool DEDUPE>
 __device__ __forceinline__ void scatter_body(const IngestParams& p, Ctx& c) {
     // CTA b handles record pairs (b + k * gridDim) * 1024 + tid, k = 0, 1, ...  Three 32-byte loads
     // rotate per thread: while one is consumed the next two are in flight.  Rounds in which every
@@ -425,13 +359,13 @@ __device__ __forceinline__ void scatter_body(const IngestParams& p, Ctx& c) {
         }
     };
     auto consume_full = [&](const uint32_t (&raw)[8]) {
-        one_record<LP, HOT, DEDUPE, PAIR, true>(p, c, raw[0], raw[1], raw[2], raw[3], true);
-        one_record<LP, HOT, DEDUPE, PAIR, true>(p, c, raw[4], raw[5], raw[6], raw[7], true);
+        one_record<LP, HOT, DEDUPE, true>(p, c, raw[0], raw[1], raw[2], raw[3], true);
+        one_record<LP, HOT, DEDUPE, true>(p, c, raw[4], raw[5], raw[6], raw[7], true);
     };
     auto consume_tail = [&](uint32_t round, const uint32_t (&raw)[8]) {
         const bool present = round < rounds && first + (ull)round * stride < p.n_pairs;
-        one_record<LP, HOT, DEDUPE, PAIR, false>(p, c, raw[0], raw[1], raw[2], raw[3], present);
-        one_record<LP, HOT, DEDUPE, PAIR, false>(p, c, raw[4], raw[5], raw[6], raw[7], present);
+        one_record<LP, HOT, DEDUPE, false>(p, c, raw[0], raw[1], raw[2], raw[3], present);
+        one_record<LP, HOT, DEDUPE, false>(p, c, raw[4], raw[5], raw[6], raw[7], present);
     };
     fetch(0, bufA);
     fetch(1, bufB);
@@ -464,7 +398,7 @@ __device__ __forceinline__ void scatter_body(const IngestParams& p, Ctx& c) {
         uint4 v = make_uint4(0, 0, 0, 0);
         const bool present = threadIdx.x < p.n_single;
         if (present) v = *reinterpret_cast<const uint4*>(threadIdx.x == 0 ? p.single[0] : p.single[1]);
-        one_record<LP, HOT, DEDUPE, PAIR, false>(p, c, v.x, v.y, v.z, v.w, present);
+        one_record<LP, HOT, DEDUPE, false>(p, c, v.x, v.y, v.z, v.w, present);
     }
 }
 
@@ -512,7 +446,7 @@ __device__ __forceinline__ uint4 lds_record(uint32_t a) {
     return v;
 }
 
-template <uint32_t LP, bool HOT, bool DEDUPE, bool PAIR>
+template <uint32_t LP, bool HOT, bool DEDUPE>
 __device__ __forceinline__ void ring_body(const IngestParams& p, Ctx& c, ull* full_bar, ull* empty_bar, volatile uint32_t* abort_flag) {
     constexpr uint32_t S = SCATTER_RING_STAGES > 0 ? SCATTER_RING_STAGES : 1;
     constexpr uint32_t TILE_RECS = SCATTER_CONSUMER_WARPS * 32;
@@ -575,21 +509,20 @@ __device__ __forceinline__ void ring_body(const IngestParams& p, Ctx& c, ull* fu
         const uint32_t w[2][4] = {{r0.x, r0.y, r0.z, r0.w}, {r1.x, r1.y, r1.z, r1.w}};
         const bool full = second && first1 + TILE_RECS <= p.n_recs;     // both tiles complete (uniform)
         if (full) {
-            process<LP, HOT, DEDUPE, PAIR, true, 2>(p, c, w, true);
+            process<LP, HOT, DEDUPE, true, 2>(p, c, w, true);
         } else {
             // ragged end: one record at a time, each with its own mask
             const uint32_t wa[1][4] = {{r0.x, r0.y, r0.z, r0.w}}, wb[1][4] = {{r1.x, r1.y, r1.z, r1.w}};
-            process<LP, HOT, DEDUPE, PAIR, false, 1>(p, c, wa, p0);
-            process<LP, HOT, DEDUPE, PAIR, false, 1>(p, c, wb, p1);
+            process<LP, HOT, DEDUPE, false, 1>(p, c, wa, p0);
+            process<LP, HOT, DEDUPE, false, 1>(p, c, wb, p1);
         }
     }
 }
 
-template <uint32_t LP, bool HOT, bool PAIR>
+template <uint32_t LP, bool HOT>
 __global__ void __launch_bounds__(SCATTER_THREADS, 1) scatter_kernel(IngestParams p) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     using L = Smem<LP>;
-    ulonglong2* g_mbox = reinterpret_cast<ulonglong2*>(smem_raw + L::MBOX);
     uint32_t* g_cursor = reinterpret_cast<uint32_t*>(smem_raw + L::CUR);
     uint32_t* g_appw = reinterpret_cast<uint32_t*>(smem_raw + L::APPW);
     uint32_t* g_tag = reinterpret_cast<uint32_t*>(smem_raw + L::TAG);
@@ -611,17 +544,11 @@ __global__ void __launch_bounds__(SCATTER_THREADS, 1) scatter_kernel(IngestParam
     Ctx c;
     c.sb = smem_addr(smem_raw);
     c.mult = HOT ? (uint32_t)p.t.ctl->dir_mult : 1u;
-    c.my_spill = p.spill + ((size_t)blockIdx.x << LP) * p.cap * 16u;
+    c.my_spill = p.spill + ((size_t)blockIdx.x << LP) * p.cap * SPILL_ENTRY_BYTES;
     asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(c.keep));
 
     // The buffers persist across launches until the partition pass drains them: resume the cursors.
-    // A buffer holding an odd number of entries gets its last one back into the mailbox, where the
-    // next entry will join it (the sector is then rewritten whole).
-    for (uint32_t i = threadIdx.x; i < L::P; i += blockDim.x) {
-        const uint32_t n = p.spill_cnt[((size_t)blockIdx.x << LP) + i];
-        g_cursor[i] = PAIR ? (n | (n << 16)) : n;
-        if (PAIR && (n & 1u)) g_mbox[i] = *reinterpret_cast<const ulonglong2*>(c.my_spill + ((size_t)i * p.cap + (n - 1u)) * 16u);
-    }
+    for (uint32_t i = threadIdx.x; i < L::P; i += blockDim.x) g_cursor[i] = p.spill_cnt[((size_t)blockIdx.x << LP) + i];
     if (p.appw_in_smem != 0)
         for (uint32_t i = threadIdx.x; i < p.n_apps; i += blockDim.x) g_appw[i] = p.app_w[i];
     if (HOT) {
@@ -639,33 +566,27 @@ __global__ void __launch_bounds__(SCATTER_THREADS, 1) scatter_kernel(IngestParam
 
     if (SCATTER_RING_STAGES > 0) {
         if (HOT && p.t.ctl->hot_skew != 0)
-            ring_body<LP, HOT, true, PAIR>(p, c, s_full, s_empty, &s_abort);
+            ring_body<LP, HOT, true>(p, c, s_full, s_empty, &s_abort);
         else
-            ring_body<LP, HOT, false, PAIR>(p, c, s_full, s_empty, &s_abort);
+            ring_body<LP, HOT, false>(p, c, s_full, s_empty, &s_abort);
     } else {
         if (HOT && p.t.ctl->hot_skew != 0)
-            scatter_body<LP, HOT, true, PAIR>(p, c);
+            scatter_body<LP, HOT, true>(p, c);
         else
-            scatter_body<LP, HOT, false, PAIR>(p, c);
+            scatter_body<LP, HOT, false>(p, c);
     }
 
     __syncthreads();
     uint32_t spilled = 0, fullest = 0;
-    bool crowded = false, unfinished = false;
+    bool crowded = false;
     for (uint32_t i = threadIdx.x; i < L::P; i += blockDim.x) {
         const size_t at = ((size_t)blockIdx.x << LP) + i;
-        const uint32_t before = p.spill_cnt[at], word = g_cursor[i], n = PAIR ? (word & 0xFFFFu) : min(word, p.cap);
-        if (PAIR) {
-            unfinished |= (word >> 16) != n;   // a ticket that never got its turn (only after ST_TIMEOUT)
-            // an entry without a partner leaves on its own (one partial sector per buffer and launch at most)
-            if (n & 1u) *reinterpret_cast<ulonglong2*>(c.my_spill + ((size_t)i * p.cap + (n - 1u)) * 16u) = g_mbox[i];
-        }
+        const uint32_t before = p.spill_cnt[at], n = min(g_cursor[i], p.cap);
         p.spill_cnt[at] = n;
         spilled += n - before;
         crowded |= n > p.drain_above;
         fullest = max(fullest, n);
     }
-    if (unfinished) atomicOr(&p.t.ctl->status, ST_TIMEOUT);
     fullest = __reduce_max_sync(0xFFFFFFFFu, fullest);
     spilled = __reduce_add_sync(0xFFFFFFFFu, spilled);
     crowded = __any_sync(0xFFFFFFFFu, crowded);
@@ -704,23 +625,21 @@ __global__ void __launch_bounds__(SCATTER_THREADS, 1) scatter_kernel(IngestParam
     }
 }
 
-constexpr bool PAIR_DEFAULT = SCATTER_PAIR;
-
 template <uint32_t LP>
 cudaError_t prepare_lp() {
-    cudaError_t e = cudaFuncSetAttribute(scatter_kernel<LP, true, PAIR_DEFAULT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    cudaError_t e = cudaFuncSetAttribute(scatter_kernel<LP, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)SCATTER_SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(scatter_kernel<LP, false, PAIR_DEFAULT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(scatter_kernel<LP, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)SCATTER_SMEM_BYTES);
 }
 
 template <uint32_t LP>
 void launch_lp(const IngestParams& p, bool hot, int grid, cudaStream_t stream) {
     if (hot)
-        scatter_kernel<LP, true, PAIR_DEFAULT><<<grid, SCATTER_THREADS, Smem<LP>::TOTAL, stream>>>(p);
+        scatter_kernel<LP, true><<<grid, SCATTER_THREADS, Smem<LP>::TOTAL, stream>>>(p);
     else
-        scatter_kernel<LP, false, PAIR_DEFAULT><<<grid, SCATTER_THREADS, Smem<LP>::TOTAL, stream>>>(p);
+        scatter_kernel<LP, false><<<grid, SCATTER_THREADS, Smem<LP>::TOTAL, stream>>>(p);
 }
 
 }  // namespace

@@ -30,12 +30,11 @@ def test_parity_cases_under_the_bounds_checked_build():
     assert " passed" in run.stdout
 
 
-@pytest.mark.parametrize("variant", ["ring4", "pair"])
+@pytest.mark.parametrize("variant", ["ring4"])
 def test_parity_cases_under_the_scatter_variants(variant):
-    """The scatter pass's build-time variants -- the shared-memory record ring filled by bulk asynchronous
-    copies, and spill entries leaving as whole sectors through the pairing mailboxes -- are slower than
-    the default and therefore not what ships, but they are kept buildable and exact: the same parity
-    cases, bit for bit against the oracle."""
+    """The scatter pass's build-time variant -- the shared-memory record ring filled by bulk asynchronous
+    copies -- is slower than the default and therefore not what ships, but it is kept buildable and
+    exact: the same parity cases, bit for bit against the oracle."""
     import importlib.util
     spec = importlib.util.spec_from_file_location("atrex_build", os.path.join(ROOT, "paper_2607_14541_b200", "build.py"))
     mod = importlib.util.module_from_spec(spec)
