@@ -5,8 +5,8 @@
 // the L2's atomic rate, not by bandwidth, so the hot path avoids global atomics altogether:
 //
 // Pass 1  SCATTER  (scatter.cu) accumulates the records of hot keys in a shared-memory directory
-//   and appends every other record as a 16-byte {key, product} entry to the CTA's private buffer
-//   of the key's partition.
+//   and appends every other record as a 12-byte entry to the CTA's private buffer of the key's
+//   partition.
 //
 // Pass 2  PARTITION  (persistent CTAs, one partition at a time each).  Runs lazily: only when a
 //   buffer is filling up, or when results are about to be read.  The CTA copies its
@@ -34,28 +34,12 @@ __device__ __forceinline__ uint32_t dir_bucket_of_key(ull key, uint32_t mult, ui
 }
 __constant__ uint32_t DIR_MULTS[4] = {0xC2B2AE35u, 0x27D4EB2Fu, 0x165667B1u, 0x9E3779B9u};
 
-__device__ __forceinline__ void ld_stream_256(const void* p, uint32_t (&w)[8]) {
-    asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
-                 : "l"(p));
-}
-
 // Shared memory is addressed explicitly through 32-bit shared-window addresses in the hot
 // loops: one integer add per access instead of generic 64-bit pointer arithmetic.
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
-    return v;
-}
 __device__ __forceinline__ ulonglong2 lds_v2u64(uint32_t a) {
     ulonglong2 v;
     asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ ull lds_u64(uint32_t a) {
-    ull v;
-    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(a));
     return v;
 }
 __device__ __forceinline__ uint32_t atoms_add(uint32_t a, uint32_t v) {
@@ -74,26 +58,6 @@ __device__ __forceinline__ uint32_t atoms_exch(uint32_t a, uint32_t v) {
     asm volatile("atom.shared.exch.b32 %0, [%1], %2;" : "=r"(o) : "r"(a), "r"(v) : "memory");
     return o;
 }
-__device__ __forceinline__ uint32_t lds_u32_volatile(uint32_t a) {
-    uint32_t v;
-    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ void sts_v2u64(uint32_t a, ull x, ull y) {
-    asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(a), "l"(x), "l"(y) : "memory");
-}
-// zero, in a form the compiler cannot fold: makes one instruction's operand depend on a loaded value
-__device__ __forceinline__ uint32_t zero_after(ull loaded) {
-    uint32_t z;
-    asm volatile("and.b32 %0, %1, 0;" : "=r"(z) : "r"((uint32_t)loaded));
-    return z;
-}
-__device__ __forceinline__ void stg_sector(void* at, ull a, ull b, ull c, ull d) {
-    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(at), "r"((uint32_t)a), "r"((uint32_t)(a >> 32)),
-                 "r"((uint32_t)b), "r"((uint32_t)(b >> 32)), "r"((uint32_t)c), "r"((uint32_t)(c >> 32)), "r"((uint32_t)d),
-                 "r"((uint32_t)(d >> 32))
-                 : "memory");
-}
 __device__ __forceinline__ ull atoms_cas64(uint32_t a, ull expected, ull desired) {
     ull o;
     asm volatile("atom.shared.cas.b64 %0, [%1], %2, %3;" : "=l"(o) : "r"(a), "l"(expected), "l"(desired) : "memory");
@@ -103,23 +67,11 @@ __device__ __forceinline__ ull atoms_cas64(uint32_t a, ull expected, ull desired
 // Shared-memory accumulation uses native 32-bit atomics only (64-bit shared atomics are
 // compare-and-swap loops).  A slot's weighted time is kept in two limbs: the returning add on
 // the low limb tells the adder whether it wrapped, and the adder then adds the carry, with the
-// value's high word, to the high limb.  One add raises the high limb by at most 2^21 (a warp's
+// value's high word, to the high limb (part_accumulate).  One add raises the high limb by at most 2^21 (a warp's
 // combined 32 records of < 2^48 each), so the adder that takes it across 2^30 drains both
 // limbs; the adds that can slip in before its exchange (one per thread of the CTA) stay below
 // 2^31, so the high limb never wraps.
 constexpr uint32_t DRAIN_BIT = 0x40000000u;
-
-// returns true when the caller must drain the slot.  Most products fit 32 bits and most low-limb adds
-// do not wrap: the high limb is then left alone.
-__device__ __forceinline__ bool limbs_add(uint32_t a0, uint32_t a1, uint32_t cnt, ull v, uint32_t count) {
-    const uint32_t v0 = (uint32_t)v;
-    const uint32_t o0 = atoms_add(a0, v0);
-    reds_add(cnt, count);
-    const uint32_t x = (uint32_t)(v >> 32) + ((o0 + v0 < o0) ? 1u : 0u);
-    if (x == 0) return false;
-    const uint32_t o1 = atoms_add(a1, x);
-    return ((o1 + x) & ~o1 & DRAIN_BIT) != 0;
-}
 
 __device__ __forceinline__ ull limbs_drain(uint32_t a0, uint32_t a1, ull* hi_out) {
     // the two exchanges need not be simultaneous: whatever lands between them stays in the
@@ -184,10 +136,17 @@ __global__ void __launch_bounds__(FOLD_WARPS * 32) hot_fold_kernel(const ull* ho
 // round, once the warp's share of the stream is through; then write the deltas back.
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
-// Shared-window addresses of the partition pass's arrays.
+// Shared-window addresses of the partition pass's arrays: keys ull[C] (the pass's own key form, 0 =
+// empty), acc {u32 low limb, u32 count | NEW_KEY_FLAG}[C], a1 u32[C] (high limb).
 struct PartSmem {
-    uint32_t keys, a0, a1, cnt;
+    uint32_t keys, acc, a1;
 };
+
+__device__ __forceinline__ uint4 lds_v4u32(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
 
 // General probe, one entry per lane (busy = this lane has one): walks the key's probe sequence from
 // the pair at `slot`, claims the first free slot if the key is not there.  Warp-convergent.  Returns
@@ -208,7 +167,7 @@ __device__ __forceinline__ uint32_t probe_general(const PartSmem& m, ull skey, u
                 // claim the first empty slot of the pair; a lost race re-reads the pair
                 const uint32_t at = slot + (kk.x == 0 ? 0u : 1u);
                 const ull old = atoms_cas64(m.keys + at * 8, 0ull, skey);
-                if (old == 0) reds_or(m.cnt + at * 4, NEW_KEY_FLAG);
+                if (old == 0) reds_or(m.acc + at * 8 + 4, NEW_KEY_FLAG);
                 if (old == 0 || old == skey) {
                     slot = at;
                     busy = false;
@@ -228,16 +187,28 @@ __device__ __forceinline__ uint32_t probe_general(const PartSmem& m, ull skey, u
     return slot;
 }
 
-// One entry's product and count into its slot's limbs; the adder that fills the high limb moves the
-// slot's sums to HBM (this CTA owns the slot, so those adds are exact; the write-back adds on top).
-__device__ __forceinline__ void part_accumulate(const PartSmem& m, uint32_t slot, ull v, ulonglong2* vals_of_partition, uint32_t C, Control* ctl) {
+// A slot whose high limb filled up: its sums move to HBM (this CTA owns the slot, so those adds are
+// exact; the write-back adds on top).  Rare, hence not inlined.
+__device__ __noinline__ void part_drain_slot(uint32_t acc, uint32_t a1, ulonglong2* val) {
+    ull hi, lo = limbs_drain(acc, a1, &hi);
+    ull* vp = reinterpret_cast<ull*>(val);
+    ull old = atomicAdd(vp, lo);
+    hi += (old + lo < old) ? 1ull : 0ull;
+    if (hi) atomicAdd(vp + 1, hi << HI_SHIFT);
+}
+
+// One entry's product (vlo + 2^32 vhi, vhi < 2^16) and count into its slot's limbs: a returning add on
+// the low limb, whose wrap is the carry; the high limb is touched only when there is something to add.
+__device__ __forceinline__ void part_accumulate(const PartSmem& m, uint32_t slot, uint32_t vlo, uint32_t vhi,
+                                                ulonglong2* vals_of_partition, uint32_t C, Control* ctl) {
     slot = ATREX_INDEX(slot, C, ctl);
-    if (limbs_add(m.a0 + slot * 4, m.a1 + slot * 4, m.cnt + slot * 4, v, 1u)) {
-        ull hi, lo = limbs_drain(m.a0 + slot * 4, m.a1 + slot * 4, &hi);
-        ull* vp = reinterpret_cast<ull*>(vals_of_partition + slot);
-        ull old = atomicAdd(vp, lo);
-        hi += (old + lo < old) ? 1ull : 0ull;
-        if (hi) atomicAdd(vp + 1, hi << HI_SHIFT);
+    const uint32_t acc = m.acc + slot * 8;
+    const uint32_t o0 = atoms_add(acc, vlo);
+    reds_add(acc + 4, 1u);
+    const uint32_t x = vhi + ((o0 + vlo < o0) ? 1u : 0u);
+    if (x != 0) {
+        const uint32_t o1 = atoms_add(m.a1 + slot * 4, x);
+        if (((o1 + x) & ~o1 & DRAIN_BIT) != 0) part_drain_slot(acc, m.a1 + slot * 4, vals_of_partition + slot);
     }
 }
 
@@ -247,15 +218,21 @@ __device__ __forceinline__ void prefetch_entries(const PartitionParams& q, ull s
     if (lane < 24 && lane * 128u < bytes) prefetch_l2(q.spill + sb * q.cap * SPILL_ENTRY_BYTES + lane * 128u);
 }
 
+// A queued entry: {key, product}; bit 63 of the product word says that the key's first pair was full
+// of other keys when the entry was looked up, so its probe may start at the second pair.
+constexpr ull QUEUED_SKIP_FIRST = 1ull << 63;
+
 // One batch of 128 entries of a sub-buffer, four consecutive ones (48 bytes) per lane.  FULL: the
-// batch is complete (no masks).
-// Entry state is two bit sets per lane -- `open` (present, slot not known yet) and `hit` (slot known).
+// batch is complete (no masks).  Keys are handled as their two 32-bit halves (kh: mark, phase,
+// operator; kl: hash).  Entry state is bit sets per lane -- `open` (present, slot not known yet), `hit`
+// (slot known), `room` (the first pair of the probe sequence had a free slot when it was read).
+// part_bits = the partition's index in the hash's top bits, hmask = the hash bits below them.
 template <bool FULL>
 __device__ __forceinline__ void stream_batch(const PartitionParams& q, const PartSmem& m, const unsigned char* src,
-                                             uint32_t part, uint32_t e0, uint32_t n_e, uint32_t C, ull base, ulonglong2* my_queue,
-                                             uint32_t queue_cap_w, uint32_t& qn_w, unsigned char* s_owner_w, uint32_t lane) {
-    ull key[4], v[4];   // key: the partition pass's form (ckey_of)
-    uint32_t slot[4];
+                                             uint32_t part_bits, uint32_t hmask, uint32_t e0, uint32_t n_e, uint32_t C, ull base,
+                                             ulonglong2* my_queue, uint32_t queue_cap_w, uint32_t& qn_w, unsigned char* s_owner_w,
+                                             uint32_t lane) {
+    uint32_t kh[4], kl[4], vlo[4], vhi[4], slot[4];
     uint32_t open = 0;
     {
         // the lane's entries e, e + 1, e + 2, e + 3 (e a multiple of 4) as twelve words; in an even
@@ -272,54 +249,52 @@ __device__ __forceinline__ void stream_batch(const PartitionParams& q, const Par
 #pragma unroll
             for (int j = 0; j < 3; ++j) w[j] = make_uint4(0, 0, 0, 0);
         }
-        const ull a[4] = {w[0].x | ((ull)w[0].y << 32), w[1].x | ((ull)w[1].y << 32), w[1].z | ((ull)w[1].w << 32), w[2].z | ((ull)w[2].w << 32)};
+        const uint32_t alo[4] = {w[0].x, w[1].x, w[1].z, w[2].z}, ahi[4] = {w[0].y, w[1].y, w[1].w, w[2].w};
         const uint32_t b[4] = {w[0].z, w[0].w, w[2].x, w[2].y};
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            key[u] = ckey_of_spill(a[u], b[u], part, q.t.lp);
-            v[u] = a[u] & 0x0000FFFFFFFFFFFFull;
+            kh[u] = 0x80000000u | ((b[u] >> 8) & 0x00FF0000u) | (ahi[u] >> 16);
+            kl[u] = part_bits | (b[u] & hmask);
+            vlo[u] = alo[u];
+            vhi[u] = ahi[u] & 0xFFFFu;
+            slot[u] = local_of(kl[u], b[u] >> 24, C) & ~1u;  // first pair of the probe sequence
         }
     }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) slot[u] = local_of((uint32_t)key[u], ckey_phase(key[u]), C) & ~1u;  // first pair of the probe sequence
     // First look, straight-line for all four entries: most keys sit in the first pair of slots of
-    // their probe sequence.
-    uint32_t hit = 0;
+    // their probe sequence.  (Pairs fill from the even slot, and slots never empty again.)
+    uint32_t hit = 0, room = 0, even_taken = 0;
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
-        const ulonglong2 kk = lds_v2u64(m.keys + ATREX_INDEX(slot[u], C - 1u, q.t.ctl) * 8);
-        const ull skey = key[u];
-        const bool h1 = kk.y == skey;
+        const uint4 kk = lds_v4u32(m.keys + ATREX_INDEX(slot[u], C - 1u, q.t.ctl) * 8);
+        const bool h0 = kk.x == kl[u] && kk.y == kh[u];
+        const bool h1 = kk.z == kl[u] && kk.w == kh[u];
         if (h1) slot[u] |= 1u;
-        if (kk.x == skey || h1) hit |= 1u << u;
+        if (h0 || h1) hit |= 1u << u;
+        if (kk.w == 0) room |= 1u << u;
+        if (kk.y != 0) even_taken |= 1u << u;
     }
     hit &= open;     // (an absent entry is a well-formed key too)
     open &= ~hit;
-    if (__any_sync(0xFFFFFFFFu, open != 0)) {
-        // A new key whose first pair has room is inserted at once, so that its later occurrences find
-        // it there; losing the slot to another key defers the entry.
+    // A new key whose first pair has room is inserted at once, so that its later occurrences find it
+    // there; a slot lost to another key defers the entry.
+    if (__any_sync(0xFFFFFFFFu, (open & room) != 0)) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            if (open & (1u << u)) {
-                const ulonglong2 kk = lds_v2u64(m.keys + slot[u] * 8);
-                const ull skey = key[u];
-                if (kk.x == skey || kk.y == skey) {            // it appeared meanwhile
-                    slot[u] += kk.x == skey ? 0u : 1u;
+            if (open & room & (1u << u)) {
+                const uint32_t at = slot[u] + ((even_taken >> u) & 1u);
+                const ull skey = ((ull)kh[u] << 32) | kl[u];
+                const ull old = atoms_cas64(m.keys + at * 8, 0ull, skey);
+                if (old == 0) reds_or(m.acc + at * 8 + 4, NEW_KEY_FLAG);
+                if (old == 0 || old == skey) {
+                    slot[u] = at;
                     hit |= 1u << u;
                     open &= ~(1u << u);
-                } else if (kk.x == 0 || kk.y == 0) {
-                    const uint32_t at = slot[u] + (kk.x == 0 ? 0u : 1u);
-                    const ull old = atoms_cas64(m.keys + at * 8, 0ull, skey);
-                    if (old == 0) reds_or(m.cnt + at * 4, NEW_KEY_FLAG);
-                    if (old == 0 || old == skey) {
-                        slot[u] = at;
-                        hit |= 1u << u;
-                        open &= ~(1u << u);
-                    }
                 }
             }
         }
-        // The rest (collisions, keys further down their probe sequence: a few per batch) is not settled
+    }
+    if (__any_sync(0xFFFFFFFFu, open != 0)) {
+        // The rest (keys further down their probe sequence, lost races: a few per batch) is not settled
         // here, where the fixed cost of a general probe round would be paid for a handful of entries: it
         // goes to this warp's queue and is settled after the partition's stream, 32 entries per warp round.
         uint32_t pend[4], before[4], total = 0;
@@ -329,81 +304,79 @@ __device__ __forceinline__ void stream_batch(const PartitionParams& q, const Par
             before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
             total += __popc(pend[u]);
         }
-        if (total != 0) {
-            uint32_t qbase = qn_w;
-            qn_w = min(qn_w + total, queue_cap_w);
+        uint32_t qbase = qn_w;
+        qn_w = min(qn_w + total, queue_cap_w);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if ((open & (1u << u)) && qbase + before[u] < queue_cap_w) {
+                const ull v = vlo[u] | ((ull)vhi[u] << 32) | ((room >> u) & 1u ? 0ull : QUEUED_SKIP_FIRST);
+                my_queue[ATREX_INDEX(qbase + before[u], queue_cap_w, q.t.ctl)] = make_ulonglong2(((ull)kh[u] << 32) | kl[u], v);
+                open &= ~(1u << u);
+            }
+        }
+        // Queue full (a partition made of new keys only): settle the remainder in line.  The pending
+        // entries are handed out one per lane: each one's owner publishes (round, lane) at the entry's
+        // position; lane t serves position t.
+        while (qbase + total > queue_cap_w) {
+            total = 0;
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                if ((open & (1u << u)) && qbase + before[u] < queue_cap_w) {
-                    my_queue[ATREX_INDEX(qbase + before[u], queue_cap_w, q.t.ctl)] = make_ulonglong2(key[u], v[u]);
+                pend[u] = __ballot_sync(0xFFFFFFFFu, (open >> u) & 1u);
+                before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
+                total += __popc(pend[u]);
+            }
+            if (total == 0) break;
+            qbase = queue_cap_w;  // stay in this loop until nothing is pending
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if ((open & (1u << u)) && before[u] < 32) s_owner_w[before[u]] = (unsigned char)((u << 5) | lane);
+            __syncwarp();
+            const bool serving = lane < total;
+            const uint32_t code = serving ? s_owner_w[lane] : lane;
+            const uint32_t from = code & 31u, su = code >> 5;
+            uint32_t kh_s = 0, kl_s = 0, slot_s = 0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t h = __shfl_sync(0xFFFFFFFFu, kh[u], from);
+                const uint32_t l = __shfl_sync(0xFFFFFFFFu, kl[u], from);
+                const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u] & ~1u, from);
+                if (su == (uint32_t)u) {
+                    kh_s = h;
+                    kl_s = l;
+                    slot_s = sl;
+                }
+            }
+            const uint32_t found_s = probe_general(m, ((ull)kh_s << 32) | kl_s, slot_s, 2u * stride_of(q.t, stride_index(kl_s)), serving, C,
+                                                   q.t.ctl);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const uint32_t found = __shfl_sync(0xFFFFFFFFu, found_s, before[u] & 31u);
+                if ((open & (1u << u)) && before[u] < 32) {
                     open &= ~(1u << u);
-                }
-            }
-            // Queue full (a partition made of new keys only): settle the remainder in line.  The pending
-            // entries are handed out one per lane: each one's owner publishes (round, lane) at the entry's
-            // position; lane t serves position t.
-            while (qbase + total > queue_cap_w) {
-                total = 0;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    pend[u] = __ballot_sync(0xFFFFFFFFu, (open >> u) & 1u);
-                    before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
-                    total += __popc(pend[u]);
-                }
-                if (total == 0) break;
-                qbase = queue_cap_w;  // stay in this loop until nothing is pending
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if ((open & (1u << u)) && before[u] < 32) s_owner_w[before[u]] = (unsigned char)((u << 5) | lane);
-                __syncwarp();
-                const bool serving = lane < total;
-                const uint32_t code = serving ? s_owner_w[lane] : lane;
-                const uint32_t from = code & 31u, su = code >> 5;
-                ull key_s = 0;
-                uint32_t slot_s = 0;
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const ull k = __shfl_sync(0xFFFFFFFFu, key[u], from);
-                    const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u] & ~1u, from);
-                    if (su == (uint32_t)u) {
-                        key_s = k;
-                        slot_s = sl;
+                    if (found != PROBE_FAILED) {
+                        slot[u] = found;
+                        hit |= 1u << u;
                     }
                 }
-                const uint32_t found_s = probe_general(m, key_s, slot_s, 2u * stride_of(q.t, stride_index((uint32_t)key_s)), serving, C,
-                                                       q.t.ctl);
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint32_t found = __shfl_sync(0xFFFFFFFFu, found_s, before[u] & 31u);
-                    if ((open & (1u << u)) && before[u] < 32) {
-                        open &= ~(1u << u);
-                        if (found != PROBE_FAILED) {
-                            slot[u] = found;
-                            hit |= 1u << u;
-                        }
-                    }
-                }
-                __syncwarp();  // the owner table is rewritten in the next round
             }
+            __syncwarp();  // the owner table is rewritten in the next round
         }
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
-        if (hit & (1u << u)) part_accumulate(m, slot[u], v[u], q.t.vals + base, C, q.t.ctl);
+        if (hit & (1u << u)) part_accumulate(m, slot[u], vlo[u], vhi[u], q.t.vals + base, C, q.t.ctl);
 }
 
 __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionParams q) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t C = q.t.C;
     ull* s_keys = reinterpret_cast<ull*>(smem_raw);
-    uint32_t* s_a0 = reinterpret_cast<uint32_t*>(s_keys + C);
-    uint32_t* s_a1 = s_a0 + C;
-    uint32_t* s_cnt = s_a1 + C;
+    uint2* s_acc = reinterpret_cast<uint2*>(s_keys + C);      // {low limb, count | NEW_KEY_FLAG}
+    uint32_t* s_a1 = reinterpret_cast<uint32_t*>(s_acc + C);  // high limb
     PartSmem m;
     m.keys = smem_addr(s_keys);
-    m.a0 = smem_addr(s_a0);
+    m.acc = smem_addr(s_acc);
     m.a1 = smem_addr(s_a1);
-    m.cnt = smem_addr(s_cnt);
     __shared__ uint32_t s_total;
     // each warp owns a segment of the CTA's queue: no shared counter, and a warp can settle its own
     // leftovers as soon as its share of the stream is through
@@ -454,9 +427,8 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 const uint32_t i = i0 + u * blockDim.x;
                 if (i < C) {
                     s_keys[i] = k[u] == 0 ? 0ull : ckey_of_key(~k[u]);   // the table stores complemented keys, 0 = empty
-                    s_a0[i] = 0;
+                    s_acc[i] = make_uint2(0, 0);
                     s_a1[i] = 0;
-                    s_cnt[i] = 0;
                 }
             }
         }
@@ -466,6 +438,7 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
         }
         __syncthreads();
 
+        const uint32_t part_bits = part << (32 - q.t.lp), hmask = 0xFFFFFFFFu >> q.t.lp;
         uint32_t qn_w = 0;  // entries in this warp's queue segment (warp-uniform)
         for (uint32_t g = warp; g < q.n_used; g += n_warps) {
             const ull sb = ((ull)g << q.t.lp) + part;
@@ -479,9 +452,9 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 if (lane < 12 && (e0 + 256u) * SPILL_ENTRY_BYTES + lane * 128u < n_e * SPILL_ENTRY_BYTES)
                     prefetch_l2(buf + (e0 + 256u) * SPILL_ENTRY_BYTES + lane * 128u);
                 if (e0 + 128u <= n_e)
-                    stream_batch<true>(q, m, buf, part, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
+                    stream_batch<true>(q, m, buf, part_bits, hmask, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
                 else
-                    stream_batch<false>(q, m, buf, part, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
+                    stream_batch<false>(q, m, buf, part_bits, hmask, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
             }
         }
         {   // this warp's queued entries, one per lane (other warps may still be streaming: the general
@@ -491,9 +464,15 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
                 const bool serving = i0 + lane < qn_w;
                 const ulonglong2 ent = serving ? __ldcg(my_queue + i0 + lane) : make_ulonglong2(0, 0);
                 const uint32_t hh = (uint32_t)ent.x;
-                const uint32_t start = local_of(hh, ckey_phase(ent.x), C) & ~1u;
-                const uint32_t found = probe_general(m, ent.x, start, 2u * stride_of(q.t, stride_index(hh)), serving, C, q.t.ctl);
-                if (serving && found != PROBE_FAILED) part_accumulate(m, found, ent.y, q.t.vals + base, C, q.t.ctl);
+                const uint32_t advance = 2u * stride_of(q.t, stride_index(hh));
+                uint32_t start = local_of(hh, ckey_phase(ent.x), C) & ~1u;
+                if (ent.y & QUEUED_SKIP_FIRST) {
+                    start += advance;
+                    if (start >= C) start -= C;
+                }
+                const uint32_t found = probe_general(m, ent.x, start, advance, serving, C, q.t.ctl);
+                if (serving && found != PROBE_FAILED)
+                    part_accumulate(m, found, (uint32_t)ent.y, (uint32_t)(ent.y >> 32) & 0xFFFFu, q.t.vals + base, C, q.t.ctl);
             }
         }
         __syncthreads();
@@ -508,29 +487,29 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
         // read-modify-write of the touched slots, four per thread in flight (the loads miss L1 by
         // design and mostly come from L2, where the prefetch at the start of the partition put them)
         for (uint32_t i0 = threadIdx.x; i0 < C; i0 += 4 * blockDim.x) {
-            uint32_t c[4];
+            uint2 c[4];   // {low limb, count | NEW_KEY_FLAG}
             ulonglong2 old[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const uint32_t i = i0 + u * blockDim.x;
-                c[u] = i < C ? s_cnt[i] : 0u;
+                c[u] = i < C ? s_acc[i] : make_uint2(0, 0);
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 old[u] = make_ulonglong2(0, 0);
-                if (c[u]) {
+                if (c[u].y) {
                     const ull* vp = reinterpret_cast<const ull*>(q.t.vals + base + i0 + u * blockDim.x);
                     asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(old[u].x), "=l"(old[u].y) : "l"(vp));
                 }
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                if (c[u] == 0) continue;
+                if (c[u].y == 0) continue;
                 const uint32_t i = i0 + u * blockDim.x;
-                const ull nlo = old[u].x + ((ull)s_a0[i] | ((ull)s_a1[i] << 32));
-                const ull cnthi = old[u].y + (ull)(c[u] & ~NEW_KEY_FLAG) + ((nlo < old[u].x ? 1ull : 0ull) << HI_SHIFT);
+                const ull nlo = old[u].x + ((ull)c[u].x | ((ull)s_a1[i] << 32));
+                const ull cnthi = old[u].y + (ull)(c[u].y & ~NEW_KEY_FLAG) + ((nlo < old[u].x ? 1ull : 0ull) << HI_SHIFT);
                 q.t.vals[base + i] = make_ulonglong2(nlo, cnthi);
-                if (c[u] & NEW_KEY_FLAG) q.t.keys[base + i] = ~key_of_ckey(s_keys[i]);
+                if (c[u].y & NEW_KEY_FLAG) q.t.keys[base + i] = ~key_of_ckey(s_keys[i]);
             }
         }
         // this partition's buffers are empty again
