@@ -175,6 +175,18 @@ struct atrex_agg {
     int last_cuda_error = 0;
     uint64_t launches = 0;
 
+    // eight odd primes, one per byte, that do not divide m (m even or a power of two times such a number:
+    // the strides are then coprime to it)
+    static ull strides_for(uint32_t m) {
+        ull strides = 0;
+        uint32_t n = 0;
+        for (uint32_t c = 7; n < 8; c += 2) {
+            bool prime = true;
+            for (uint32_t d = 3; d * d <= c; d += 2) prime = prime && (c % d != 0);
+            if (prime && m % c != 0) strides |= (ull)c << (8 * n++);
+        }
+        return strides;
+    }
     TableRef table_ref() const {
         TableRef t;
         t.keys = keys;
@@ -182,14 +194,7 @@ struct atrex_agg {
         t.lp = L.lp;
         t.C = L.C;
         t.ctl = ctl;
-        // eight odd primes that do not divide the number of slot pairs
-        uint32_t n = 0;
-        t.strides = 0;
-        for (uint32_t c = 7; n < 8; c += 2) {
-            bool prime = true;
-            for (uint32_t d = 3; d * d <= c; d += 2) prime = prime && (c % d != 0);
-            if (prime && (L.C / 2) % c != 0) t.strides |= (ull)c << (8 * n++);
-        }
+        t.strides = strides_for(L.C / 2);   // in slot pairs
         return t;
     }
     WorkRef work_ref() const {
@@ -197,6 +202,7 @@ struct atrex_agg {
         w.table = L.work_slots ? work : nullptr;
         w.lp = L.lp;
         w.Cw = L.Cw;
+        w.strides = strides_for(L.Cw ? L.Cw : 1);
         return w;
     }
     int scan_grid(ull n_items, int threads) const {

@@ -87,6 +87,12 @@ __global__ void __launch_bounds__(TOT_THREADS) totals_kernel(TableRef tab, ull n
 }
 
 // ---- per-key results ----------------------------------------------------------------------
+// The work table is probed by double hashing (strides coprime to the partition's slot count): with
+// linear probing the longest of a warp's 32 probe sequences -- which is what the warp waits for --
+// was several times the average.
+__device__ __forceinline__ uint32_t work_stride(const WorkRef& w, uint32_t h) {
+    return (uint32_t)(w.strides >> (8 * stride_index(h))) & 0xFFu;
+}
 __device__ __forceinline__ double roofline_time(const WorkRef& w, const atrex_hw_peaks_t& pk, ull key) {
     const double qnan = __longlong_as_double(0x7FF8000000000000ll);
     if (w.table == nullptr) return qnan;
@@ -95,6 +101,7 @@ __device__ __forceinline__ double roofline_time(const WorkRef& w, const atrex_hw
     const uint32_t h = hash32(pair);
     const WorkSlot* part = w.table + (ull)part_of(h, w.lp) * w.Cw;
     uint32_t s = local_of(h, 0u, w.Cw);
+    const uint32_t advance = work_stride(w, h);
     for (uint32_t probe = 0; probe < w.Cw; ++probe) {
         const WorkSlot* e = part + s;
         ull k = e->skey;
@@ -104,7 +111,8 @@ __device__ __forceinline__ double roofline_time(const WorkRef& w, const atrex_hw
             return fmax(t_compute, t_memory);
         }
         if (k == 0) break;
-        s = (s + 1 == w.Cw) ? 0u : s + 1;
+        s += advance;
+        if (s >= w.Cw) s -= w.Cw;
     }
     return qnan;
 }
@@ -206,6 +214,7 @@ __global__ void __launch_bounds__(256) work_insert_kernel(const atrex_work_t* ro
         const uint32_t h = hash32(pair);
         WorkSlot* part = w.table + (ull)part_of(h, w.lp) * w.Cw;
         uint32_t s = local_of(h, 0u, w.Cw);
+        const uint32_t advance = work_stride(w, h);
         bool done = false;
         for (uint32_t probe = 0; probe < w.Cw && !done; ++probe) {
             WorkSlot* e = part + s;
@@ -219,7 +228,8 @@ __global__ void __launch_bounds__(256) work_insert_kernel(const atrex_work_t* ro
                 atomicOr(&ctl->work_status, ST_WORK_DUP);
                 done = true;
             } else {
-                s = (s + 1 == w.Cw) ? 0u : s + 1;
+                s += advance;
+                if (s >= w.Cw) s -= w.Cw;
             }
         }
         if (!done) atomicOr(&ctl->work_status, ST_WORK_FULL);

@@ -84,6 +84,7 @@ struct WorkRef {
     WorkSlot* table;     // [P * Cw], nullptr when no work table was provisioned
     uint32_t lp;         // log2(P), same partitioning as the key table
     uint32_t Cw;         // slots per partition
+    ull strides;         // eight probe strides, one byte each: odd primes that do not divide Cw (double hashing)
 };
 
 struct FinalizeParams {
