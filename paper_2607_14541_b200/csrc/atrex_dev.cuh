@@ -133,8 +133,6 @@ __device__ __forceinline__ ull key_of_ckey(ull ckey) {
 // The two words of a spill entry (12 bytes): a = product (48 bits) | operator << 48,
 // b = phase << 24 | the hash bits below the partition's log2 P (at most 24: there are at least 2^8 partitions).
 constexpr uint32_t SPILL_ENTRY_BYTES = 12;
-__device__ __forceinline__ ull spill_word_a(ull prod, uint32_t op) { return prod | ((ull)op << 48); }
-__device__ __forceinline__ uint32_t spill_word_b(uint32_t phase, uint32_t h, uint32_t lp) { return (phase << 24) | (h & (0xFFFFFFFFu >> lp)); }
 __device__ __forceinline__ ull ckey_of_spill(ull a, uint32_t b, uint32_t part, uint32_t lp) {
     return ckey_of(((b >> 24) << 16) | (uint32_t)(a >> 48), (part << (32 - lp)) | (b & (0xFFFFFFFFu >> lp)));
 }

@@ -166,11 +166,15 @@ __device__ __forceinline__ void spill_append(const IngestParams& p, Ctx& c, bool
         // line, that line is pulled into L2 (a partial store into a line that is not cached stalls on a
         // fill), and the stores ask the L2 to evict their lines last: a buffer's current line is
         // written to some 20 times over ~40 K cycles while 16 GiB of records stream through the same cache.
-        unsigned char* at = c.my_spill + ((size_t)part * p.cap + ATREX_INDEX(tk, p.cap, p.t.ctl)) * SPILL_ENTRY_BYTES;
-        const uint32_t odd = tk & 1u;
-        stg_u64(at + odd * 4u, spill_word_a(prod, khi & 0xFFFFu), c.keep);
-        stg_u32(at + 8u - odd * 8u, spill_word_b(khi >> 16, h, LP), c.keep);
-        if (((tk * SPILL_ENTRY_BYTES) & 127u) - 96u < 12u) asm volatile("prefetch.global.L2 [%0];" ::"l"(at + 64));
+        // (a CTA's buffers together stay below 4 GB: 2^12 partitions x 2^15 entries x 12 bytes)
+        const uint32_t off = (part * p.cap + ATREX_INDEX(tk, p.cap, p.t.ctl)) * SPILL_ENTRY_BYTES;
+        const uint32_t odd4 = (tk << 2) & 4u;
+        // word a = product | operator << 48, word b = phase << 24 | low hash bits, put together bytewise
+        const uint32_t a_hi = __byte_perm((uint32_t)(prod >> 32), khi, 0x5410);
+        const uint32_t b = __byte_perm(h & (0xFFFFFFFFu >> LP), khi, 0x6210);
+        stg_u64(c.my_spill + (off + odd4), ((ull)a_hi << 32) | (uint32_t)prod, c.keep);
+        stg_u32(c.my_spill + (off + 8u - 2u * odd4), b, c.keep);
+        if ((off & 127u) - 96u < 12u) asm volatile("prefetch.global.L2 [%0];" ::"l"(c.my_spill + (off + 64u)));
     } else {
         spill_overflow<LP>(p.t, cw, ((ull)khi << 32) | shape, prod, h);
         count_one(&p.t.ctl->n_overflow);
