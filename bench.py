@@ -33,10 +33,10 @@ METRIC = "trace records aggregated/sec"
 # DRAM bytes (read + written) per 2^27-record ingest call of this workload, from the one-kernel ncu
 # captures of the 2^25-record case summarised under profiles/ (traffic grows in proportion to the
 # records of a launch, so refresh this constant from the small case, never from a full-size capture):
-# scatter_kernel 4 x 1.1426 GB per 2^27-record launch, plus the two drains inside a step's eight calls
-# (557 M spilled entries x 16 B read, and per drain 1.2 GB of table reads and write-backs) spread over
-# the eight calls.
-NCU_DRAM_BYTES_PER_INGEST_CALL = 4 * 1.1426e9 + (557e6 * 16 + 2 * 1.2e9) / 8
+# scatter_kernel 4 x 0.9895 GB per 2^27-record launch, plus the two drains inside a step's eight calls
+# (557 M spilled 12-byte entries at 14.8 B of traffic each -- queued entries and prefetched lines are
+# read twice -- and per drain 1.0 GB of table reads and write-backs) spread over the eight calls.
+NCU_DRAM_BYTES_PER_INGEST_CALL = 4 * 0.9895e9 + (557e6 * 14.8 + 2 * 1.0e9) / 8
 UNIT = "records/s"
 WORKLOAD_INDEX = 3
 RECORD_BYTES = 16
@@ -329,7 +329,7 @@ def run_ours(args):
 # DRAM bytes moved per record by the ingest pass (scatter launches + the drains they trigger), from
 # one-kernel ncu captures of 2^25..2^27-record cases summarised under profiles/ (traffic grows in
 # proportion to the records of a launch); None where no capture was taken.
-NCU_DRAM_BYTES_PER_RECORD = {0: 18.1, 1: 24.4, 2: 56.5, 3: NCU_DRAM_BYTES_PER_INGEST_CALL / float(1 << 27), 4: 21.4}
+NCU_DRAM_BYTES_PER_RECORD = {0: 17.8, 1: 21.5, 2: 46.8, 3: NCU_DRAM_BYTES_PER_INGEST_CALL / float(1 << 27), 4: 19.9}
 
 
 def per_config(torch, p, records3, n3, peak):

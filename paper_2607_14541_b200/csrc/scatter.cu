@@ -80,13 +80,6 @@ __device__ __forceinline__ uint32_t atoms_exch(uint32_t a, uint32_t v) {
     asm volatile("atom.shared.exch.b32 %0, [%1], %2;" : "=r"(o) : "r"(a), "r"(v) : "memory");
     return o;
 }
-__device__ __forceinline__ void stg_u64(void* at, ull v, ull policy) {
-    asm volatile("st.global.L2::cache_hint.u64 [%0], %1, %2;" ::"l"(at), "l"(v), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void stg_u32(void* at, uint32_t v, ull policy) {
-    asm volatile("st.global.L2::cache_hint.u32 [%0], %1, %2;" ::"l"(at), "r"(v), "l"(policy) : "memory");
-}
-
 // What the hot loop keeps in registers (everything else is read from the kernel's parameter block,
 // i.e. straight from the constant bank).
 struct Ctx {
@@ -168,13 +161,22 @@ __device__ __forceinline__ void spill_append(const IngestParams& p, Ctx& c, bool
         // written to some 20 times over ~40 K cycles while 16 GiB of records stream through the same cache.
         // (a CTA's buffers together stay below 4 GB: 2^12 partitions x 2^15 entries x 12 bytes)
         const uint32_t off = (part * p.cap + ATREX_INDEX(tk, p.cap, p.t.ctl)) * SPILL_ENTRY_BYTES;
-        const uint32_t odd4 = (tk << 2) & 4u;
+        const uint32_t odd = tk & 1u;
         // word a = product | operator << 48, word b = phase << 24 | low hash bits, put together bytewise
         const uint32_t a_hi = __byte_perm((uint32_t)(prod >> 32), khi, 0x5410);
         const uint32_t b = __byte_perm(h & (0xFFFFFFFFu >> LP), khi, 0x6210);
-        stg_u64(c.my_spill + (off + odd4), ((ull)a_hi << 32) | (uint32_t)prod, c.keep);
-        stg_u32(c.my_spill + (off + 8u - 2u * odd4), b, c.keep);
-        if ((off & 127u) - 96u < 12u) asm volatile("prefetch.global.L2 [%0];" ::"l"(c.my_spill + (off + 64u)));
+        {   // one address: the entry's parity picks between two pairs of stores at immediate offsets (the
+            // 8-byte word goes to the 8-byte aligned end), which is cheaper than computing two addresses
+            unsigned char* at = c.my_spill + off;
+            asm volatile(
+                "{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %5, 0;\n\t"
+                "@q  st.global.L2::cache_hint.u32 [%0], %3, %4;\n\t"
+                "@q  st.global.L2::cache_hint.v2.u32 [%0+4], {%1, %2}, %4;\n\t"
+                "@!q st.global.L2::cache_hint.v2.u32 [%0], {%1, %2}, %4;\n\t"
+                "@!q st.global.L2::cache_hint.u32 [%0+8], %3, %4;\n\t}"
+                ::"l"(at), "r"((uint32_t)prod), "r"(a_hi), "r"(b), "l"(c.keep), "r"(odd) : "memory");
+            if ((off & 127u) - 96u < 12u) asm volatile("prefetch.global.L2 [%0+64];" ::"l"(at));
+        }
     } else {
         spill_overflow<LP>(p.t, cw, ((ull)khi << 32) | shape, prod, h);
         count_one(&p.t.ctl->n_overflow);
