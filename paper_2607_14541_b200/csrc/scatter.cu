@@ -200,7 +200,7 @@ __device__ __forceinline__ void one_record(const IngestParams& p, Ctx& c, uint32
     const uint32_t h = hash32(khi & 0xFFFFu, w2);
     const ull key = ((ull)khi << 32) | w2;
     bool todo = ok;
-    // The limb arithmetic and the 16-byte spill entries assume products below 2^48 (e.g. weights
+    // The limb arithmetic and the 12-byte spill entries assume products below 2^48 (e.g. weights
     // < 2^20, durations < 2^28).  Anything larger is still exact: straight to the table.
     if (ok && (uint32_t)(prod >> 32) >= 0x10000u) {
         table_route(p.t, key, h, prod);
@@ -291,7 +291,7 @@ __device__ __forceinline__ void process(const IngestParams& p, Ctx& c, const uin
 #pragma unroll
     for (int r = 0; r < R; ++r) {
         const ull key = ((ull)khi[r] << 32) | w[r][2];
-        // The limb arithmetic and the 16-byte spill entries assume products below 2^48 (e.g. weights
+        // The limb arithmetic and the 12-byte spill entries assume products below 2^48 (e.g. weights
         // < 2^20, durations < 2^28).  Anything larger is still exact: straight to the table.
         if (todo[r] && (uint32_t)(prod[r] >> 32) >= 0x10000u) {
             table_route(p.t, key, h[r], prod[r]);
