@@ -10,7 +10,7 @@ LIB = os.path.join(_HERE, "libatrex_agg.so")
 SOURCES = ["api.cu", "scatter.cu", "ingest.cu", "finalize.cu", "static_topk.cu", "score.cu", "eq3.cu", "release.cu", "exchange.cu"]
 HEADERS = ["atrex_dev.cuh", "kernels.h", os.path.join("..", "..", "include", "atrex_agg.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-              "-fmad=false", "-shared", "-Xcompiler", "-fPIC"]
+              "-fmad=false", "-shared", "-Xcompiler", "-fPIC", "-ldl"]
 
 
 def _stale(target: str, deps) -> bool:

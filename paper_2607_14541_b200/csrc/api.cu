@@ -6,6 +6,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "kernels.h"
 
 using namespace atrex;
@@ -25,6 +27,15 @@ constexpr size_t HOT_SCRATCH_BYTES = SKETCH_BYTES + ((size_t)12 << CAND_BITS);
 constexpr uint32_t SEL_CAP = ATREX_MAX_TOPK + TOPK_CAND_CAP;
 
 size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// A named range around each entry point's host work, for timelines taken with a tracing tool (the
+// header-only NVTX: a no-op costing one pointer check when no tool is attached).
+struct TraceRange {
+    explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+    ~TraceRange() { nvtxRangePop(); }
+    TraceRange(const TraceRange&) = delete;
+    TraceRange& operator=(const TraceRange&) = delete;
+};
 
 ull pow2_at_least(ull x) {
     ull p = 1;
@@ -347,6 +358,7 @@ void atrex_agg_destroy(atrex_agg_t* h) {
 }
 
 int atrex_agg_reset(atrex_agg_t* h, void* stream) {
+    TraceRange range("atrex_agg_reset");
     if (!h) return ATREX_ERR_INVALID;
     DeviceGuard guard(h->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
@@ -363,6 +375,7 @@ int atrex_agg_reset(atrex_agg_t* h, void* stream) {
 }
 
 int atrex_agg_set_work_table(atrex_agg_t* h, const atrex_work_t* rows, uint64_t n, void* stream) {
+    TraceRange range("atrex_agg_set_work_table");
     if (!h || (n && !rows) || n > h->cfg.max_work_rows) return ATREX_ERR_INVALID;
     DeviceGuard guard(h->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
@@ -477,6 +490,7 @@ static int ingest_launch(atrex_agg* h, const atrex_record_t* recs, uint64_t n, c
 }
 
 int atrex_agg_ingest(atrex_agg_t* h, const atrex_record_t* d_records, uint64_t n, void* stream) {
+    TraceRange range("atrex_agg_ingest");
     if (!h) return ATREX_ERR_INVALID;
     if (n == 0) return ATREX_OK;
     if (!d_records || ((uintptr_t)d_records & 15u) != 0) return ATREX_ERR_INVALID;
@@ -494,6 +508,7 @@ int atrex_agg_ingest(atrex_agg_t* h, const atrex_record_t* d_records, uint64_t n
 }
 
 int atrex_agg_ingest_host(atrex_agg_t* h, const atrex_record_t* h_records, uint64_t n, void* stream) {
+    TraceRange range("atrex_agg_ingest_host");
     if (!h) return ATREX_ERR_INVALID;
     if (n == 0) return ATREX_OK;
     if (!h_records) return ATREX_ERR_INVALID;
@@ -518,6 +533,7 @@ int atrex_agg_ingest_host(atrex_agg_t* h, const atrex_record_t* h_records, uint6
 }
 
 int atrex_agg_merge(atrex_agg_t* h, const atrex_entry_t* d_entries, uint64_t n, void* stream) {
+    TraceRange range("atrex_agg_merge");
     if (!h) return ATREX_ERR_INVALID;
     if (n == 0) return ATREX_OK;
     if (!d_entries || ((uintptr_t)d_entries & 15u) != 0) return ATREX_ERR_INVALID;
@@ -567,6 +583,7 @@ int atrex_agg_finalize_with_totals(atrex_agg_t* h, const atrex_hw_peaks_t* peaks
 static int finalize_impl(atrex_agg_t* h, const atrex_hw_peaks_t* peaks, const uint64_t* total_lo,
                          const uint64_t* total_hi, atrex_entry_t* d_out, uint64_t out_cap, uint64_t* n_out,
                          void* stream) {
+    TraceRange range("atrex_agg_finalize");
     if (!h || !peaks || !n_out) return ATREX_ERR_INVALID;
     if (d_out && ((uintptr_t)d_out & 15u) != 0) return ATREX_ERR_INVALID;
     if (!d_out) out_cap = 0;
@@ -652,6 +669,7 @@ static int plan_phase(atrex_agg_t* h, uint32_t q, uint32_t k, TopkAllParams* all
 }
 
 int atrex_agg_topk(atrex_agg_t* h, uint32_t phase, uint32_t k, atrex_entry_t* h_out, uint32_t* n_out, void* stream) {
+    TraceRange range("atrex_agg_topk");
     if (!h || !n_out || (k && !h_out) || k > ATREX_MAX_TOPK || phase >= h->cfg.n_phases) return ATREX_ERR_INVALID;
     *n_out = 0;
     if (!h->finalized) return ATREX_ERR_STATE;
@@ -734,6 +752,7 @@ int atrex_agg_totals(const atrex_agg_t* h, uint64_t* h_lo, uint64_t* h_hi) {
 }
 
 int atrex_agg_stats(atrex_agg_t* h, atrex_stats_t* out, void* stream) {
+    TraceRange range("atrex_agg_stats");
     if (!h || !out) return ATREX_ERR_INVALID;
     DeviceGuard guard(h->cfg.device);
     cudaStream_t s = (cudaStream_t)stream;
