@@ -112,6 +112,13 @@ __device__ __noinline__ void drain_slot(TableRef t, uint32_t acc, ull key, uint3
 
 // (rare) A record that cannot take the limb route: straight to the table with full 64-bit adds.
 __device__ __noinline__ void table_route(TableRef t, ull key, uint32_t h, ull prod) { table_accumulate(t, key, h, prod, 0, 1); }
+// (rare) An invalid record is counted; a valid one whose product has bits at or above 2^48 goes to the table.
+__device__ __noinline__ void rare_record(TableRef t, bool valid, ull key, uint32_t h, ull prod) {
+    if (valid)
+        table_accumulate(t, key, h, prod, 0, 1);
+    else
+        atomicAdd(&t.ctl->n_rejected, 1ull);
+}
 
 // Add (count, v) to a directory slot, v < 2^53, count <= 32.  Most products fit 32 bits and most
 // low-limb adds do not wrap: the high limb is then left alone (one returning atomic and one reduction
@@ -135,6 +142,7 @@ template <uint32_t LP>
 __device__ __noinline__ void spill_overflow(TableRef t, uint32_t cw, ull key, ull prod, uint32_t h) {
     reds_add(cw, 0xFFFFFFFFu);
     table_accumulate(t, key, h, prod, 0, 1);
+    atomicAdd(&t.ctl->n_overflow, 1ull);
 }
 
 // Spill: the record becomes a 12-byte entry in this CTA's buffer of the key's partition -- an 8-byte
@@ -179,7 +187,6 @@ __device__ __forceinline__ void spill_append(const IngestParams& p, Ctx& c, bool
         }
     } else {
         spill_overflow<LP>(p.t, cw, ((ull)khi << 32) | shape, prod, h);
-        count_one(&p.t.ctl->n_overflow);
     }
 }
 
@@ -192,20 +199,19 @@ __device__ __forceinline__ void one_record(const IngestParams& p, Ctx& c, uint32
     const uint32_t khi = w1 & 0x00FFFFFFu;                  // phase << 16 | op_id: the key's high word
     bool ok = w0 < p.n_apps && khi < p.phase_lim;
     if (!FULL) ok = ok && present;
-    if ((FULL || present) && !ok) count_one(&p.t.ctl->n_rejected);
     // card-hour weight: from shared memory when the table fits there (an out-of-range index reads
     // some other weight, which is not used), else from global memory
     const uint32_t wgt = (p.appw_in_smem != 0) ? lds_u32(c.sb + L::APPW + (w0 & (APPW_SMEM_MAX - 1u)) * 4u) : __ldg(p.app_w + (ok ? w0 : 0u));
     const ull prod = (ull)wgt * (ull)w3;
     const uint32_t h = hash32(khi & 0xFFFFu, w2);
     const ull key = ((ull)khi << 32) | w2;
-    bool todo = ok;
     // The limb arithmetic and the 12-byte spill entries assume products below 2^48 (e.g. weights
-    // < 2^20, durations < 2^28).  Anything larger is still exact: straight to the table.
-    if (ok && (uint32_t)(prod >> 32) >= 0x10000u) {
-        table_route(p.t, key, h, prod);
-        todo = false;
-    }
+    // < 2^20, durations < 2^28).  Anything larger is still exact: straight to the table.  That and
+    // the count of invalid records share one rarely taken branch (two separate ones cost the
+    // configurations whose records mostly hit the directory 4-9 %).
+    const bool todo_in = ok && (uint32_t)(prod >> 32) < 0x10000u;
+    bool todo = todo_in;
+    if ((FULL || present) && !todo_in) rare_record(p.t, ok, key, h, prod);
     if (HOT) {
         // Directory look-up: one 32-bit word per 4-slot bucket holds an 8-bit tag per slot (hash bits
         // the bucket choice does not use); the lowest slot whose tag matches is confirmed against the
