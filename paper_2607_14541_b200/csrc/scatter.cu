@@ -146,14 +146,9 @@ __device__ __noinline__ void spill_overflow(TableRef t, uint32_t cw, ull key, ul
 }
 
 // Spill: the record becomes a 12-byte entry in this CTA's buffer of the key's partition -- an 8-byte
-// word {product (48 bits), operator} and a 4-byte word {phase, the hash bits below the partition's},
-// kept as two arrays per buffer.  Inside its partition (the hash's top bits) the pair (phase,
-// operator, hash) identifies the key: for a given operator the hash is a bijection of the shape
-// (shape_of_hash).  Each word is stored on its own; two entries before a buffer's 8-byte array reaches
-// its next 128-byte line (and likewise for the 4-byte array) that line is pulled into L2 -- a partial
-// store into a line that is not cached stalls on a fill -- and the stores ask the L2 to evict their
-// lines last: a buffer's current lines are written to 16 and 32 times over tens of thousands of cycles
-// while 16 GiB of records stream through the same cache.
+// word {product (48 bits), operator} and a 4-byte word {phase, the hash bits below the partition's}.
+// Inside its partition (the hash's top bits) the triple (phase, operator, hash) identifies the key:
+// for a given operator the hash is a bijection of the shape (shape_of_hash).
 template <uint32_t LP>
 __device__ __forceinline__ void spill_append(const IngestParams& p, Ctx& c, bool todo, uint32_t khi, uint32_t shape, ull prod,
                                              uint32_t h) {
