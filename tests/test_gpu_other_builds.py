@@ -24,7 +24,7 @@ def test_parity_cases_under_the_bounds_checked_build():
                            cwd=ROOT, env=env, capture_output=True, text=True, timeout=300)
     assert probe.returncode == 0 and probe.stdout.strip() == "1", probe.stderr[-2000:]
     run = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "-x", "-q", "-k",
-                          "five_configs or misaligned or carry or invalid_records or full_u32 or largest_geometry or crowded or exactly_to_max_keys or merge_of_partial"],
+                          "five_configs or misaligned or carry or invalid_records or full_u32 or largest_geometry or crowded or exactly_to_max_keys or merge_of_partial or every_partition_count"],
                          cwd=ROOT, env=env, capture_output=True, text=True, timeout=1200)
     assert run.returncode == 0, run.stdout[-3000:] + run.stderr[-2000:]
     assert " passed" in run.stdout

@@ -425,3 +425,39 @@ def test_table_filled_exactly_to_max_keys(lib, max_keys):
     assert n_keys == 2 * len(pairs) and max_keys - 1 <= n_keys <= max_keys
     agg = gpu_aggregate(lib, recs, weights, 2, max_keys=n_keys)
     assert_same_as_oracle(agg, o, 2)
+
+
+@pytest.mark.parametrize("max_keys,partitions", [(2_000_000, 256), (4_000_000, 512), (9_000_000, 1024), (18_000_000, 2048),
+                                                 (1 << 25, 4096)])
+@pytest.mark.parametrize("hot", [True, False])
+def test_every_partition_count_with_full_range_keys(lib, max_keys, partitions, hot):
+    """A spill entry carries (phase, operator, hash bits below the partition's) instead of the key, and
+    the partition pass recovers a new key's shape by inverting the hash: every partition count the
+    library can choose (2^8 .. 2^12, i.e. 24 .. 20 stored hash bits), operators over all 16 bits, shapes
+    over all 32, eight phases, and two drains, so that keys written back by the first are found again
+    by the second."""
+    rng = np.random.default_rng(partitions + (1 if hot else 0))
+    n = 600_011
+    recs = np.zeros(n, dtype=RECORD_DTYPE)
+    pool_op = rng.integers(0, 1 << 16, size=200_000).astype(np.uint16)
+    pool_shape = rng.integers(0, 1 << 32, size=200_000, dtype=np.uint64).astype(np.uint32)
+    pool_shape[:64] = np.array([0, 1, 0xFFFFFFFF, 0x80000000] * 16, dtype=np.uint32)   # the corners too
+    pick = rng.integers(0, 200_000, size=n)
+    pick[: n // 4] = rng.integers(0, 500, size=n // 4)            # a few keys frequent enough for the directory
+    recs["op_id"], recs["shape_id"] = pool_op[pick], pool_shape[pick]
+    recs["phase"] = rng.integers(0, 8, size=n)
+    recs["app_id"] = rng.integers(0, 16, size=n)
+    recs["duration_ns"] = rng.integers(0, 1 << 28, size=n)
+    rng.shuffle(recs)
+    weights = rng.integers(1, 1 << 20, size=16).astype(np.uint32)
+    o = oracle_of(recs, weights, 8)
+    agg = lib.Aggregator(weights, 8, max_keys, flags=0 if hot else lib.ATREX_FLAG_NO_HOT_DIRECTORY)
+    half = n // 2
+    agg.ingest(to_dev(recs[:half]), n=half)
+    first = agg.stats()                                            # forces the first drain
+    assert first["table_slots"] % partitions == 0 and first["table_slots"] // partitions <= 11520
+    assert first["table_slots"] // partitions >= 8192 or partitions == 256
+    agg.ingest(to_dev(recs[half:]), n=n - half)
+    assert_same_as_oracle(agg, o, 8, ks=(5,))
+    st = agg.stats()
+    assert st["n_spilled"] > n // 2 and st["n_drains"] >= 2 and st["n_overflow"] == 0
