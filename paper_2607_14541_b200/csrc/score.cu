@@ -8,9 +8,10 @@
 //   Eq. 6  S_agg = sum_i w_i S_i, accumulated in operator order
 //
 // Every floating-point step is one explicit round-to-nearest operation in a fixed order, so
-// the result has one bit pattern.  The median is found by ranking (each value's rank is the
-// number of values that sort before it, ties broken by position), which needs no sorting
-// network and no scratch memory beyond the CTA's shared memory.
+// the result has one bit pattern.  The median of a small group is found by ranking (each value's
+// rank is the number of values that sort before it, ties broken by position), that of a large one
+// by a bitwise search for the wanted order statistics; neither needs a sorting network or scratch
+// memory beyond the CTA's shared memory.
 #include <mutex>
 
 #include "kernels.h"
@@ -20,6 +21,28 @@ using namespace atrex;
 namespace {
 
 constexpr int SCORE_THREADS = 256;
+
+// Order statistics of a large group.  A double's bit pattern, with the sign bit flipped for positive
+// values and all bits flipped for negative ones, orders like the value; the k-th smallest key (k from
+// 0) is the largest v with #{key < v} <= k, found one bit at a time.  Called by a whole warp; every
+// lane returns the value.
+constexpr uint32_t SELECT_ABOVE = 128;   // below this, ranking every value against every other is cheaper
+__device__ __forceinline__ unsigned long long order_key(double x) {
+    const unsigned long long b = (unsigned long long)__double_as_longlong(x);
+    return b ^ ((b >> 63) ? ~0ull : (1ull << 63));
+}
+__device__ __forceinline__ double select_kth(const double* v, uint32_t m, uint32_t k, uint32_t lane) {
+    unsigned long long ans = 0;
+    for (int bit = 63; bit >= 0; --bit) {
+        const unsigned long long trial = ans | (1ull << bit);
+        uint32_t below = 0;
+        for (uint32_t a = lane; a < m; a += 32) below += order_key(v[a]) < trial ? 1u : 0u;
+        below = __reduce_add_sync(0xFFFFFFFFu, below);
+        if (below <= k) ans = trial;
+    }
+    const unsigned long long b = ans ^ ((ans >> 63) ? (1ull << 63) : ~0ull);
+    return __longlong_as_double((long long)b);
+}
 
 __global__ void __launch_bounds__(SCORE_THREADS) score_kernel(const double* __restrict__ roofline_s,
                                                               const uint32_t* __restrict__ unit_op, uint32_t n_units,
@@ -83,6 +106,14 @@ __global__ void __launch_bounds__(SCORE_THREADS) score_kernel(const double* __re
         }
         const uint32_t want_hi = m / 2, want_lo = (m & 1u) ? m / 2 : m / 2 - 1;
         double v_hi = 0.0, v_lo = 0.0;
+        if (m > SELECT_ABOVE) {
+            // a large group: the wanted order statistics by a bitwise search over order-preserving keys
+            // (64 counting passes over the group instead of m)
+            const double hi = select_kth(s_val + lo, m, want_hi, lane);
+            const double lw = (m & 1u) ? hi : select_kth(s_val + lo, m, want_lo, lane);
+            if (lane == 0) s_med[op] = (m & 1u) ? hi : __dmul_rn(__dadd_rn(lw, hi), 0.5);
+            continue;
+        }
         for (uint32_t a = lane; a < m; a += 32) {
             const double x = s_val[lo + a];
             uint32_t rank = 0;
