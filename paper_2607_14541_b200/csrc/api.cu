@@ -93,11 +93,12 @@ void compute_layout(const atrex_agg_config_t* c, size_t smem_optin, int n_sms, L
     if (per_buf < 64) per_buf = 64;
     if (per_buf > 32768) per_buf = 32768;   // the scatter pass counts a buffer's entries in 16 bits, with headroom
     L->cap = (uint32_t)((per_buf + 31) / 32 * 32);   // a buffer is a whole number of 128-byte lines
-    // entries of one partition whose first look fails wait in a per-CTA queue: room for a quarter of
-    // the partition's worst-case stream, at most 32 K entries (the rest is settled in line)
+    // entries of one partition whose first look fails wait in a per-CTA queue, one segment per warp:
+    // room for a quarter of the partition's worst-case stream, at most 32 K entries (a warp whose
+    // segment could not take another batch of 128 settles it first), at least two batches per warp
     {
         ull q = (ull)L->cap * n_sms / 4;
-        L->queue_cap = (uint32_t)(q < 1024 ? 1024 : (q > 32768 ? 32768 : q));
+        L->queue_cap = (uint32_t)(q < 8192 ? 8192 : (q > 32768 ? 32768 : q));
     }
     // work table: same partitions as the key table, 1.5 slots per row plus slack for uneven partitions
     L->Cw = c->max_work_rows ? (uint32_t)((((c->max_work_rows * 3 / 2) >> L->lp) + 64 + 31) / 32 * 32) : 0;

@@ -130,10 +130,11 @@ __global__ void __launch_bounds__(FOLD_WARPS * 32) hot_fold_kernel(const ull* ho
 // persistent and take partitions blockIdx.x, blockIdx.x + gridDim.x, ...; while one partition
 // is processed, the next one's keys and spill entries are pulled into L2.  Per partition: copy the
 // keys in, each in the pass's own 64-bit form (phase, operator, 32-bit hash: unique inside a
-// partition, and what a spill entry carries); stream the entries of all scatter CTAs, four per lane, and settle each with one look at
-// the first pair of its probe sequence (hit, or a new key with room there); entries that need more
-// than that wait in the warp's segment of a per-CTA queue in global memory and are settled, 32 per
-// round, once the warp's share of the stream is through; then write the deltas back.
+// partition, and what a spill entry carries); stream the entries of all scatter CTAs, four per lane,
+// and settle each with one look at the first pair of its probe sequence (hit, or a new key with room
+// there); entries that need more than that wait in the warp's segment of a per-CTA queue in global
+// memory and are settled, 32 per round, once the warp's share of the stream is through (or earlier,
+// when the segment could not take another batch); then write the deltas back.
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 // Shared-window addresses of the partition pass's arrays: keys ull[C] (the pass's own key form, 0 =
@@ -218,6 +219,13 @@ __device__ __forceinline__ void prefetch_entries(const PartitionParams& q, ull s
     if (lane < 24 && lane * 128u < bytes) prefetch_l2(q.spill + sb * q.cap * SPILL_ENTRY_BYTES + lane * 128u);
 }
 
+// Settles a warp's queued entries, one per lane and round, by the general probe.  Other warps may
+// still be streaming: the probe copes with keys that appear meanwhile.  Called once the warp's share of
+// the partition's stream is through, and before a batch that might not fit the queue (a crowded
+// partition of new keys).  Not inlined: it runs a few times per partition and warp.
+__device__ __noinline__ void settle_queue(const TableRef t, const PartSmem m, const ulonglong2* my_queue, uint32_t qn_w, uint32_t C,
+                                          ull base, uint32_t lane);
+
 // A queued entry: {key, product}; bit 63 of the product word says that the key's first pair was full
 // of other keys when the entry was looked up, so its probe may start at the second pair.
 constexpr ull QUEUED_SKIP_FIRST = 1ull << 63;
@@ -230,8 +238,7 @@ constexpr ull QUEUED_SKIP_FIRST = 1ull << 63;
 template <bool FULL>
 __device__ __forceinline__ void stream_batch(const PartitionParams& q, const PartSmem& m, const unsigned char* src,
                                              uint32_t part_bits, uint32_t hmask, uint32_t e0, uint32_t n_e, uint32_t C, ull base,
-                                             ulonglong2* my_queue, uint32_t queue_cap_w, uint32_t& qn_w, unsigned char* s_owner_w,
-                                             uint32_t lane) {
+                                             ulonglong2* my_queue, uint32_t queue_cap_w, uint32_t& qn_w, uint32_t lane) {
     uint32_t kh[4], kl[4], vlo[4], vhi[4], slot[4];
     uint32_t open = 0;
     {
@@ -296,75 +303,48 @@ __device__ __forceinline__ void stream_batch(const PartitionParams& q, const Par
     if (__any_sync(0xFFFFFFFFu, open != 0)) {
         // The rest (keys further down their probe sequence, lost races: a few per batch) is not settled
         // here, where the fixed cost of a general probe round would be paid for a handful of entries: it
-        // goes to this warp's queue and is settled after the partition's stream, 32 entries per warp round.
-        uint32_t pend[4], before[4], total = 0;
+        // goes to this warp's queue and is settled by settle_queue, 32 entries per warp round.
+        uint32_t before[4], total = 0;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            pend[u] = __ballot_sync(0xFFFFFFFFu, (open >> u) & 1u);
-            before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
-            total += __popc(pend[u]);
+            const uint32_t pend = __ballot_sync(0xFFFFFFFFu, (open >> u) & 1u);
+            before[u] = total + __popc(pend & ((1u << lane) - 1u));
+            total += __popc(pend);
         }
-        uint32_t qbase = qn_w;
-        qn_w = min(qn_w + total, queue_cap_w);
+        // (the caller settles the queue before a batch that might not fit: there is room for all 128)
+        const uint32_t qbase = qn_w;
+        qn_w += total;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            if ((open & (1u << u)) && qbase + before[u] < queue_cap_w) {
+            if (open & (1u << u)) {
                 const ull v = vlo[u] | ((ull)vhi[u] << 32) | ((room >> u) & 1u ? 0ull : QUEUED_SKIP_FIRST);
                 my_queue[ATREX_INDEX(qbase + before[u], queue_cap_w, q.t.ctl)] = make_ulonglong2(((ull)kh[u] << 32) | kl[u], v);
-                open &= ~(1u << u);
             }
-        }
-        // Queue full (a partition made of new keys only): settle the remainder in line.  The pending
-        // entries are handed out one per lane: each one's owner publishes (round, lane) at the entry's
-        // position; lane t serves position t.
-        while (qbase + total > queue_cap_w) {
-            total = 0;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                pend[u] = __ballot_sync(0xFFFFFFFFu, (open >> u) & 1u);
-                before[u] = total + __popc(pend[u] & ((1u << lane) - 1u));
-                total += __popc(pend[u]);
-            }
-            if (total == 0) break;
-            qbase = queue_cap_w;  // stay in this loop until nothing is pending
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if ((open & (1u << u)) && before[u] < 32) s_owner_w[before[u]] = (unsigned char)((u << 5) | lane);
-            __syncwarp();
-            const bool serving = lane < total;
-            const uint32_t code = serving ? s_owner_w[lane] : lane;
-            const uint32_t from = code & 31u, su = code >> 5;
-            uint32_t kh_s = 0, kl_s = 0, slot_s = 0;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t h = __shfl_sync(0xFFFFFFFFu, kh[u], from);
-                const uint32_t l = __shfl_sync(0xFFFFFFFFu, kl[u], from);
-                const uint32_t sl = __shfl_sync(0xFFFFFFFFu, slot[u] & ~1u, from);
-                if (su == (uint32_t)u) {
-                    kh_s = h;
-                    kl_s = l;
-                    slot_s = sl;
-                }
-            }
-            const uint32_t found_s = probe_general(m, ((ull)kh_s << 32) | kl_s, slot_s, 2u * stride_of(q.t, stride_index(kl_s)), serving, C,
-                                                   q.t.ctl);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const uint32_t found = __shfl_sync(0xFFFFFFFFu, found_s, before[u] & 31u);
-                if ((open & (1u << u)) && before[u] < 32) {
-                    open &= ~(1u << u);
-                    if (found != PROBE_FAILED) {
-                        slot[u] = found;
-                        hit |= 1u << u;
-                    }
-                }
-            }
-            __syncwarp();  // the owner table is rewritten in the next round
         }
     }
 #pragma unroll
     for (int u = 0; u < 4; ++u)
         if (hit & (1u << u)) part_accumulate(m, slot[u], vlo[u], vhi[u], q.t.vals + base, C, q.t.ctl);
+}
+
+__device__ __noinline__ void settle_queue(const TableRef t, const PartSmem m, const ulonglong2* my_queue, uint32_t qn_w, uint32_t C,
+                                          ull base, uint32_t lane) {
+    __syncwarp();   // the queue was written by other lanes of this warp
+    for (uint32_t i0 = 0; i0 < qn_w; i0 += 32u) {
+        const bool serving = i0 + lane < qn_w;
+        const ulonglong2 ent = serving ? __ldcg(my_queue + i0 + lane) : make_ulonglong2(0, 0);
+        const uint32_t hh = (uint32_t)ent.x;
+        const uint32_t advance = 2u * stride_of(t, stride_index(hh));
+        uint32_t start = local_of(hh, ckey_phase(ent.x), C) & ~1u;
+        if (ent.y & QUEUED_SKIP_FIRST) {
+            start += advance;
+            if (start >= C) start -= C;
+        }
+        const uint32_t found = probe_general(m, ent.x, start, advance, serving, C, t.ctl);
+        if (serving && found != PROBE_FAILED)
+            part_accumulate(m, found, (uint32_t)ent.y, (uint32_t)(ent.y >> 32) & 0xFFFFu, t.vals + base, C, t.ctl);
+    }
+    __syncwarp();   // the queue may be overwritten from here on
 }
 
 __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionParams q) {
@@ -382,7 +362,6 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
     // leftovers as soon as its share of the stream is through
     const uint32_t queue_cap_w = q.queue_cap / (INGEST_THREADS / 32);
     ulonglong2* const my_queue = q.queue + (size_t)blockIdx.x * q.queue_cap + (size_t)(threadIdx.x >> 5) * queue_cap_w;
-    __shared__ unsigned char s_owner[INGEST_THREADS / 32][32];  // in-line fallback, per warp: (round, lane) owning hand-out position t
     const uint32_t n_parts = 1u << q.t.lp;
     const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31u, n_warps = blockDim.x >> 5;
     // the spill buffers are drained lazily: unless forced, only when the scatter launch just
@@ -451,30 +430,17 @@ __global__ void __launch_bounds__(INGEST_THREADS, 1) partition_kernel(PartitionP
             for (uint32_t e0 = 0; e0 < n_e; e0 += 128) {
                 if (lane < 12 && (e0 + 256u) * SPILL_ENTRY_BYTES + lane * 128u < n_e * SPILL_ENTRY_BYTES)
                     prefetch_l2(buf + (e0 + 256u) * SPILL_ENTRY_BYTES + lane * 128u);
-                if (e0 + 128u <= n_e)
-                    stream_batch<true>(q, m, buf, part_bits, hmask, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
-                else
-                    stream_batch<false>(q, m, buf, part_bits, hmask, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, s_owner[warp], lane);
-            }
-        }
-        {   // this warp's queued entries, one per lane (other warps may still be streaming: the general
-            // probe copes with keys appearing meanwhile)
-            __syncwarp();
-            for (uint32_t i0 = 0; i0 < qn_w; i0 += 32u) {
-                const bool serving = i0 + lane < qn_w;
-                const ulonglong2 ent = serving ? __ldcg(my_queue + i0 + lane) : make_ulonglong2(0, 0);
-                const uint32_t hh = (uint32_t)ent.x;
-                const uint32_t advance = 2u * stride_of(q.t, stride_index(hh));
-                uint32_t start = local_of(hh, ckey_phase(ent.x), C) & ~1u;
-                if (ent.y & QUEUED_SKIP_FIRST) {
-                    start += advance;
-                    if (start >= C) start -= C;
+                if (qn_w + 128u > queue_cap_w) {   // (warp-uniform) the next batch might not fit the queue
+                    settle_queue(q.t, m, my_queue, qn_w, C, base, lane);
+                    qn_w = 0;
                 }
-                const uint32_t found = probe_general(m, ent.x, start, advance, serving, C, q.t.ctl);
-                if (serving && found != PROBE_FAILED)
-                    part_accumulate(m, found, (uint32_t)ent.y, (uint32_t)(ent.y >> 32) & 0xFFFFu, q.t.vals + base, C, q.t.ctl);
+                if (e0 + 128u <= n_e)
+                    stream_batch<true>(q, m, buf, part_bits, hmask, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, lane);
+                else
+                    stream_batch<false>(q, m, buf, part_bits, hmask, e0, n_e, C, base, my_queue, queue_cap_w, qn_w, lane);
             }
         }
+        settle_queue(q.t, m, my_queue, qn_w, C, base, lane);
         __syncthreads();
         {   // while the deltas are written back, pull the next partition's keys and each warp's
             // first sub-buffer towards L2 (used within microseconds, so they are still there)
