@@ -184,12 +184,18 @@ def run_ours(args):
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device(f"cuda:{local}"))
     elif args.force_exchange:
         # one GPU, but the step of a multi-GPU run: a process group of one rank (exercises the exchange path)
-        import socket
-        with socket.socket() as sock:
-            sock.bind(("127.0.0.1", 0))
-            port = sock.getsockname()[1]
-        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
-                                device_id=torch.device(f"cuda:{local}"))
+        if "MASTER_PORT" in os.environ and "RANK" in os.environ:
+            # started by torch.distributed.run with one process: its store is the rendezvous (a tcp://
+            # address of our own would be taken for the agent's and never answer)
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device(f"cuda:{local}"))
+        else:
+            import socket
+            with socket.socket() as sock:
+                sock.bind(("127.0.0.1", 0))
+                port = sock.getsockname()[1]
+            dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                                    device_id=torch.device(f"cuda:{local}"))
     sharded = world > 1 or args.force_exchange
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
