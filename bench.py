@@ -225,6 +225,7 @@ def run_ours(args):
         from paper_2607_14541_b200 import distributed as D
         owner = p.Aggregator(spec.app_weights, spec.n_phases, spec.max_keys, max_work_rows=len(work), device=local)
         owner.set_work_table(work)
+        out_owner = torch.empty(spec.max_keys * 48, dtype=torch.uint8, device=dev)
 
     def step(timed: bool):
         agg.reset()
@@ -241,7 +242,7 @@ def run_ours(args):
             else:
                 agg.ingest(view, n=chunk)
         if owner is not None:
-            _, n_out = D.aggregate_sharded(agg, owner, spec.peak_bw, spec.peak_flops)
+            _, n_out = D.aggregate_sharded(agg, owner, spec.peak_bw, spec.peak_flops, out_local=out, out_owner=out_owner)
             tops = [D.global_topk(owner, phase, spec.topk) for phase in range(spec.n_phases)]
             return n_out, tops
         _, n_out = agg.finalize(spec.peak_bw, spec.peak_flops, out=out)

@@ -55,22 +55,25 @@ class Outgoing:
         return self.grouped[begin: begin + self.counts[dst] * ENTRY_BYTES]
 
 
-def prepare_outgoing(local_agg, peak_bw: float, peak_flops, world: int) -> Outgoing:
-    """Sender side: finalize this rank's partial aggregate and group its entries by owner on the device."""
-    local, n = local_agg.finalize(peak_bw, peak_flops)
+def prepare_outgoing(local_agg, peak_bw: float, peak_flops, world: int, out=None) -> Outgoing:
+    """Sender side: finalize this rank's partial aggregate and group its entries by owner on the device.
+    ``out``: an optional CUDA byte tensor with room for every key's 48-byte entry; with it the finalize
+    is one pass (without it, a counting pass sizes the output first)."""
+    local, n = local_agg.finalize(peak_bw, peak_flops, out=out)
     lo, hi = local_agg.totals_words()                 # the totals the finalize just computed: no second pass
     grouped, counts = B.bucket_entries_by_owner(local, n, world)
     return Outgoing(grouped, counts, lo, hi)
 
 
-def fold_incoming(owner_agg, received, peak_bw: float, peak_flops, totals_lo_rows, totals_hi_rows):
+def fold_incoming(owner_agg, received, peak_bw: float, peak_flops, totals_lo_rows, totals_hi_rows, out=None):
     """Owner side: fold the received entries (a CUDA byte tensor, any order) into ``owner_agg``, combine the
-    shards' totals exactly and finalize the owned keys against them.  Returns (entries, n)."""
+    shards' totals exactly and finalize the owned keys against them (into ``out`` when given).  Returns
+    (entries, n)."""
     n = received.numel() // ENTRY_BYTES
     if n:
         owner_agg.merge(received, n)
     lo, hi = B.combine_totals(totals_lo_rows, totals_hi_rows)
-    return owner_agg.finalize(peak_bw, peak_flops, global_totals=(lo, hi))
+    return owner_agg.finalize(peak_bw, peak_flops, out=out, global_totals=(lo, hi))
 
 
 # ---------------------------------------------------------------- the exchange over torch.distributed
@@ -95,14 +98,15 @@ def exchange(outgoing: Outgoing, group=None):
     return received, table[:, :B.ATREX_MAX_PHASES].copy(), table[:, B.ATREX_MAX_PHASES:].copy()
 
 
-def aggregate_sharded(local_agg, owner_agg, peak_bw: float, peak_flops, group=None):
+def aggregate_sharded(local_agg, owner_agg, peak_bw: float, peak_flops, group=None, out_local=None, out_owner=None):
     """Full multi-GPU step for one rank, after ``local_agg`` has ingested this rank's slice: group the
     local entries by owner, exchange, fold what arrives into ``owner_agg`` and finalize the owned keys
-    against the totals over all shards.  Returns (entries, n) of the keys this rank owns."""
+    against the totals over all shards.  Returns (entries, n) of the keys this rank owns.  ``out_local`` /
+    ``out_owner``: optional output buffers for the two finalize calls (one pass each instead of two)."""
     import torch.distributed as dist
-    out = prepare_outgoing(local_agg, peak_bw, peak_flops, dist.get_world_size(group))
+    out = prepare_outgoing(local_agg, peak_bw, peak_flops, dist.get_world_size(group), out=out_local)
     received, lo_rows, hi_rows = exchange(out, group)
-    return fold_incoming(owner_agg, received, peak_bw, peak_flops, lo_rows, hi_rows)
+    return fold_incoming(owner_agg, received, peak_bw, peak_flops, lo_rows, hi_rows, out=out_owner)
 
 
 def global_topk(owner_agg, phase: int, k: int, group=None):
